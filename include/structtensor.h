@@ -1,0 +1,174 @@
+/*
+ * structtensor.h -- C ABI of the structured-tensor hot path for NVIDIA B200 (sm_100a).
+ *
+ * The library executes tensor contractions only over the iteration space that is
+ * left once the sparsity structure T_U (unique set) and the redundancy structure
+ * T_R (redundancy map) of "Compiling Structured Tensor Algebra" (StructTensor,
+ * arXiv 2211.10482) are applied, and it reads and writes tensors in packed layouts
+ * that hold T_C = T * T_U contiguously (Section 4, "Compressed Tensor").
+ *
+ * Conventions for every call
+ *   - All tensor pointers are DEVICE pointers owned by the caller.  The library
+ *     never allocates, frees or keeps them.  Base pointers must be 16-byte aligned.
+ *   - Everything is row-major; extents are int64_t.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream).
+ *     Calls are asynchronous on that stream and do not synchronise, except
+ *     st_check_status.
+ *   - Outputs are overwritten, not accumulated into.
+ *   - `ws` is caller-provided scratch of at least st_workspace_bytes(...) bytes,
+ *     256-byte aligned.  It needs no initialisation.  Two calls that share one
+ *     workspace must be ordered on the same stream.
+ *   - Argument errors are found on the host and returned before anything is
+ *     launched.  There is no CPU fallback: a shape a kernel does not support
+ *     returns ST_ERR_UNSUPPORTED.
+ *
+ * Packed layouts (lexicographic order of the unique set; `inner` = length of a
+ * trailing dense mode carried by every position, 1 if there is none):
+ *   ST_TRI_UPPER  T_U(i,j) = 0<=i<=j<d (Section 4, upper-triangular example;
+ *                 Figure "structures in STUR", symmetric):
+ *                 row p(i,j) = i(2d-i+1)/2 + (j-i);  d(d+1)/2 rows.
+ *   ST_TET        T_U(i,j,k) = 0<=i<=j<=k<d (Section 2, "Tensor Structures"):
+ *                 all (j,k) of slab i follow those of slab i-1; d(d+1)(d+2)/6 rows.
+ *   ST_BAND       T_U(i,j) = i-kl<=j<=i+ku: fixed width kl+ku+1 per row, slot
+ *                 (i, j-i+kl); slots outside the matrix are written as zero bytes
+ *                 by st_pack and ignored by st_unpack.
+ *   ST_BLOCKDIAG  direct sum of nblocks square blocks of size bs (Figure
+ *                 "operations in STUR", e1 (+) e2): row (b*bs+i')*bs+j'.
+ *   The dense counterpart is [d,d,inner] (ST_TET: [d,d,d,inner]).
+ */
+#ifndef STRUCTTENSOR_H
+#define STRUCTTENSOR_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    ST_OK = 0,
+    ST_ERR_NULL = 1,         /* a required pointer is NULL */
+    ST_ERR_SHAPE = 2,        /* non-positive or inconsistent extent */
+    ST_ERR_ALIGN = 3,        /* pointer or leading dimension not aligned as required */
+    ST_ERR_DTYPE = 4,        /* element type not supported by this call */
+    ST_ERR_WORKSPACE = 5,    /* workspace missing or too small */
+    ST_ERR_UNSUPPORTED = 6,  /* well-formed request outside what the kernels cover */
+    ST_ERR_CUDA = 7,         /* a CUDA runtime / driver call failed */
+    ST_ERR_DEV_TIMEOUT = 8,  /* a bounded wait inside a kernel ran out (see st_check_status) */
+    ST_ERR_DEV_BOUNDS = 9    /* a kernel-side consistency check failed */
+} st_status;
+
+typedef enum { ST_F32 = 0, ST_BF16 = 1, ST_F64 = 2 } st_dtype;
+typedef enum { ST_TRI_UPPER = 0, ST_TET = 1, ST_BAND = 2, ST_BLOCKDIAG = 3 } st_kind;
+typedef enum { ST_FILL_ZERO = 0, ST_FILL_SYMMETRIC = 1 } st_fill;
+typedef enum { ST_OP_SYM_MOMENT2 = 0, ST_OP_SYM_MOMENT3 = 1, ST_OP_MTTKRP_TRI = 2,
+               ST_OP_TTM_BLOCKDIAG = 3 } st_op;
+
+/* flags (bit mask) */
+#define ST_FLAG_DENSE_CONTROL 1u /* run the same kernel over the dense, unstructured iteration
+                                    space (a control for measurements; see each call) */
+#define ST_FLAG_TC_TF32       2u /* st_ttm_blockdiag: tensor cores, operands read as TF32 */
+
+typedef struct {
+    int32_t kind;      /* st_kind */
+    int32_t reserved;  /* must be 0 */
+    int64_t d;         /* structured extent: the matrix is d x d, ST_TET is d x d x d */
+    int64_t inner;     /* trailing dense extent carried by every position (>= 1) */
+    int64_t kl, ku;    /* ST_BAND: sub- and super-diagonals kept (>= 0) */
+    int64_t nblocks;   /* ST_BLOCKDIAG: number of blocks; d must equal nblocks*bs */
+    int64_t bs;        /* ST_BLOCKDIAG: block size */
+} st_layout;
+
+/* Number of packed positions times `inner` (elements of the packed array), or -1 for an
+ * invalid layout.  Host only. */
+int64_t st_packed_elems(const st_layout *layout);
+
+/* Number of elements of the dense counterpart (d*d*inner or d*d*d*inner), or -1. */
+int64_t st_dense_elems(const st_layout *layout);
+
+/* T_C = T * T_U, stored contiguously (Section 4, "Compressed Tensor"; Section 6,
+ * Property 2).  Gathers the positions of the unique set of `dense` into `packed`;
+ * positions outside T_U are not read.  A bit copy for any dtype (NaN payloads and
+ * -0.0 are preserved).  dense: [d,d,inner] ([d,d,d,inner] for ST_TET); packed:
+ * st_packed_elems(layout) elements.  The two arrays must not overlap. */
+st_status st_pack(const st_layout *layout, st_dtype dtype, const void *dense, void *packed,
+                  void *stream);
+
+/* Reconstruction T = T_C + T_R * T_C (Section 6, Property 5; Section 5.5).  Writes
+ * every element of `dense`: positions of T_U from `packed`, the others +0.0
+ * (ST_FILL_ZERO: sparsity structure, T_R empty) or through the redundancy map of the
+ * symmetric structure (ST_FILL_SYMMETRIC; ST_TRI_UPPER: T(i,j) = T_C(j,i) for j<i,
+ * Figure "structures in STUR"; ST_TET: T(i,j,k) = T_C(sorted (i,j,k))).
+ * ST_FILL_SYMMETRIC with ST_BAND / ST_BLOCKDIAG returns ST_ERR_UNSUPPORTED. */
+st_status st_unpack(const st_layout *layout, st_dtype dtype, const void *packed, void *dense,
+                    st_fill fill, void *stream);
+
+/* Scratch bytes needed by one compute call.  Arguments by op:
+ *   ST_OP_SYM_MOMENT2   a=N, b=d, c=st_dtype of X, e unused
+ *   ST_OP_SYM_MOMENT3   a=N, b=d
+ *   ST_OP_MTTKRP_TRI    a=I, b=K, c=R
+ *   ST_OP_TTM_BLOCKDIAG a=nblocks, b=bs, c=K, e=R
+ * Returns 0 for an invalid request (the call itself reports the error).  The current
+ * device is queried for its SM count. */
+size_t st_workspace_bytes(st_op op, int64_t a, int64_t b, int64_t c, int64_t e, unsigned flags);
+
+/* Second moment over the unique set of the symmetric output (Section 3, M1 = f (x) f
+ * summed over samples; Section 5.5, "Vector Self-Outer-Product": y_U = 0<=i<=j<n):
+ *     out[p(i,j)] = sum_n X[n,i] * X[n,j]      for 0 <= i <= j < d
+ * X: [N, ldx] with ldx >= d, dtype ST_F32 (fp32 FMA path, any d) or ST_BF16 (tensor-core
+ * path: bf16 products, fp32 accumulation; needs d % 64 == 0, ldx % 8 == 0).
+ * out_packed: d(d+1)/2 floats in ST_TRI_UPPER order.
+ * ST_FLAG_DENSE_CONTROL: all d*d products are computed (lower-triangle tiles too) and
+ * the lower results discarded; the output is the same. */
+st_status st_sym_moment2(const void *X, st_dtype xdt, int64_t N, int64_t d, int64_t ldx,
+                         float *out_packed, void *ws, size_t ws_bytes, unsigned flags,
+                         void *stream);
+
+/* Third moment over the unique set (Section 3, M2 = f (x) vec(f (x) f) summed over
+ * samples; its unique elements are i<=j<=k, Section 2 "Tensor Structures"):
+ *     out[q(i,j,k)] = sum_n X[n,i] * X[n,j] * X[n,k]   for 0 <= i <= j <= k < d
+ * X: fp32 [N, ldx], ldx >= d, ldx % 4 == 0.  out_packed: d(d+1)(d+2)/6 floats in ST_TET
+ * order.  Supported: d % 8 == 0, 8 <= d <= 64.
+ * ST_FLAG_DENSE_CONTROL: all d*d*d products are computed and the results outside the
+ * unique set discarded; the output is the same. */
+st_status st_sym_moment3(const float *X, int64_t N, int64_t d, int64_t ldx,
+                         float *out_packed, void *ws, size_t ws_bytes, unsigned flags,
+                         void *stream);
+
+/* MTTKRP (Table 1) on a tensor whose unique set is the "upper half cube" of Table 1,
+ * B_U(i,j,k) = (0<=i<I)*(i<=j<I)*(0<=k<K):
+ *     A[i,r] = sum_{j>=i} sum_k Bp[p(i,j), k] * C[j,r] * D[k,r]
+ * Bp: packed [I(I+1)/2, K] fp32 (ST_TRI_UPPER with inner=K); C: [I,R]; D: [K,R];
+ * A: [I,R] fp32 (dense: its unique set is every (i,r)).  Needs K % 4 == 0, R in {8,16,32,64}.
+ * ST_FLAG_DENSE_CONTROL: Bp is instead a dense [I,I,K] tensor and all j are visited. */
+st_status st_mttkrp_tri(const float *Bp, int64_t I, int64_t K, const float *C, const float *D,
+                        int64_t R, float *A, void *ws, size_t ws_bytes, unsigned flags,
+                        void *stream);
+
+/* TTM (Table 1) on a tensor that is block-diagonal in its first two modes (a direct sum
+ * of nblocks blocks of bs x bs fibres):
+ *     Ap[b,i',j',r] = sum_k Bp[b,i',j',k] * U[k,r]
+ * The output keeps the structure of the input (A_U(i,j,r) = B_U(i,j,.)).
+ * Bp: packed [nblocks*bs*bs, K] fp32; U: [K,R] fp32; Ap: packed [nblocks*bs*bs, R] fp32.
+ * Needs K % 4 == 0 and R % 4 == 0.  ST_FLAG_TC_TF32 selects the tensor-core path
+ * (operands truncated to TF32, fp32 accumulation; needs K % 32 == 0, R % 16 == 0, R <= 256).
+ * ST_FLAG_DENSE_CONTROL: Bp is a dense [d,d,K] tensor and Ap a dense [d,d,R] one,
+ * d = nblocks*bs; all d*d fibres are multiplied. */
+st_status st_ttm_blockdiag(const float *Bp, int64_t nblocks, int64_t bs, int64_t K,
+                           const float *U, int64_t R, float *Ap, void *ws, size_t ws_bytes,
+                           unsigned flags, void *stream);
+
+/* Synchronises `stream`, then reads the status word a kernel may have written into the
+ * workspace (a bounded wait that ran out, a failed consistency check).  ws may be NULL. */
+st_status st_check_status(const void *ws, void *stream);
+
+const char *st_status_string(st_status s);
+
+/* Version of the ABI described in this header. */
+int st_abi_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* STRUCTTENSOR_H */

@@ -50,6 +50,7 @@ def _load():
         lib.oracle_moment2.argtypes = [vp, i64, i64, i64, vp, vp]
         lib.oracle_moment2_at.argtypes = [vp, i64, i64, i64, vp, vp, i64, vp, vp]
         lib.oracle_moment3.argtypes = [vp, i64, i64, i64, vp, vp]
+        lib.oracle_moment3_at.argtypes = [vp, i64, i64, i64, vp, vp, vp, i64, vp, vp]
         lib.oracle_moment4.argtypes = [vp, i64, i64, i64, vp, vp]
         lib.oracle_mttkrp.argtypes = [vp, i64, i64, i64, vp, vp, i64, i64, i64, vp, vp]
         lib.oracle_ttm.argtypes = [vp, i64, i64, vp, i64, vp, vp]
@@ -119,6 +120,21 @@ def moment3(X):
     T = np.zeros((d, d, d), np.float64)
     S = np.zeros((d, d, d), np.float64)
     _load().oracle_moment3(_ptr(X), N, d, ldx, _ptr(T), _ptr(S))
+    return T, S
+
+
+def moment3_at(X, ii, jj, kk):
+    """The same sums for sampled entries (ii[e], jj[e], kk[e]) only."""
+    X, N, d, ldx = _x2d(X)
+    idx = [np.ascontiguousarray(a, dtype=np.int64) for a in (ii, jj, kk)]
+    assert idx[0].ndim == 1 and idx[0].shape == idx[1].shape == idx[2].shape
+    for a in idx:
+        if a.size and (a.min() < 0 or a.max() >= d):
+            raise IndexError("sample index out of range")
+    T = np.zeros(idx[0].size, np.float64)
+    S = np.zeros(idx[0].size, np.float64)
+    _load().oracle_moment3_at(_ptr(X), N, d, ldx, _ptr(idx[0]), _ptr(idx[1]), _ptr(idx[2]), idx[0].size,
+                              _ptr(T), _ptr(S))
     return T, S
 
 

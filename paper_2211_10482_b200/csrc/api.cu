@@ -1,0 +1,59 @@
+// Entry points that are not tied to one kernel: workspace sizes, status, version.
+#include "st_common.cuh"
+
+namespace st {
+size_t moment2_workspace(int64_t N, int64_t d, int xdt, unsigned flags);
+size_t moment3_workspace(int64_t N, int64_t d, unsigned flags);
+size_t ttm_tf32_tc_workspace(int64_t rows, int64_t K, int64_t R);
+}  // namespace st
+
+extern "C" {
+
+size_t st_workspace_bytes(st_op op, int64_t a, int64_t b, int64_t c, int64_t e, unsigned flags)
+{
+    switch (op) {
+    case ST_OP_SYM_MOMENT2: return st::moment2_workspace(a, b, (int)c, flags);
+    case ST_OP_SYM_MOMENT3: return st::moment3_workspace(a, b, flags);
+    case ST_OP_MTTKRP_TRI: return (a > 0 && b > 0 && c > 0) ? st::kWsHeaderBytes : 0;
+    case ST_OP_TTM_BLOCKDIAG:
+        if (a <= 0 || b <= 0 || c <= 0 || e <= 0) return 0;
+        if (flags & ST_FLAG_TC_TF32) {
+            const int64_t d = a * b;
+            return st::ttm_tf32_tc_workspace((flags & ST_FLAG_DENSE_CONTROL) ? d * d : a * b * b, c, e);
+        }
+        return st::kWsHeaderBytes;
+    default: return 0;
+    }
+}
+
+st_status st_check_status(const void *ws, void *stream)
+{
+    if (cudaStreamSynchronize((cudaStream_t)stream) != cudaSuccess) return ST_ERR_CUDA;
+    if (!ws) return ST_OK;
+    unsigned words[2] = {0, 0};
+    if (cudaMemcpy(words, ws, sizeof(words), cudaMemcpyDeviceToHost) != cudaSuccess) return ST_ERR_CUDA;
+    if (words[0] == ST_ERR_DEV_TIMEOUT) return ST_ERR_DEV_TIMEOUT;
+    if (words[0] == ST_ERR_DEV_BOUNDS) return ST_ERR_DEV_BOUNDS;
+    return ST_OK;
+}
+
+const char *st_status_string(st_status s)
+{
+    switch (s) {
+    case ST_OK: return "ok";
+    case ST_ERR_NULL: return "null pointer";
+    case ST_ERR_SHAPE: return "bad shape";
+    case ST_ERR_ALIGN: return "misaligned pointer or leading dimension";
+    case ST_ERR_DTYPE: return "unsupported element type";
+    case ST_ERR_WORKSPACE: return "workspace missing or too small";
+    case ST_ERR_UNSUPPORTED: return "request not supported by the kernels";
+    case ST_ERR_CUDA: return "CUDA call failed";
+    case ST_ERR_DEV_TIMEOUT: return "a bounded wait inside a kernel ran out";
+    case ST_ERR_DEV_BOUNDS: return "kernel-side consistency check failed";
+    default: return "unknown status";
+    }
+}
+
+int st_abi_version(void) { return 1; }
+
+}  // extern "C"

@@ -1,0 +1,328 @@
+// st_sym_moment3: out[q(i,j,k)] = sum_n X[n,i] X[n,j] X[n,k] over the unique set
+// 0<=i<=j<=k<d (Section 3, M2; Section 2, "Tensor Structures").  fp32 FMA bound.
+//
+// Work decomposition.  The unique set is cut into register tiles (i; 8 values of j; 8 values
+// of k) aligned to blocks of 8: tile (i, jb, kb) with block(i) <= jb <= kb.  One thread owns
+// one tile for a slice of the samples and keeps its <= 64 sums in registers; per sample it
+// reads x_i, the 8 x_j and the 8 x_k of the row from shared memory, forms the pair product
+// p = x_i * x_j once per j (loop-invariant code motion of Section 5.5 applied to the k loop)
+// and issues one FMA per unique triple -- nothing outside i<=j<=k is computed:
+//     variant 0        full 8x8 tile            (jb > block(i) or i at a block start, kb > jb)
+//     variant 1        triangular, k >= j       (kb == jb; rows j < i are not stored)
+//     variant 1+s      rows j >= i only, s=i%8  (jb == block(i), kb > jb), s = 1..7
+// Threads are grouped into warps of one variant so no lane diverges; warps are dealt to
+// G thread blocks x 4 schedulers so that every scheduler gets the same FMA count.  The
+// tile table is built on the host for the given d and travels as a kernel parameter.
+//
+// The sample range is split over gridDim.y slices; every slice writes its partial sums to
+// the workspace and a second kernel adds the slices in a fixed order.
+#include "st_common.cuh"
+#include "st_index.cuh"
+#include <algorithm>
+#include <vector>
+
+namespace st {
+
+constexpr int M3_THREADS = 512;            // 16 warps per block
+constexpr int M3_WPB = M3_THREADS / 32;
+constexpr int M3_STAGE_ROWS = 64;          // sample rows per shared-memory stage
+constexpr int M3_MAX_D = 64;
+
+template <int WARPS>
+struct M3Table {
+    int groups;                            // thread blocks per sample slice
+    int nbk;                               // d / 8
+    unsigned char variant[WARPS];          // per warp slot (group-major): variant id, 255 = idle
+    unsigned short tile[WARPS * 32];       // per thread slot: i | jb<<6 | kb<<9 | valid<<15
+};
+
+__device__ __forceinline__ void cp_async16(void *smem, const void *gmem, bool valid)
+{
+    const unsigned s = (unsigned)__cvta_generic_to_shared(smem);
+    const int sz = valid ? 16 : 0;         // src-size 0: the 16 bytes are zero-filled
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;\n" ::"r"(s), "l"(gmem), "r"(sz));
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;\n" ::); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;\n" ::"n"(N)); }
+
+// One stage of rows for one tile.  Row layout in shared memory ("split halves"): columns
+// 8b..8b+3 of block b sit at floats 4b.., columns 8b+4..8b+7 at floats 4*nbk+4b.., so that a
+// 128-bit load of "the first (second) half of block b" by lanes with arbitrary b touches
+// each bank once.
+template <int J0, bool DIAG>
+__device__ __forceinline__ void m3_stage(const float *__restrict__ xs, int d, int pi, int oj, int ok, int half,
+                                         float (&acc)[8][8])
+{
+#pragma unroll 2
+    for (int r = 0; r < M3_STAGE_ROWS; ++r) {
+        const float *row = xs + r * d;
+        const float xi = row[pi];
+        const float4 ja = *reinterpret_cast<const float4 *>(row + oj);
+        const float4 jb = *reinterpret_cast<const float4 *>(row + oj + half);
+        float4 ka, kb;
+        if (DIAG) {
+            ka = ja;
+            kb = jb;
+        } else {
+            ka = *reinterpret_cast<const float4 *>(row + ok);
+            kb = *reinterpret_cast<const float4 *>(row + ok + half);
+        }
+        const float xj[8] = {ja.x, ja.y, ja.z, ja.w, jb.x, jb.y, jb.z, jb.w};
+        const float xk[8] = {ka.x, ka.y, ka.z, ka.w, kb.x, kb.y, kb.z, kb.w};
+#pragma unroll
+        for (int a = J0; a < 8; ++a) {
+            const float p = xi * xj[a];
+#pragma unroll
+            for (int b = (DIAG ? a : 0); b < 8; ++b) acc[a][b] = fmaf(p, xk[b], acc[a][b]);
+        }
+    }
+}
+
+template <int WARPS>
+__global__ void __launch_bounds__(M3_THREADS, 1)
+moment3_kernel(const float *__restrict__ X, int64_t N, int d, int64_t ldx, float *__restrict__ partials,
+               int64_t rows_per_slice, int out_elems, const __grid_constant__ M3Table<WARPS> tab)
+{
+    extern __shared__ __align__(16) float smem[];   // 2 stages of M3_STAGE_ROWS x d floats
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int group = blockIdx.x;
+    const int slot = group * M3_WPB + warp;
+    const int variant = tab.variant[slot];
+    const unsigned t = tab.tile[slot * 32 + lane];
+    const bool valid = (t >> 15) & 1u;
+    const int ti = t & 63, tjb = (t >> 6) & 7, tkb = (t >> 9) & 7;
+    const int nbk = tab.nbk;
+    const int half = 4 * nbk;
+    // shared-memory float offset of column c: block c/8, half (c%8)/4
+    const int pi = ((ti & 7) < 4) ? 4 * (ti >> 3) + (ti & 3) : half + 4 * (ti >> 3) + (ti & 3);
+    const int oj = 4 * tjb, ok = 4 * tkb;
+
+    float acc[8][8];
+#pragma unroll
+    for (int a = 0; a < 8; ++a)
+#pragma unroll
+        for (int b = 0; b < 8; ++b) acc[a][b] = 0.f;
+
+    const int64_t n_begin = (int64_t)blockIdx.y * rows_per_slice;
+    int64_t n_end = n_begin + rows_per_slice;
+    if (n_end > N) n_end = N;
+    const int stage_floats = M3_STAGE_ROWS * d;
+    const int chunks_per_row = d / 4;
+    const int stage_chunks = M3_STAGE_ROWS * chunks_per_row;
+
+    auto load_stage = [&](int buf, int64_t n0) {
+        float *dst = smem + buf * stage_floats;
+        for (int c = tid; c < stage_chunks; c += M3_THREADS) {
+            const int r = c / chunks_per_row, g = c - r * chunks_per_row;
+            const int64_t n = n0 + r;
+            const int sc = (g & 1) ? nbk + (g >> 1) : (g >> 1);   // split-half position of chunk g
+            const bool ok_row = n < n_end;
+            cp_async16(dst + r * d + 4 * sc, X + (ok_row ? n : n_begin) * ldx + 4 * g, ok_row);
+        }
+        cp_async_commit();
+    };
+
+    const int64_t nstages = (n_end > n_begin) ? (n_end - n_begin + M3_STAGE_ROWS - 1) / M3_STAGE_ROWS : 0;
+    if (nstages > 0) load_stage(0, n_begin);
+    for (int64_t s = 0; s < nstages; ++s) {
+        const int buf = (int)(s & 1);
+        if (s + 1 < nstages) {
+            load_stage(buf ^ 1, n_begin + (s + 1) * M3_STAGE_ROWS);
+            cp_async_wait<1>();
+        } else {
+            cp_async_wait<0>();
+        }
+        __syncthreads();
+        const float *xs = smem + buf * stage_floats;
+        switch (variant) {
+        case 0: m3_stage<0, false>(xs, d, pi, oj, ok, half, acc); break;
+        case 1: m3_stage<0, true>(xs, d, pi, oj, ok, half, acc); break;
+        case 2: m3_stage<1, false>(xs, d, pi, oj, ok, half, acc); break;
+        case 3: m3_stage<2, false>(xs, d, pi, oj, ok, half, acc); break;
+        case 4: m3_stage<3, false>(xs, d, pi, oj, ok, half, acc); break;
+        case 5: m3_stage<4, false>(xs, d, pi, oj, ok, half, acc); break;
+        case 6: m3_stage<5, false>(xs, d, pi, oj, ok, half, acc); break;
+        case 7: m3_stage<6, false>(xs, d, pi, oj, ok, half, acc); break;
+        case 8: m3_stage<7, false>(xs, d, pi, oj, ok, half, acc); break;
+        default: break;
+        }
+        __syncthreads();
+    }
+
+    if (!valid || variant == 255) return;
+    float *mine = partials + (size_t)blockIdx.y * out_elems;
+#pragma unroll
+    for (int a = 0; a < 8; ++a) {
+        const int j = 8 * tjb + a;
+        if (j < ti) continue;
+        const int base = (int)tet_encode(d, ti, j, j);   // row (i,j,*) is contiguous in k
+#pragma unroll
+        for (int b = 0; b < 8; ++b) {
+            const int k = 8 * tkb + b;
+            if (k >= j) mine[base + (k - j)] = acc[a][b];
+        }
+    }
+}
+
+__global__ void __launch_bounds__(256)
+sum_slices_kernel(const float *__restrict__ partials, float *__restrict__ out, int64_t elems, int slices)
+{
+    const int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (e >= elems) return;
+    float s = 0.f;
+    for (int k = 0; k < slices; ++k) s += __ldcg(&partials[(size_t)k * elems + e]);
+    out[e] = s;
+}
+
+// ---- host side: tile table ------------------------------------------------------------
+
+struct WarpDesc {
+    int variant;
+    int cost;
+    std::vector<unsigned short> tiles;
+};
+
+static int variant_cost(int v)
+{
+    if (v == 0) return 64 + 8 + 6;
+    if (v == 1) return 36 + 8 + 4;
+    const int rows = 8 - (v - 1);
+    return rows * 8 + rows + 6;
+}
+
+// Builds the per-thread tile table for side d.  Returns the number of groups.
+template <int WARPS>
+static bool build_table(int d, bool dense, M3Table<WARPS> &tab)
+{
+    const int nbk = d / 8;
+    std::vector<std::vector<unsigned short>> lists(9);
+    for (int i = 0; i < d; ++i) {
+        const int ib = i / 8, s = i % 8;
+        for (int jb = dense ? 0 : ib; jb < nbk; ++jb)
+            for (int kb = dense ? 0 : jb; kb < nbk; ++kb) {
+                const unsigned short t = (unsigned short)(i | (jb << 6) | (kb << 9) | (1u << 15));
+                int v;
+                if (dense) v = 0;
+                else if (kb == jb) v = 1;
+                else if (jb == ib && s != 0) v = 1 + s;
+                else v = 0;
+                lists[v].push_back(t);
+            }
+    }
+    std::vector<WarpDesc> warps;
+    for (int v = 0; v < 9; ++v)
+        for (size_t o = 0; o < lists[v].size(); o += 32) {
+            WarpDesc w;
+            w.variant = v;
+            w.cost = variant_cost(v);
+            w.tiles.assign(lists[v].begin() + o, lists[v].begin() + std::min(lists[v].size(), o + 32));
+            warps.push_back(w);
+        }
+    const int nw = (int)warps.size();
+    const int groups = (nw + M3_WPB - 1) / M3_WPB;
+    if (groups * M3_WPB > WARPS) return false;
+    // deal warps, most expensive first, to the scheduler bin (group, warp%4) with the least load
+    std::stable_sort(warps.begin(), warps.end(), [](const WarpDesc &a, const WarpDesc &b) { return a.cost > b.cost; });
+    const int bins = groups * 4;
+    std::vector<int> load(bins, 0), count(bins, 0);
+    tab.groups = groups;
+    tab.nbk = nbk;
+    for (int w = 0; w < WARPS; ++w) tab.variant[w] = 255;
+    for (int e = 0; e < WARPS * 32; ++e) tab.tile[e] = 0;
+    for (const WarpDesc &w : warps) {
+        int best = -1;
+        for (int b = 0; b < bins; ++b)
+            if (count[b] < M3_WPB / 4 && (best < 0 || load[b] < load[best])) best = b;
+        if (best < 0) return false;
+        const int g = best / 4, sched = best % 4;
+        const int slot = g * M3_WPB + sched + 4 * count[best];   // warp index % 4 = scheduler
+        load[best] += w.cost;
+        count[best] += 1;
+        tab.variant[slot] = (unsigned char)w.variant;
+        for (size_t l = 0; l < w.tiles.size(); ++l) tab.tile[slot * 32 + l] = w.tiles[l];
+    }
+    return true;
+}
+
+struct M3Plan {
+    int groups, slices;
+    int64_t rows_per_slice;
+    int64_t out_elems;
+};
+
+// One block group per sample slice; slices fill the SMs once.
+static M3Plan moment3_plan(int64_t N, int64_t d, int groups)
+{
+    M3Plan p;
+    p.groups = groups;
+    p.out_elems = tet_rows(d);
+    const int sms = sm_count_or_default();
+    int64_t slices = sms / groups;
+    if (slices < 1) slices = 1;
+    const int64_t max_slices = (N + M3_STAGE_ROWS - 1) / M3_STAGE_ROWS;
+    if (slices > max_slices) slices = max_slices;
+    p.rows_per_slice = (N + slices - 1) / slices;
+    p.slices = (int)((N + p.rows_per_slice - 1) / p.rows_per_slice);
+    return p;
+}
+
+template <int WARPS>
+static st_status moment3_launch(const float *X, int64_t N, int64_t d, int64_t ldx, float *out, void *ws,
+                                size_t ws_bytes, unsigned flags, cudaStream_t stream)
+{
+    M3Table<WARPS> local;   // rebuilt on every call: a few microseconds of host work
+    if (!build_table<WARPS>((int)d, (flags & ST_FLAG_DENSE_CONTROL) != 0, local)) return ST_ERR_UNSUPPORTED;
+    const M3Plan p = moment3_plan(N, d, local.groups);
+    const size_t need = kWsHeaderBytes + (size_t)p.slices * p.out_elems * sizeof(float);
+    if (!ws || ws_bytes < need) return ST_ERR_WORKSPACE;
+    if (!aligned256(ws)) return ST_ERR_ALIGN;
+    float *partials = (float *)((unsigned char *)ws + kWsHeaderBytes);
+    const size_t smem = 2 * (size_t)M3_STAGE_ROWS * d * sizeof(float);
+    if (smem > 48 * 1024) {
+        if (cudaFuncSetAttribute(moment3_kernel<WARPS>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
+            cudaSuccess)
+            return ST_ERR_CUDA;
+    }
+    dim3 grid(p.groups, p.slices);
+    moment3_kernel<WARPS><<<grid, M3_THREADS, smem, stream>>>(X, N, (int)d, ldx, partials, p.rows_per_slice,
+                                                              (int)p.out_elems, local);
+    if (cudaGetLastError() != cudaSuccess) return ST_ERR_CUDA;
+    const int64_t e = p.out_elems;
+    sum_slices_kernel<<<(unsigned)((e + 255) / 256), 256, 0, stream>>>(partials, out, e, p.slices);
+    return launch_status();
+}
+
+static int moment3_groups(int64_t d, unsigned flags)
+{
+    if (flags & ST_FLAG_DENSE_CONTROL) {
+        M3Table<128> t;
+        return build_table<128>((int)d, true, t) ? t.groups : 0;
+    }
+    M3Table<32> t;
+    return build_table<32>((int)d, false, t) ? t.groups : 0;
+}
+
+size_t moment3_workspace(int64_t N, int64_t d, unsigned flags)
+{
+    if (N <= 0 || d < 8 || d > M3_MAX_D || d % 8) return 0;
+    const int groups = moment3_groups(d, flags);
+    if (groups == 0) return 0;
+    const M3Plan p = moment3_plan(N, d, groups);
+    return kWsHeaderBytes + (size_t)p.slices * p.out_elems * sizeof(float);
+}
+
+}  // namespace st
+
+extern "C" st_status st_sym_moment3(const float *X, int64_t N, int64_t d, int64_t ldx, float *out_packed,
+                                    void *ws, size_t ws_bytes, unsigned flags, void *stream)
+{
+    if (!X || !out_packed) return ST_ERR_NULL;
+    if (N <= 0 || d <= 0 || ldx < d) return ST_ERR_SHAPE;
+    if (flags & ~(ST_FLAG_DENSE_CONTROL)) return ST_ERR_UNSUPPORTED;
+    if (d < 8 || d > st::M3_MAX_D || d % 8) return ST_ERR_UNSUPPORTED;
+    if (!st::aligned16(X) || !st::aligned16(out_packed) || ldx % 4) return ST_ERR_ALIGN;
+    if (flags & ST_FLAG_DENSE_CONTROL)
+        return st::moment3_launch<128>(X, N, d, ldx, out_packed, ws, ws_bytes, flags, (cudaStream_t)stream);
+    return st::moment3_launch<32>(X, N, d, ldx, out_packed, ws, ws_bytes, flags, (cudaStream_t)stream);
+}

@@ -1,0 +1,235 @@
+// st_pack / st_unpack: gather the unique set T_U of a dense tensor into the packed layout
+// (T_C = T * T_U, Section 4) and reconstruct the dense tensor from it
+// (T = T_C + T_R * T_C, Section 6, Property 5).  HBM-bound index-decode copies.
+//
+// Both kernels are organised by rows: a row is one position of the structured modes
+// carrying `inner` contiguous elements.  A group of G lanes (G a power of two <= 32) owns
+// one row of the array being WRITTEN, decodes its index tuple once with the closed forms
+// of st_index.cuh, and copies the row in units of U bytes (16 where the row width allows),
+// so stores are always coalesced and loads are coalesced within a row.
+#include "st_common.cuh"
+#include "st_index.cuh"
+
+namespace st {
+
+struct LayoutArgs {
+    int kind;
+    int fill;
+    int64_t d, kl, ku, nb, bs;
+    int64_t width;       // band: kl+ku+1
+    int64_t packed_rows;
+    int64_t dense_rows;
+    int64_t chunks;      // units of U bytes per row
+};
+
+// Dense row index of packed row p, or -1 for a band slot outside the matrix.
+template <int KIND>
+__device__ __forceinline__ int64_t dense_row_of_packed(const LayoutArgs &a, int64_t p)
+{
+    if (KIND == ST_TRI_UPPER) {
+        int64_t i, j;
+        tri_decode(a.d, p, i, j);
+        return i * a.d + j;
+    } else if (KIND == ST_TET) {
+        int64_t i, j, k;
+        tet_decode(a.d, p, i, j, k);
+        return (i * a.d + j) * a.d + k;
+    } else if (KIND == ST_BAND) {
+        const int64_t i = p / a.width;
+        const int64_t j = i + (p - i * a.width) - a.kl;
+        return (j >= 0 && j < a.d) ? i * a.d + j : -1;
+    } else {
+        const int64_t bb = a.bs * a.bs;
+        const int64_t b = p / bb;
+        const int64_t rem = p - b * bb;
+        const int64_t ii = rem / a.bs;
+        const int64_t jj = rem - ii * a.bs;
+        return (b * a.bs + ii) * a.d + b * a.bs + jj;
+    }
+}
+
+// Packed row that dense row r is read from, or -1 when the position is a structural zero.
+template <int KIND>
+__device__ __forceinline__ int64_t packed_row_of_dense(const LayoutArgs &a, int64_t r)
+{
+    if (KIND == ST_TRI_UPPER) {
+        int64_t i = r / a.d, j = r - i * a.d;
+        if (i > j) {
+            if (a.fill != ST_FILL_SYMMETRIC) return -1;
+            int64_t t = i; i = j; j = t;     // T_R(i,j,i',j') = (j<i)*(i'=j)*(j'=i)
+        }
+        return tri_encode(a.d, i, j);
+    } else if (KIND == ST_TET) {
+        const int64_t ij = r / a.d;
+        int64_t k = r - ij * a.d;
+        int64_t i = ij / a.d, j = ij - i * a.d;
+        if (!(i <= j && j <= k)) {
+            if (a.fill != ST_FILL_SYMMETRIC) return -1;
+            int64_t t;                        // representative = sorted index triple
+            if (i > j) { t = i; i = j; j = t; }
+            if (j > k) { t = j; j = k; k = t; }
+            if (i > j) { t = i; i = j; j = t; }
+        }
+        return tet_encode(a.d, i, j, k);
+    } else if (KIND == ST_BAND) {
+        const int64_t i = r / a.d, j = r - i * a.d;
+        const int64_t s = j - i + a.kl;
+        return (s >= 0 && s < a.width) ? i * a.width + s : -1;
+    } else {
+        const int64_t i = r / a.d, j = r - i * a.d;
+        const int64_t b = i / a.bs;
+        if (j / a.bs != b) return -1;
+        return (i * a.bs) + (j - b * a.bs);   // ((b*bs + i')*bs + j') with b*bs+i' = i
+    }
+}
+
+template <typename U>
+__device__ __forceinline__ U zero_unit();
+template <> __device__ __forceinline__ uint4 zero_unit<uint4>() { return make_uint4(0, 0, 0, 0); }
+template <> __device__ __forceinline__ uint2 zero_unit<uint2>() { return make_uint2(0, 0); }
+template <> __device__ __forceinline__ uint32_t zero_unit<uint32_t>() { return 0u; }
+template <> __device__ __forceinline__ uint16_t zero_unit<uint16_t>() { return 0; }
+
+// PACK = true : rows of `dst` are packed rows, source rows are dense rows.
+// PACK = false: rows of `dst` are dense rows, source rows are packed rows.
+template <int KIND, typename U, bool PACK>
+__global__ void __launch_bounds__(256)
+structured_copy_kernel(const U *__restrict__ src, U *__restrict__ dst, LayoutArgs a, int group_shift)
+{
+    const int64_t rows = PACK ? a.packed_rows : a.dense_rows;
+    const int g = 1 << group_shift;
+    const int64_t tid = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    const int64_t groups = ((int64_t)gridDim.x * blockDim.x) >> group_shift;
+    const int lane = (int)(tid & (g - 1));
+    for (int64_t row = tid >> group_shift; row < rows; row += groups) {
+        const int64_t srow = PACK ? dense_row_of_packed<KIND>(a, row) : packed_row_of_dense<KIND>(a, row);
+        U *out = dst + row * a.chunks;
+        if (srow >= 0) {
+            const U *in = src + srow * a.chunks;
+            for (int64_t c = lane; c < a.chunks; c += g) out[c] = in[c];
+        } else {
+            for (int64_t c = lane; c < a.chunks; c += g) out[c] = zero_unit<U>();
+        }
+    }
+}
+
+static bool layout_ok(const st_layout *L)
+{
+    if (!L) return false;
+    if (L->reserved != 0) return false;
+    if (L->d <= 0 || L->inner <= 0) return false;
+    if (L->d > (int64_t(1) << 31)) return false;
+    switch (L->kind) {
+    case ST_TRI_UPPER: return true;
+    case ST_TET: return L->d <= (int64_t(1) << 20);
+    case ST_BAND: return L->kl >= 0 && L->ku >= 0 && L->kl < (int64_t(1) << 31) && L->ku < (int64_t(1) << 31);
+    case ST_BLOCKDIAG: return L->nblocks > 0 && L->bs > 0 && L->nblocks * L->bs == L->d;
+    default: return false;
+    }
+}
+
+static int64_t packed_rows_of(const st_layout *L)
+{
+    switch (L->kind) {
+    case ST_TRI_UPPER: return tri_rows(L->d);
+    case ST_TET: return tet_rows(L->d);
+    case ST_BAND: return L->d * (L->kl + L->ku + 1);
+    default: return L->nblocks * L->bs * L->bs;
+    }
+}
+
+static int64_t dense_rows_of(const st_layout *L)
+{
+    return L->kind == ST_TET ? L->d * L->d * L->d : L->d * L->d;
+}
+
+static int dtype_bytes(st_dtype t)
+{
+    switch (t) {
+    case ST_F32: return 4;
+    case ST_BF16: return 2;
+    case ST_F64: return 8;
+    default: return 0;
+    }
+}
+
+template <int KIND, typename U, bool PACK>
+static st_status launch_copy(const void *src, void *dst, const LayoutArgs &a, cudaStream_t s)
+{
+    const int64_t rows = PACK ? a.packed_rows : a.dense_rows;
+    int shift = 0;
+    while ((1 << shift) < 32 && (int64_t(1) << shift) < a.chunks) ++shift;
+    const int64_t threads = rows << shift;
+    const int64_t want = (threads + 255) / 256;
+    const int64_t cap = (int64_t)sm_count_or_default() * 16;
+    const int grid = (int)(want < cap ? (want < 1 ? 1 : want) : cap);
+    structured_copy_kernel<KIND, U, PACK><<<grid, 256, 0, s>>>((const U *)src, (U *)dst, a, shift);
+    return launch_status();
+}
+
+template <typename U, bool PACK>
+static st_status dispatch_kind(const void *src, void *dst, const LayoutArgs &a, cudaStream_t s)
+{
+    switch (a.kind) {
+    case ST_TRI_UPPER: return launch_copy<ST_TRI_UPPER, U, PACK>(src, dst, a, s);
+    case ST_TET: return launch_copy<ST_TET, U, PACK>(src, dst, a, s);
+    case ST_BAND: return launch_copy<ST_BAND, U, PACK>(src, dst, a, s);
+    default: return launch_copy<ST_BLOCKDIAG, U, PACK>(src, dst, a, s);
+    }
+}
+
+template <bool PACK>
+static st_status copy_entry(const st_layout *L, st_dtype dtype, const void *src, void *dst, int fill,
+                            void *stream)
+{
+    if (!L || !src || !dst) return ST_ERR_NULL;
+    if (!layout_ok(L)) return ST_ERR_SHAPE;
+    const int es = dtype_bytes(dtype);
+    if (es == 0) return ST_ERR_DTYPE;
+    if (fill != ST_FILL_ZERO && fill != ST_FILL_SYMMETRIC) return ST_ERR_UNSUPPORTED;
+    if (fill == ST_FILL_SYMMETRIC && (L->kind == ST_BAND || L->kind == ST_BLOCKDIAG)) return ST_ERR_UNSUPPORTED;
+    if (!aligned16(src) || !aligned16(dst)) return ST_ERR_ALIGN;
+    LayoutArgs a;
+    a.kind = L->kind;
+    a.fill = fill;
+    a.d = L->d; a.kl = L->kl; a.ku = L->ku; a.nb = L->nblocks; a.bs = L->bs;
+    a.width = L->kl + L->ku + 1;
+    a.packed_rows = packed_rows_of(L);
+    a.dense_rows = dense_rows_of(L);
+    const int64_t w = L->inner * es;   // bytes per row
+    cudaStream_t s = (cudaStream_t)stream;
+    if (w % 16 == 0) { a.chunks = w / 16; return dispatch_kind<uint4, PACK>(src, dst, a, s); }
+    if (w % 8 == 0)  { a.chunks = w / 8;  return dispatch_kind<uint2, PACK>(src, dst, a, s); }
+    if (w % 4 == 0)  { a.chunks = w / 4;  return dispatch_kind<uint32_t, PACK>(src, dst, a, s); }
+    a.chunks = w / 2;
+    return dispatch_kind<uint16_t, PACK>(src, dst, a, s);
+}
+
+}  // namespace st
+
+extern "C" {
+
+int64_t st_packed_elems(const st_layout *layout)
+{
+    if (!st::layout_ok(layout)) return -1;
+    return st::packed_rows_of(layout) * layout->inner;
+}
+
+int64_t st_dense_elems(const st_layout *layout)
+{
+    if (!st::layout_ok(layout)) return -1;
+    return st::dense_rows_of(layout) * layout->inner;
+}
+
+st_status st_pack(const st_layout *layout, st_dtype dtype, const void *dense, void *packed, void *stream)
+{
+    return st::copy_entry<true>(layout, dtype, dense, packed, ST_FILL_ZERO, stream);
+}
+
+st_status st_unpack(const st_layout *layout, st_dtype dtype, const void *packed, void *dense, st_fill fill,
+                    void *stream)
+{
+    return st::copy_entry<false>(layout, dtype, packed, dense, (int)fill, stream);
+}
+
+}  // extern "C"

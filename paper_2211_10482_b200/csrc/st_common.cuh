@@ -1,0 +1,59 @@
+// Shared host-side helpers of the library (not part of the ABI).
+#pragma once
+#include <cuda_runtime.h>
+#include <cstdint>
+#include <cstddef>
+#include "structtensor.h"
+
+namespace st {
+
+// The first 256 bytes of every workspace: word 0 = device status (st_status written by a
+// kernel), word 1 = detail, words 8.. = arrival counters.  Cleared by each call that uses it.
+constexpr size_t kWsHeaderBytes = 256;
+constexpr int kWsStatusWord = 0;
+constexpr int kWsDetailWord = 1;
+constexpr int kWsTicketWord = 8;
+
+inline bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+inline bool aligned256(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 255u) == 0; }
+inline size_t round_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+struct DeviceInfo {
+    int device = -1;
+    int sm_count = 0;
+    int max_smem_optin = 0;
+    bool ok = false;
+};
+
+// Properties of the current device (cached per device index).
+inline DeviceInfo device_info()
+{
+    static DeviceInfo cache[64];
+    DeviceInfo bad;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return bad;
+    if (!cache[dev].ok) {
+        DeviceInfo di;
+        di.device = dev;
+        if (cudaDeviceGetAttribute(&di.sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return bad;
+        if (cudaDeviceGetAttribute(&di.max_smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev) != cudaSuccess) return bad;
+        di.ok = true;
+        cache[dev] = di;
+    }
+    return cache[dev];
+}
+
+// SM count used to size grids; 148 (B200) when no device can be queried, so that the
+// host-only size queries still answer.
+inline int sm_count_or_default()
+{
+    DeviceInfo di = device_info();
+    return di.ok ? di.sm_count : 148;
+}
+
+inline st_status launch_status()
+{
+    return cudaGetLastError() == cudaSuccess ? ST_OK : ST_ERR_CUDA;
+}
+
+}  // namespace st

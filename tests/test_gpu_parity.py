@@ -1,0 +1,296 @@
+"""GPU parity tests: every C-ABI call against the CPU oracle, element by element, on the same
+seeded inputs.  Integer / byte work must be bit-exact; fp32 paths must satisfy
+max |gpu - oracle| / sum|terms| <= 1e-4."""
+import itertools
+
+import numpy as np
+import pytest
+
+import oracle
+import workloads
+
+torch = pytest.importorskip("torch")
+pytestmark = pytest.mark.gpu
+
+TOL_F32 = 1e-4
+
+
+@pytest.fixture(scope="module")
+def st():
+    import paper_2211_10482_b200 as m
+    m.lib()
+    return m
+
+
+def dev(a):
+    return torch.from_numpy(np.ascontiguousarray(a)).cuda()
+
+
+def okw(layout):
+    return dict(kl=layout.kl, ku=layout.ku, nb=layout.nblocks, bs=layout.bs)
+
+
+# ------------------------------------------------------------------------------ pack / unpack
+
+def layouts(st):
+    out = []
+    for d in (1, 2, 3, 5, 8, 17, 64, 130):
+        out.append(st.Layout(st.ST_TRI_UPPER, d))
+    for d in (1, 2, 3, 5, 17, 40):
+        out.append(st.Layout(st.ST_TET, d))
+    out += [st.Layout(st.ST_BAND, 9, kl=2, ku=3), st.Layout(st.ST_BAND, 4, kl=6, ku=0),
+            st.Layout(st.ST_BAND, 33, kl=0, ku=0), st.Layout(st.ST_BAND, 70, kl=1, ku=5)]
+    out += [st.Layout(st.ST_BLOCKDIAG, 12, nblocks=3, bs=4), st.Layout(st.ST_BLOCKDIAG, 7, nblocks=7, bs=1),
+            st.Layout(st.ST_BLOCKDIAG, 64, nblocks=1, bs=64), st.Layout(st.ST_BLOCKDIAG, 96, nblocks=3, bs=32)]
+    return out
+
+
+@pytest.mark.parametrize("inner,dtype", [(1, np.float32), (3, np.float32), (4, np.float32), (36, np.float32),
+                                         (1, np.uint16), (5, np.uint16), (8, np.uint16), (1, np.float64),
+                                         (3, np.float64), (130, np.float32)])
+def test_pack_unpack_bit_exact(st, inner, dtype):
+    import dataclasses
+    for base in layouts(st):
+        lay = dataclasses.replace(base, inner=inner)
+        nd = st.st_dense_elems(lay)
+        if nd > 3_000_000:
+            continue
+        rng = np.random.default_rng(nd + inner)
+        bits = rng.integers(0, 2 ** 16, size=nd * np.dtype(dtype).itemsize // 2, dtype=np.uint16)
+        if dtype == np.float32:      # keep NaN payloads and -0.0 in the mix
+            dense = bits.view(np.float32)
+        elif dtype == np.float64:
+            dense = bits.view(np.float64)
+        else:
+            dense = bits
+        u = {4: np.uint32, 8: np.uint64, 2: np.uint16}[np.dtype(dtype).itemsize]
+        tdt = {4: torch.int32, 8: torch.int64, 2: torch.int16}[np.dtype(dtype).itemsize]
+        dense_t = torch.from_numpy(dense.view(u).view({4: np.int32, 8: np.int64, 2: np.int16}[dense.itemsize])).cuda()
+        want_p = oracle.pack(dense.view(u), lay.kind, lay.d, inner=inner, **okw(lay))
+        got_p = st.st_pack(dense_t, lay)
+        assert got_p.dtype == tdt
+        assert np.array_equal(got_p.cpu().numpy().view(u), want_p), (lay, "pack")
+        fills = [st.ST_FILL_ZERO] + ([st.ST_FILL_SYMMETRIC] if lay.kind in (st.ST_TRI_UPPER, st.ST_TET) else [])
+        for fill in fills:
+            want_d = oracle.unpack(want_p, lay.kind, lay.d, inner=inner, fill=fill, **okw(lay)).reshape(-1)
+            got_d = st.st_unpack(got_p, lay, fill=fill)
+            assert np.array_equal(got_d.cpu().numpy().view(u), want_d), (lay, "unpack", fill)
+            # pack(unpack(P)) == P always (band: corner slots are zero both times)
+            again = st.st_pack(got_d, lay)
+            assert torch.equal(again, got_p), (lay, "round trip")
+
+
+def test_unpack_of_symmetric_tensor_restores_it(st):
+    """Property 5: T = T_C + T_R * T_C for a tensor that has the structure."""
+    d = 37
+    X = workloads.draw((50, d), "normal", 3)
+    T2 = (X.T.astype(np.float64) @ X.astype(np.float64)).astype(np.float32)
+    T2 = np.triu(T2) + np.triu(T2, 1).T
+    lay = st.Layout(st.ST_TRI_UPPER, d)
+    back = st.st_unpack(st.st_pack(dev(T2), lay), lay, fill=st.ST_FILL_SYMMETRIC).cpu().numpy().reshape(d, d)
+    assert np.array_equal(back.view(np.uint32), T2.view(np.uint32))
+
+
+def test_pack_unpack_at_config_sizes(st):
+    # tri d=1024 (moment2-large output) and tet d=64 (moment3 output): full comparison
+    for lay in (st.Layout(st.ST_TRI_UPPER, 1024), st.Layout(st.ST_TET, 64)):
+        n = st.st_packed_elems(lay)
+        P = np.random.default_rng(n).integers(0, 2 ** 32, size=n, dtype=np.uint32)
+        Pt = torch.from_numpy(P.view(np.int32)).cuda()
+        for fill in (st.ST_FILL_ZERO, st.ST_FILL_SYMMETRIC):
+            want = oracle.unpack(P, lay.kind, lay.d, fill=fill).reshape(-1)
+            got = st.st_unpack(Pt, lay, fill=fill)
+            assert np.array_equal(got.cpu().numpy().view(np.uint32), want)
+            assert torch.equal(st.st_pack(got, lay), Pt)
+    # tri x K with I=512, K=512 (MTTKRP operand): full comparison of pack, unpack on device
+    lay = st.Layout(st.ST_TRI_UPPER, 512, inner=512)
+    dense = np.random.default_rng(1).integers(0, 2 ** 32, size=512 * 512 * 512, dtype=np.uint32)
+    want = oracle.pack(dense, lay.kind, lay.d, inner=512)
+    dense_t = torch.from_numpy(dense.view(np.int32)).cuda()
+    got = st.st_pack(dense_t, lay)
+    assert np.array_equal(got.cpu().numpy().view(np.uint32), want)
+    back = st.st_unpack(got, lay).view(512, 512, 512)
+    mask = torch.triu(torch.ones(512, 512, dtype=torch.bool, device="cuda"))
+    assert torch.equal(back[mask], dense_t.view(512, 512, 512)[mask])
+    assert int(torch.count_nonzero(back[~mask])) == 0
+    del dense_t, back, got
+    # block-diagonal 64 blocks of 64x64 with K=256 (TTM operand): 16 GiB dense, sampled fibres
+    lay = st.Layout(st.ST_BLOCKDIAG, 4096, inner=256, nblocks=64, bs=64)
+    n = st.st_packed_elems(lay)
+    Pt = torch.randint(-2 ** 31, 2 ** 31 - 1, (n,), dtype=torch.int32, device="cuda",
+                       generator=torch.Generator(device="cuda").manual_seed(7))
+    dense_t = st.st_unpack(Pt, lay).view(4096, 4096, 256)
+    rng = np.random.default_rng(11)
+    samples = [(0, 0), (63, 63), (63, 64), (64, 63), (4095, 4095), (4095, 4032), (4032, 4031), (100, 70)]
+    samples += [tuple(int(v) for v in rng.integers(0, 4096, 2)) for _ in range(24)]
+    samples += [(int(b) * 64 + int(a), int(b) * 64 + int(c)) for b, a, c in rng.integers(0, 64, (24, 3))]
+    Pv = Pt.view(-1, 256)
+    for (i, j) in samples:
+        row = oracle.locate(oracle.KIND_BLOCKDIAG, 4096, i, j, nb=64, bs=64)
+        if row < 0:
+            assert int(torch.count_nonzero(dense_t[i, j])) == 0
+        else:
+            assert torch.equal(dense_t[i, j], Pv[row])
+    assert int(torch.count_nonzero(dense_t)) == int(torch.count_nonzero(Pt))
+    assert torch.equal(st.st_pack(dense_t.view(-1), lay), Pt)
+
+
+# ------------------------------------------------------------------------------ moments
+
+def expand2(st, packed, d):
+    return oracle.unpack(packed.cpu().numpy(), oracle.KIND_TRI, d, fill=oracle.FILL_SYMMETRIC).astype(np.float64)
+
+
+def expand3(st, packed, d):
+    return oracle.unpack(packed.cpu().numpy(), oracle.KIND_TET, d, fill=oracle.FILL_SYMMETRIC).astype(np.float64)
+
+
+@pytest.mark.parametrize("d", [1, 2, 3, 5, 8, 17, 64, 100, 130])
+@pytest.mark.parametrize("N", [1, 31, 32, 33, 257, 4096])
+def test_moment2_f32_small(st, N, d):
+    X = workloads.draw((N, d), "uniform", 100 + N + d)
+    T, S = oracle.moment2(X)
+    for flags in (0, st.ST_FLAG_DENSE_CONTROL):
+        got = expand2(st, st.st_sym_moment2(dev(X), flags=flags), d)
+        assert oracle.rel_err(got, T, S) <= TOL_F32, (N, d, flags)
+
+
+def test_moment2_f32_strided_rows_and_all_ones(st):
+    N, d, ldx = 300, 20, 28
+    buf = workloads.draw((N, ldx), "normal", 5)
+    Xt = dev(buf)[:, :d]
+    T, S = oracle.moment2(np.ascontiguousarray(buf[:, :d]))
+    out = torch.empty(d * (d + 1) // 2, dtype=torch.float32, device="cuda")
+    nbytes = st.st_workspace_bytes(st.ST_OP_SYM_MOMENT2, N, d, st.ST_F32)
+    ws = torch.empty(nbytes, dtype=torch.uint8, device="cuda")
+    rc = st.lib().st_sym_moment2(Xt.data_ptr(), st.ST_F32, N, d, ldx, out.data_ptr(), ws.data_ptr(), nbytes, 0,
+                                 torch.cuda.current_stream().cuda_stream)
+    assert rc == st.ST_OK
+    assert oracle.rel_err(expand2(st, out, d), T, S) <= TOL_F32
+    ones = torch.ones((777, 64), dtype=torch.float32, device="cuda")
+    assert torch.all(st.st_sym_moment2(ones) == 777.0)
+
+
+def test_moment2_config(st):
+    X = workloads.moment_input("moment2")
+    assert X.shape == (4096, 64)
+    T, S = oracle.moment2(X)
+    got = st.st_sym_moment2(dev(X))
+    assert got.numel() == 2080
+    assert oracle.rel_err(expand2(st, got, 64), T, S) <= TOL_F32
+    # two calls give the same bits (fixed-order reduction)
+    assert torch.equal(got, st.st_sym_moment2(dev(X)))
+
+
+@pytest.mark.parametrize("d", [8, 16, 24, 40, 64])
+@pytest.mark.parametrize("N", [1, 63, 64, 65, 1000])
+def test_moment3_small(st, N, d):
+    X = workloads.draw((N, d), "normal", 200 + N + d)
+    T, S = oracle.moment3(X)
+    got = st.st_sym_moment3(dev(X))
+    assert got.numel() == workloads.tet(d)
+    assert oracle.rel_err(expand3(st, got, d), T, S) <= TOL_F32, (N, d)
+
+
+def test_moment3_dense_control_and_all_ones(st):
+    X = workloads.draw((500, 32), "normal", 9)
+    T, S = oracle.moment3(X)
+    a = st.st_sym_moment3(dev(X))
+    b = st.st_sym_moment3(dev(X), flags=st.ST_FLAG_DENSE_CONTROL)
+    assert oracle.rel_err(expand3(st, b, 32), T, S) <= TOL_F32
+    assert oracle.rel_err(expand3(st, a, 32), T, S) <= TOL_F32
+    ones = torch.ones((1234, 64), dtype=torch.float32, device="cuda")
+    assert torch.all(st.st_sym_moment3(ones) == 1234.0)
+
+
+def test_moment3_config(st):
+    X = workloads.moment_input("moment3")
+    N, d = X.shape
+    assert (N, d) == (65536, 64)
+    got = st.st_sym_moment3(dev(X)).cpu().numpy()
+    assert got.size == 45760
+    # sampled entries at full N: all (i,i,i), block corners, and seeded random triples
+    rng = np.random.default_rng(42)
+    tri = [(i, i, i) for i in range(d)]
+    tri += [(a, b, c) for a in (0, 7, 8, 63) for b in (0, 7, 8, 56, 63) for c in (0, 8, 15, 56, 63) if a <= b <= c]
+    tri += [tuple(sorted(int(v) for v in rng.integers(0, d, 3))) for _ in range(3000)]
+    ii, jj, kk = (np.array(v) for v in zip(*tri))
+    T, S = oracle.moment3_at(X, ii, jj, kk)
+    pos = np.array([oracle.locate(oracle.KIND_TET, d, *t) for t in tri])
+    assert oracle.rel_err(got[pos], T, S) <= TOL_F32
+    # multiplicity identity on the whole packed output (holds at any size)
+    mult = np.array([{1: 1, 2: 3, 3: 6}[len({i, j, k})]
+                     for i in range(d) for j in range(i, d) for k in range(j, d)], np.float64)
+    lhs = float(np.dot(mult, got.astype(np.float64)))
+    Xd = X.astype(np.float64)
+    rhs = float(np.sum(Xd.sum(axis=1) ** 3))
+    scale = float(np.sum(np.abs(Xd).sum(axis=1) ** 3))
+    assert abs(lhs - rhs) <= TOL_F32 * scale
+
+
+# ------------------------------------------------------------------------------ MTTKRP / TTM
+
+@pytest.mark.parametrize("I,K,R", [(1, 4, 8), (2, 8, 16), (5, 36, 32), (16, 64, 64), (40, 100, 32), (70, 32, 8),
+                                   (33, 68, 64)])
+def test_mttkrp_small(st, I, K, R):
+    Bp, C, D = workloads.mttkrp_inputs(I, K, R)
+    Bd = oracle.unpack(Bp.reshape(-1), oracle.KIND_TRI, I, inner=K)
+    A, S = oracle.mttkrp(Bd, C, D)
+    got = st.st_mttkrp_tri(dev(Bp), dev(C), dev(D)).cpu().numpy()
+    assert oracle.rel_err(got, A, S) <= TOL_F32
+    ctl = st.st_mttkrp_tri(dev(Bd), dev(C), dev(D), flags=st.ST_FLAG_DENSE_CONTROL).cpu().numpy()
+    assert oracle.rel_err(ctl, A, S) <= TOL_F32
+
+
+def test_mttkrp_closed_form(st):
+    I, K, R = 48, 16, 32
+    Bp = torch.ones((I * (I + 1) // 2, K), device="cuda")
+    got = st.st_mttkrp_tri(Bp, torch.ones((I, R), device="cuda"), torch.ones((K, R), device="cuda")).cpu().numpy()
+    for i in range(I):
+        assert np.all(got[i] == (I - i) * K)
+
+
+def test_mttkrp_config(st):
+    Bp, C, D = workloads.mttkrp_inputs()
+    assert Bp.shape == (131328, 512) and C.shape == (512, 32)
+    got = st.st_mttkrp_tri(dev(Bp), dev(C), dev(D)).cpu().numpy()
+    Bd = oracle.unpack(Bp.reshape(-1), oracle.KIND_TRI, 512, inner=512)
+    for i0 in (0, 1, 255, 256, 300, 510, 511):
+        A, S = oracle.mttkrp(Bd, C, D, i0, i0 + 1)
+        assert oracle.rel_err(got[i0:i0 + 1], A, S) <= TOL_F32, i0
+
+
+@pytest.mark.parametrize("nb,bs,K,R", [(1, 1, 4, 8), (3, 2, 8, 16), (2, 5, 36, 32), (4, 8, 64, 64), (7, 1, 32, 64),
+                                       (2, 17, 100, 8)])
+def test_ttm_small(st, nb, bs, K, R):
+    Bp, U = workloads.ttm_inputs(nb, bs, K, R)
+    d = nb * bs
+    Bd = oracle.unpack(Bp.reshape(-1), oracle.KIND_BLOCKDIAG, d, inner=K, nb=nb, bs=bs)
+    A, S = oracle.ttm(Bd, U)
+    got = st.st_ttm_blockdiag(dev(Bp), dev(U), nb, bs).cpu().numpy()
+    got_dense = oracle.unpack(got.reshape(-1), oracle.KIND_BLOCKDIAG, d, inner=R, nb=nb, bs=bs)
+    assert oracle.rel_err(got_dense, A, S) <= TOL_F32
+    ctl = st.st_ttm_blockdiag(dev(Bd), dev(U), nb, bs, flags=st.ST_FLAG_DENSE_CONTROL).cpu().numpy()
+    assert oracle.rel_err(ctl.reshape(d, d, R), A, S) <= TOL_F32
+
+
+def test_ttm_identity_is_bit_exact(st):
+    nb, bs, K = 3, 4, 32
+    Bp, _ = workloads.ttm_inputs(nb, bs, K, 32)
+    got = st.st_ttm_blockdiag(dev(Bp), torch.eye(K, device="cuda"), nb, bs).cpu().numpy()
+    assert np.array_equal(got.view(np.uint32), Bp.reshape(-1, K).view(np.uint32))
+
+
+def test_ttm_config(st):
+    Bp, U = workloads.ttm_inputs()
+    assert Bp.shape == (64, 64, 64, 256) and U.shape == (256, 64)
+    got = st.st_ttm_blockdiag(dev(Bp), dev(U), 64, 64).cpu().numpy()
+    rng = np.random.default_rng(3)
+    rows = np.unique(np.concatenate([[0, 1, 255, 256, 4095, 4096, 262143], rng.integers(0, 262144, 500)]))
+    A, S = oracle.ttm(Bp.reshape(-1, 256)[rows], U)
+    assert oracle.rel_err(got[rows], A, S) <= TOL_F32
+    # the packed row order is the lexicographic walk of the blocks
+    for (i, j) in [(0, 0), (63, 63), (64, 64), (130, 190), (4095, 4032)]:
+        row = oracle.locate(oracle.KIND_BLOCKDIAG, 4096, i, j, nb=64, bs=64)
+        a, s = oracle.ttm(Bp.reshape(-1, 256)[row:row + 1], U)
+        assert oracle.rel_err(got[row:row + 1], a, s) <= TOL_F32

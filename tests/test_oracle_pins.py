@@ -110,6 +110,16 @@ def test_moment3_einsum_permutations_and_multiplicity_identity():
     assert abs(acc - T.sum()) < 1e-8
 
 
+def test_moment3_at_matches_definition_on_samples():
+    X = rnd((90, 6), 17)
+    Xd = X.astype(np.float64)
+    ii, jj, kk = np.array([0, 1, 5, 2]), np.array([0, 3, 5, 2]), np.array([0, 4, 5, 5])
+    T, S = oracle.moment3_at(X, ii, jj, kk)
+    full = np.einsum("ni,nj,nk->ijk", Xd, Xd, Xd)
+    np.testing.assert_allclose(T, full[ii, jj, kk], rtol=1e-12, atol=1e-12)
+    np.testing.assert_allclose(S, np.einsum("ni,nj,nk->ijk", *(np.abs(Xd),) * 3)[ii, jj, kk], rtol=1e-12)
+
+
 def test_moment3_d1_is_sum_of_cubes():
     X = rnd((64, 1), 2)
     T, S = oracle.moment3(X)
