@@ -74,6 +74,25 @@ def draw_rows(N: int, d: int, dist: str, seed: int, chunk: int = 1 << 16) -> np.
     return out
 
 
+def draw_rows_bf16(N: int, d: int, dist: str, seed: int, chunk: int = 1 << 16) -> np.ndarray:
+    """bfloat16 bit patterns (uint16) of draw_rows(N, d, dist, seed), produced chunk by chunk so
+    that the float32 array is never held whole."""
+    out = np.empty((N, d), np.uint16)
+    rng = np.random.default_rng(seed)
+    for r0 in range(0, N, chunk):
+        r1 = min(N, r0 + chunk)
+        if dist == "uniform":
+            blk = rng.random((r1 - r0, d), dtype=np.float32)
+            blk *= 2.0
+            blk -= 1.0
+        elif dist == "normal":
+            blk = rng.standard_normal((r1 - r0, d), dtype=np.float32)
+        else:
+            raise ValueError(dist)
+        out[r0:r1] = f32_to_bf16_bits(blk)
+    return out
+
+
 def f32_to_bf16_bits(a: np.ndarray) -> np.ndarray:
     """Round-to-nearest-even float32 -> bfloat16, returned as uint16 bit patterns."""
     u = np.ascontiguousarray(a, dtype=np.float32).view(np.uint32)
