@@ -1,9 +1,246 @@
-// placeholder
-#include "st_common.cuh"
+// st_sym_moment2, tensor-core path: out[p(i,j)] = sum_n X[n,i] X[n,j], X in bfloat16, fp32
+// accumulation (Section 3, M1; the outer product summed over samples is a symmetric
+// rank-N update, i.e. a triangular tile GEMM X^T X).
+//
+// Output tiles of 128 (i) x 256 (j) that contain at least one entry with i <= j are the only
+// tiles launched; tiles wholly below the diagonal are never issued.  The sample range is
+// split over blocks so that tiles x splits fills the SMs; every block accumulates its tile
+// over its samples in tensor memory and writes an fp32 partial tile; a second kernel adds
+// the partials of a tile in fixed order and writes the packed upper triangle.
+//
+// Both operands of X^T X are "MN-major" for the tensor core: X is [N, d] row-major, so the
+// output index (i or j) is contiguous and the reduction index n strides by a row.  TMA
+// loads boxes of 64 columns x 64 rows with the 128-byte swizzle, which is exactly the
+// canonical MN-major layout of tcgen05 (8 rows x 128 bytes per swizzle atom).  When the
+// 128 columns of the A panel lie inside the 256 columns of the B panel (tiles on the
+// diagonal) only the B panel is loaded and A aliases it.
+//
+// Warp roles (192 threads): warp 0 = TMA producer, warp 1 = MMA issuer and TMEM owner,
+// warps 2..5 = epilogue (TMEM -> registers -> global), one per 32-lane quarter of TMEM.
+#include "tc_common.cuh"
+#include "st_index.cuh"
+
 namespace st {
-st_status moment2_bf16_tc(const void *, int64_t, int64_t, int64_t, float *, void *, size_t, unsigned, cudaStream_t)
+
+namespace m2tc {
+constexpr int BM = 128, BN = 256;
+constexpr int KROWS = 64;                       // sample rows per pipeline stage
+constexpr int BOXC = 64;                        // columns per TMA box (128 bytes of bf16)
+constexpr int BOX_BYTES = BOXC * KROWS * 2;     // 8 KiB
+constexpr int NBOX_A = BM / BOXC, NBOX_B = BN / BOXC;
+constexpr int STAGE_BYTES = (NBOX_A + NBOX_B) * BOX_BYTES;   // 48 KiB
+constexpr int STAGES = 4;
+constexpr int THREADS = 192;
+constexpr int MAX_TILES = 288;
+constexpr uint32_t TMEM_COLS = 256;
+constexpr size_t SMEM_BYTES = (size_t)STAGES * STAGE_BYTES + 1024 /*align*/ + 256 /*barriers*/;
+
+struct TileTable {
+    int ntiles;
+    unsigned short tm[MAX_TILES];
+    unsigned short tn[MAX_TILES];
+};
+}  // namespace m2tc
+
+__global__ void __launch_bounds__(m2tc::THREADS, 1)
+moment2_tc_kernel(const __grid_constant__ CUtensorMap tmap, float *__restrict__ partials, unsigned *status,
+                  int nsplit, int chunks_total, int chunks_per_split, const __grid_constant__ m2tc::TileTable tab)
 {
-    return ST_ERR_UNSUPPORTED;
+    using namespace m2tc;
+    using namespace tc;
+    extern __shared__ unsigned char smem_raw[];
+    unsigned char *smem = (unsigned char *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+    uint64_t *bars = (uint64_t *)(smem + (size_t)STAGES * STAGE_BYTES);
+    uint64_t *full = bars, *empty = bars + STAGES, *accum = bars + 2 * STAGES;
+    uint32_t *tmem_slot = (uint32_t *)(bars + 2 * STAGES + 1);
+    volatile int *abort_flag = (volatile int *)(tmem_slot + 1);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int tile = blockIdx.x / nsplit, split = blockIdx.x - tile * nsplit;
+    const int tm = tab.tm[tile], tn = tab.tn[tile];
+    const bool a_in_b = (tm >> 1) == tn;
+    const int c_begin = split * chunks_per_split;
+    int c_end = c_begin + chunks_per_split;
+    if (c_end > chunks_total) c_end = chunks_total;
+    const int nchunks = c_end > c_begin ? c_end - c_begin : 0;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < STAGES; ++s) {
+            mbar_init(&full[s], 1);
+            mbar_init(&empty[s], 1);
+        }
+        mbar_init(accum, 1);
+        *abort_flag = 0;
+        fence_barrier_init();
+    }
+    if (warp == 1) {
+        tmem_alloc(tmem_slot, TMEM_COLS);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    if (warp == 0) {
+        // ---------------- TMA producer
+        if (elect_one()) {
+            prefetch_tmap(&tmap);
+            const uint32_t tx = (uint32_t)((a_in_b ? NBOX_B : NBOX_A + NBOX_B) * BOX_BYTES);
+            for (int c = 0; c < nchunks; ++c) {
+                const int s = c % STAGES;
+                if (c >= STAGES && !mbar_wait(&empty[s], ((c / STAGES) - 1) & 1, abort_flag, status, 1)) break;
+                unsigned char *st_base = smem + (size_t)s * STAGE_BYTES;
+                mbar_expect_tx(&full[s], tx);
+                const int row = (c_begin + c) * KROWS;
+                for (int b = 0; b < NBOX_B; ++b)
+                    tma_load_2d(st_base + b * BOX_BYTES, &tmap, &full[s], tn * BN + b * BOXC, row);
+                if (!a_in_b)
+                    for (int b = 0; b < NBOX_A; ++b)
+                        tma_load_2d(st_base + (NBOX_B + b) * BOX_BYTES, &tmap, &full[s], tm * BM + b * BOXC, row);
+            }
+        }
+    } else if (warp == 1) {
+        // ---------------- MMA issuer
+        if (elect_one()) {
+            constexpr uint32_t idesc = make_idesc(1, 1, 1, BM, BN);
+            const uint32_t a_off = a_in_b ? (uint32_t)((tm & 1) * NBOX_A * BOX_BYTES) : (uint32_t)(NBOX_B * BOX_BYTES);
+            for (int c = 0; c < nchunks; ++c) {
+                const int s = c % STAGES;
+                if (!mbar_wait(&full[s], (c / STAGES) & 1, abort_flag, status, 2)) break;
+                tc_fence_after();
+                const uint32_t sb = smem_u32(smem + (size_t)s * STAGE_BYTES);
+#pragma unroll
+                for (int k = 0; k < KROWS / 16; ++k) {
+                    // 16 rows = two swizzle atoms of 8 rows x 128 bytes
+                    const uint64_t bdesc = make_smem_desc(sb + k * 2048, BOX_BYTES, 1024);
+                    const uint64_t adesc = make_smem_desc(sb + a_off + k * 2048, BOX_BYTES, 1024);
+                    mma_bf16(tmem_base, adesc, bdesc, idesc, (c > 0 || k > 0) ? 1u : 0u);
+                }
+                tc_commit(&empty[s]);      // frees the stage when these MMAs have read it
+            }
+            tc_commit(accum);              // accumulator complete
+        }
+    } else {
+        // ---------------- epilogue: TMEM lanes 32q..32q+31 belong to warp q = warp % 4
+        const int q = warp & 3;
+        const bool ok = mbar_wait(accum, 0, abort_flag, status, 3);
+        tc_fence_after();
+        if (ok) {
+            float *dst = partials + ((size_t)blockIdx.x * BM + (q * 32 + lane)) * BN;
+#pragma unroll 1
+            for (int c0 = 0; c0 < BN; c0 += 32) {
+                uint32_t r[32];
+                tmem_ld_32x32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)c0, r);
+                tmem_ld_wait();
+                if (nchunks == 0) {
+#pragma unroll
+                    for (int e = 0; e < 32; ++e) r[e] = 0u;
+                }
+#pragma unroll
+                for (int e = 0; e < 32; e += 4)
+                    *reinterpret_cast<uint4 *>(dst + c0 + e) = make_uint4(r[e], r[e + 1], r[e + 2], r[e + 3]);
+            }
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc(tmem_base, TMEM_COLS);
+    }
 }
-size_t moment2_bf16_tc_workspace(int64_t, int64_t, unsigned) { return 0; }
+
+// out[p(i,j)] = sum over splits of the partial tiles, i <= j only.
+__global__ void __launch_bounds__(256)
+moment2_tc_reduce_kernel(const float *__restrict__ partials, float *__restrict__ out, int d, int nsplit,
+                         const __grid_constant__ m2tc::TileTable tab)
+{
+    using namespace m2tc;
+    const int tile = blockIdx.x;
+    const int tm = tab.tm[tile], tn = tab.tn[tile];
+    const float *base = partials + (size_t)tile * nsplit * (BM * BN);
+    for (int e = blockIdx.y * 256 + threadIdx.x; e < BM * BN; e += gridDim.y * 256) {
+        const int r = e / BN, c = e - r * BN;
+        const int gi = tm * BM + r, gj = tn * BN + c;
+        if (gi < d && gj < d && gi <= gj) {
+            float s = 0.f;
+            for (int k = 0; k < nsplit; ++k) s += __ldcg(&base[(size_t)k * (BM * BN) + e]);
+            out[tri_encode(d, gi, gj)] = s;
+        }
+    }
+}
+
+struct M2TcPlan {
+    m2tc::TileTable tab;
+    int nsplit, chunks_total, chunks_per_split;
+    size_t partial_bytes;
+    bool ok;
+};
+
+static M2TcPlan m2tc_plan(int64_t N, int64_t d, unsigned flags)
+{
+    using namespace m2tc;
+    M2TcPlan p;
+    p.ok = false;
+    const int ntm = (int)((d + BM - 1) / BM), ntn = (int)((d + BN - 1) / BN);
+    int n = 0;
+    for (int tn = 0; tn < ntn; ++tn)
+        for (int tm = 0; tm < ntm; ++tm) {
+            const bool touches_upper = (int64_t)tm * BM <= (int64_t)tn * BN + BN - 1;
+            if (!touches_upper && !(flags & ST_FLAG_DENSE_CONTROL)) continue;
+            if (n >= MAX_TILES) return p;
+            p.tab.tm[n] = (unsigned short)tm;
+            p.tab.tn[n] = (unsigned short)tn;
+            ++n;
+        }
+    p.tab.ntiles = n;
+    for (int i = n; i < MAX_TILES; ++i) p.tab.tm[i] = p.tab.tn[i] = 0;
+    const int64_t chunks = (N + KROWS - 1) / KROWS;
+    if (chunks > (int64_t(1) << 30)) return p;
+    int64_t split = sm_count_or_default() / n;
+    if (split < 1) split = 1;
+    if (split > chunks) split = chunks;
+    p.chunks_total = (int)chunks;
+    p.chunks_per_split = (int)((chunks + split - 1) / split);
+    p.nsplit = (int)((chunks + p.chunks_per_split - 1) / p.chunks_per_split);
+    p.partial_bytes = (size_t)n * p.nsplit * BM * BN * sizeof(float);
+    p.ok = true;
+    return p;
+}
+
+size_t moment2_bf16_tc_workspace(int64_t N, int64_t d, unsigned flags)
+{
+    if (N <= 0 || d <= 0 || d % 8 != 0 || d > 4096 || N > (int64_t(1) << 31) - 64) return 0;
+    const M2TcPlan p = m2tc_plan(N, d, flags);
+    return p.ok ? kWsHeaderBytes + p.partial_bytes : 0;
+}
+
+st_status moment2_bf16_tc(const void *X, int64_t N, int64_t d, int64_t ldx, float *out, void *ws, size_t ws_bytes,
+                          unsigned flags, cudaStream_t stream)
+{
+    using namespace m2tc;
+    if (d % 8 != 0 || ldx % 8 != 0) return ST_ERR_ALIGN;
+    if (d > 4096 || N > (int64_t(1) << 31) - 64) return ST_ERR_UNSUPPORTED;
+    const M2TcPlan p = m2tc_plan(N, d, flags);
+    if (!p.ok) return ST_ERR_UNSUPPORTED;
+    const size_t need = kWsHeaderBytes + p.partial_bytes;
+    if (!ws || ws_bytes < need) return ST_ERR_WORKSPACE;
+    if (!aligned256(ws)) return ST_ERR_ALIGN;
+    CUtensorMap tmap;
+    if (!tc::make_tmap_2d(&tmap, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, X, (uint64_t)N, (uint64_t)d, (uint64_t)ldx * 2,
+                          BOXC, KROWS))
+        return ST_ERR_CUDA;
+    if (cudaMemsetAsync(ws, 0, kWsHeaderBytes, stream) != cudaSuccess) return ST_ERR_CUDA;
+    float *partials = (float *)((unsigned char *)ws + kWsHeaderBytes);
+    if (cudaFuncSetAttribute(moment2_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES) !=
+        cudaSuccess)
+        return ST_ERR_CUDA;
+    moment2_tc_kernel<<<p.tab.ntiles * p.nsplit, THREADS, SMEM_BYTES, stream>>>(
+        tmap, partials, (unsigned *)ws, p.nsplit, p.chunks_total, p.chunks_per_split, p.tab);
+    if (cudaGetLastError() != cudaSuccess) return ST_ERR_CUDA;
+    moment2_tc_reduce_kernel<<<dim3(p.tab.ntiles, 8), 256, 0, stream>>>(partials, out, (int)d, p.nsplit, p.tab);
+    return launch_status();
+}
+
 }  // namespace st

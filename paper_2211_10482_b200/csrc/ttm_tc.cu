@@ -1,9 +1,232 @@
-// placeholder
-#include "st_common.cuh"
+// st_ttm_blockdiag, tensor-core path (ST_FLAG_TC_TF32): Ap[m, r] = sum_k Bp[m, k] U[k, r] over
+// the fibres of the diagonal blocks only (Table 1, TTM; B is a direct sum of blocks).  In the
+// packed layout the whole operation is one tall-skinny GEMM [rows, K] x [K, R]; what the
+// structure buys is that the fibres of the zero blocks are never read.  HBM bound.
+//
+// Persistent blocks walk tiles of 128 packed fibres.  Per tile, K is streamed in slices of 32
+// floats by TMA (128-byte swizzle, K-major A operand read as TF32 by the tensor core: the low
+// 13 mantissa bits are ignored).  U is rounded to TF32, transposed once per block into the
+// same swizzled K-major form and stays in shared memory.  The 128 x R fp32 accumulator lives
+// in tensor memory, double buffered so that the epilogue of one tile overlaps the MMAs of the
+// next.  Warp roles: warp 0 TMA producer, warp 1 MMA issuer / TMEM owner, warps 2..5 epilogue.
+#include "tc_common.cuh"
+
 namespace st {
-st_status ttm_tf32_tc(const float *, int64_t, int64_t, const float *, int64_t, float *, void *, size_t, cudaStream_t)
+
+namespace ttmtc {
+constexpr int BM = 128;                    // fibres per tile
+constexpr int KC = 32;                     // floats per k-slice (128 bytes)
+constexpr int STAGE_BYTES = BM * KC * 4;   // 16 KiB
+constexpr int THREADS = 192;
+constexpr int MAX_STAGES = 6;
+}  // namespace ttmtc
+
+struct TtmTcArgs {
+    const float *U;
+    float *out;
+    unsigned *status;
+    int64_t rows;
+    int K, R, kchunks, ntiles, stages;
+    uint32_t tmem_cols;
+};
+
+__global__ void __launch_bounds__(ttmtc::THREADS, 1)
+ttm_tc_kernel(const __grid_constant__ CUtensorMap tmap, const TtmTcArgs a)
 {
-    return ST_ERR_UNSUPPORTED;
+    using namespace ttmtc;
+    using namespace tc;
+    extern __shared__ unsigned char smem_raw[];
+    unsigned char *smem = (unsigned char *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+    const int u_region = a.R * 128;                                  // bytes of one k-slice of U^T (multiple of 2048)
+    unsigned char *u_smem = smem;                                    // kchunks regions
+    unsigned char *stage0 = smem + (size_t)a.kchunks * u_region;
+    uint64_t *bars = (uint64_t *)(stage0 + (size_t)a.stages * STAGE_BYTES);
+    uint64_t *full = bars, *empty = bars + MAX_STAGES, *acc_full = bars + 2 * MAX_STAGES,
+             *acc_empty = bars + 2 * MAX_STAGES + 2;
+    uint32_t *tmem_slot = (uint32_t *)(bars + 2 * MAX_STAGES + 4);
+    volatile int *abort_flag = (volatile int *)(tmem_slot + 1);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < MAX_STAGES; ++s) {
+            mbar_init(&full[s], 1);
+            mbar_init(&empty[s], 1);
+        }
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(&acc_full[b], 1);
+            mbar_init(&acc_empty[b], 4);     // one arrival per epilogue warp
+        }
+        *abort_flag = 0;
+        fence_barrier_init();
+    }
+    if (warp == 1) {
+        tmem_alloc(tmem_slot, a.tmem_cols);
+        tmem_relinquish();
+    }
+    // U^T, rounded to TF32, K-major with the 128-byte swizzle: element (r, k) of slice k/32
+    // goes to byte r*128 + ((k%32/4) ^ (r%8))*16 + (k%4)*4 of that slice's region
+    for (int e = threadIdx.x; e < a.kchunks * KC * a.R; e += THREADS) {
+        const int k = e / a.R, r = e - k * a.R;                      // consecutive threads: consecutive r (coalesced)
+        const float v = (k < a.K) ? a.U[(size_t)k * a.R + r] : 0.f;
+        uint32_t t;
+        asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(t) : "f"(v));
+        const int kc = k >> 5, kk = k & 31;
+        const int off = r * 128 + (((kk >> 2) ^ (r & 7)) << 4) + ((kk & 3) << 2);
+        *reinterpret_cast<uint32_t *>(u_smem + (size_t)kc * u_region + off) = t;
+    }
+    fence_proxy_async();      // make the generic-proxy writes of U visible to the tensor core
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    const int my_tiles = (a.ntiles > (int)blockIdx.x) ? (a.ntiles - 1 - (int)blockIdx.x) / (int)gridDim.x + 1 : 0;
+
+    if (warp == 0) {
+        if (elect_one()) {
+            prefetch_tmap(&tmap);
+            int64_t step = 0;
+            bool ok = true;
+            for (int t = 0; t < my_tiles && ok; ++t) {
+                const int64_t tile = blockIdx.x + (int64_t)t * gridDim.x;
+                for (int kc = 0; kc < a.kchunks; ++kc, ++step) {
+                    const int s = (int)(step % a.stages);
+                    const int64_t use = step / a.stages;
+                    if (use > 0 && !mbar_wait(&empty[s], (uint32_t)((use - 1) & 1), abort_flag, a.status, 1)) {
+                        ok = false;
+                        break;
+                    }
+                    mbar_expect_tx(&full[s], STAGE_BYTES);
+                    tma_load_2d(stage0 + (size_t)s * STAGE_BYTES, &tmap, &full[s], kc * KC, (int)(tile * BM));
+                }
+            }
+        }
+    } else if (warp == 1) {
+        if (elect_one()) {
+            const uint32_t idesc = make_idesc(2, 0, 0, BM, (uint32_t)a.R);
+            int64_t step = 0;
+            bool ok = true;
+            for (int t = 0; t < my_tiles && ok; ++t) {
+                const int buf = t & 1;
+                const int use = t >> 1;
+                if (use > 0 && !mbar_wait(&acc_empty[buf], (uint32_t)((use - 1) & 1), abort_flag, a.status, 2)) break;
+                tc_fence_after();
+                const uint32_t d_tmem = tmem_base + (uint32_t)(buf * a.R);
+                for (int kc = 0; kc < a.kchunks; ++kc, ++step) {
+                    const int s = (int)(step % a.stages);
+                    if (!mbar_wait(&full[s], (uint32_t)((step / a.stages) & 1), abort_flag, a.status, 3)) {
+                        ok = false;
+                        break;
+                    }
+                    tc_fence_after();
+                    const uint32_t sa = smem_u32(stage0 + (size_t)s * STAGE_BYTES);
+                    const uint32_t sb = smem_u32(u_smem + (size_t)kc * u_region);
+#pragma unroll
+                    for (int kk = 0; kk < KC / 8; ++kk) {
+                        const uint64_t adesc = make_smem_desc(sa + kk * 32, 16, 1024);
+                        const uint64_t bdesc = make_smem_desc(sb + kk * 32, 16, 1024);
+                        mma_tf32(d_tmem, adesc, bdesc, idesc, (kc > 0 || kk > 0) ? 1u : 0u);
+                    }
+                    tc_commit(&empty[s]);
+                }
+                tc_commit(&acc_full[buf]);
+            }
+        }
+    } else {
+        const int q = warp & 3;
+        for (int t = 0; t < my_tiles; ++t) {
+            const int buf = t & 1;
+            const int64_t tile = blockIdx.x + (int64_t)t * gridDim.x;
+            if (!mbar_wait(&acc_full[buf], (uint32_t)((t >> 1) & 1), abort_flag, a.status, 4)) break;
+            tc_fence_after();
+            const int64_t row = tile * BM + q * 32 + lane;
+            float *dst = a.out + row * a.R;
+            for (int c0 = 0; c0 < a.R; c0 += 32) {
+                uint32_t r[32];
+                tmem_ld_32x32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * a.R + c0), r);
+                tmem_ld_wait();
+                if (row < a.rows) {
+#pragma unroll
+                    for (int e = 0; e < 32; e += 4)
+                        if (c0 + e < a.R)
+                            *reinterpret_cast<uint4 *>(dst + c0 + e) = make_uint4(r[e], r[e + 1], r[e + 2], r[e + 3]);
+                }
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&acc_empty[buf]);
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc(tmem_base, a.tmem_cols);
+    }
 }
-size_t ttm_tf32_tc_workspace(int64_t, int64_t, int64_t) { return 0; }
+
+struct TtmTcPlan {
+    int kchunks, stages;
+    uint32_t tmem_cols;
+    size_t smem;
+    bool ok;
+};
+
+static TtmTcPlan ttm_tc_plan(int64_t K, int64_t R)
+{
+    using namespace ttmtc;
+    TtmTcPlan p{};
+    p.ok = false;
+    if (K <= 0 || R <= 0 || K % 4 != 0 || R % 16 != 0 || R > 256 || K > (1 << 20)) return p;
+    p.kchunks = (int)((K + KC - 1) / KC);
+    uint32_t cols = 32;
+    while (cols < 2 * (uint32_t)R) cols *= 2;
+    p.tmem_cols = cols;
+    const size_t u_bytes = (size_t)p.kchunks * R * 128;
+    const size_t fixed = 1024 + u_bytes + 512;
+    const size_t budget = 227 * 1024;
+    if (fixed + 2 * STAGE_BYTES > budget) return p;
+    size_t st = (budget - fixed) / STAGE_BYTES;
+    if (st > MAX_STAGES) st = MAX_STAGES;
+    p.stages = (int)st;
+    p.smem = fixed + st * STAGE_BYTES;
+    p.ok = true;
+    return p;
+}
+
+size_t ttm_tf32_tc_workspace(int64_t rows, int64_t K, int64_t R)
+{
+    if (rows <= 0) return 0;
+    return ttm_tc_plan(K, R).ok ? kWsHeaderBytes : 0;
+}
+
+st_status ttm_tf32_tc(const float *Bp, int64_t rows, int64_t K, const float *U, int64_t R, float *Ap, void *ws,
+                      size_t ws_bytes, cudaStream_t stream)
+{
+    using namespace ttmtc;
+    const TtmTcPlan p = ttm_tc_plan(K, R);
+    if (!p.ok) return ST_ERR_UNSUPPORTED;
+    if (rows > (int64_t(1) << 31) - BM) return ST_ERR_UNSUPPORTED;
+    if (!ws || ws_bytes < kWsHeaderBytes) return ST_ERR_WORKSPACE;
+    if (!aligned256(ws)) return ST_ERR_ALIGN;
+    const DeviceInfo di = device_info();
+    if (!di.ok) return ST_ERR_CUDA;
+    if (p.smem > (size_t)di.max_smem_optin) return ST_ERR_UNSUPPORTED;
+    CUtensorMap tmap;
+    if (!tc::make_tmap_2d(&tmap, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, Bp, (uint64_t)rows, (uint64_t)K, (uint64_t)K * 4, KC,
+                          BM))
+        return ST_ERR_CUDA;
+    if (cudaMemsetAsync(ws, 0, kWsHeaderBytes, stream) != cudaSuccess) return ST_ERR_CUDA;
+    TtmTcArgs a;
+    a.U = U; a.out = Ap; a.status = (unsigned *)ws; a.rows = rows; a.K = (int)K; a.R = (int)R;
+    a.kchunks = p.kchunks; a.stages = p.stages; a.tmem_cols = p.tmem_cols;
+    a.ntiles = (int)((rows + BM - 1) / BM);
+    if (cudaFuncSetAttribute(ttm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)p.smem) != cudaSuccess)
+        return ST_ERR_CUDA;
+    const int grid = a.ntiles < di.sm_count ? a.ntiles : di.sm_count;
+    ttm_tc_kernel<<<grid, THREADS, p.smem, stream>>>(tmap, a);
+    return launch_status();
+}
+
 }  // namespace st

@@ -294,3 +294,75 @@ def test_ttm_config(st):
         row = oracle.locate(oracle.KIND_BLOCKDIAG, 4096, i, j, nb=64, bs=64)
         a, s = oracle.ttm(Bp.reshape(-1, 256)[row:row + 1], U)
         assert oracle.rel_err(got[row:row + 1], a, s) <= TOL_F32
+
+
+# ------------------------------------------------------------------------------ tensor-core paths
+
+TOL_TC = 5e-3          # stated tolerance of the bf16 / TF32 tensor-core paths
+
+
+def bf16_dev(bits):
+    return torch.from_numpy(np.ascontiguousarray(bits).view(np.int16)).cuda().view(torch.bfloat16)
+
+
+@pytest.mark.parametrize("d", [64, 128, 192, 256, 320, 520])
+@pytest.mark.parametrize("N", [1, 63, 64, 65, 1000, 9000])
+def test_moment2_bf16_tensor_core_small(st, N, d):
+    X = workloads.draw((N, d), "normal", 300 + N + d)
+    bits = workloads.f32_to_bf16_bits(X).reshape(N, d)
+    Xb = workloads.bf16_bits_to_f32(bits).reshape(N, d)
+    got = expand2(st, st.st_sym_moment2(bf16_dev(bits)), d)
+    Tb, Sb = oracle.moment2(Xb)         # same rounded inputs: isolates the accumulation error
+    assert oracle.rel_err(got, Tb, Sb) <= TOL_F32, (N, d)
+    T, S = oracle.moment2(X)            # against the fp32 inputs: the stated 5e-3
+    assert oracle.rel_err(got, T, S) <= TOL_TC, (N, d)
+    ctl = expand2(st, st.st_sym_moment2(bf16_dev(bits), flags=st.ST_FLAG_DENSE_CONTROL), d)
+    assert oracle.rel_err(ctl, Tb, Sb) <= TOL_F32
+    assert st.st_check_status() == st.ST_OK
+
+
+def test_moment2_bf16_all_ones(st):
+    ones = torch.ones((3001, 256), dtype=torch.bfloat16, device="cuda")
+    assert torch.all(st.st_sym_moment2(ones) == 3001.0)
+
+
+def test_moment2_large_config(st):
+    cfg = workloads.CONFIGS["moment2_large"]
+    N, d = cfg["N"], cfg["d"]
+    bits = workloads.draw_rows_bf16(N, d, cfg["dist"], workloads.SEEDS["moment2_large"])
+    got = st.st_sym_moment2(bf16_dev(bits)).cpu().numpy()
+    assert got.size == 524800
+    Xb = workloads.bf16_bits_to_f32(bits).reshape(N, d)
+    rng = np.random.default_rng(8)
+    pairs = [(i, i) for i in range(0, d, 37)] + [(0, d - 1), (127, 128), (128, 255), (255, 256), (511, 512), (767, 1023)]
+    pairs += [tuple(sorted(int(v) for v in rng.integers(0, d, 2))) for _ in range(300)]
+    ii, jj = (np.array(v) for v in zip(*pairs))
+    T, S = oracle.moment2_at(Xb, ii, jj)
+    pos = ii * (2 * d - ii + 1) // 2 + (jj - ii)
+    for (i, j), p in list(zip(pairs, pos))[:40]:
+        assert p == oracle.locate(oracle.KIND_TRI, d, i, j)
+    assert oracle.rel_err(got[pos], T, S) <= TOL_F32
+    # trace identity on the whole diagonal (holds at any size): sum_i out[p(i,i)] = ||X||_F^2
+    diag = np.array([i * (2 * d - i + 1) // 2 for i in range(d)])
+    fro = float(np.sum(Xb.astype(np.float64) ** 2))
+    assert abs(float(got[diag].astype(np.float64).sum()) - fro) <= TOL_F32 * fro
+
+
+@pytest.mark.parametrize("nb,bs,K,R", [(1, 1, 4, 16), (3, 2, 8, 16), (2, 5, 36, 32), (4, 8, 64, 64), (7, 3, 32, 48),
+                                       (2, 17, 100, 128), (5, 12, 256, 64)])
+def test_ttm_tf32_tensor_core_small(st, nb, bs, K, R):
+    Bp, U = workloads.ttm_inputs(nb, bs, K, R)
+    A, S = oracle.ttm(Bp.reshape(-1, K), U)
+    got = st.st_ttm_blockdiag(dev(Bp), dev(U), nb, bs, flags=st.ST_FLAG_TC_TF32).cpu().numpy()
+    assert oracle.rel_err(got, A, S) <= TOL_TC
+    assert st.st_check_status() == st.ST_OK
+
+
+def test_ttm_tf32_config(st):
+    Bp, U = workloads.ttm_inputs()
+    got = st.st_ttm_blockdiag(dev(Bp), dev(U), 64, 64, flags=st.ST_FLAG_TC_TF32).cpu().numpy()
+    rng = np.random.default_rng(4)
+    rows = np.unique(np.concatenate([[0, 1, 127, 128, 4095, 4096, 262143], rng.integers(0, 262144, 600)]))
+    A, S = oracle.ttm(Bp.reshape(-1, 256)[rows], U)
+    assert oracle.rel_err(got[rows], A, S) <= TOL_TC
+    assert st.st_check_status() == st.ST_OK
