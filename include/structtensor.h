@@ -56,7 +56,9 @@ typedef enum {
     ST_ERR_UNSUPPORTED = 6,  /* well-formed request outside what the kernels cover */
     ST_ERR_CUDA = 7,         /* a CUDA runtime / driver call failed */
     ST_ERR_DEV_TIMEOUT = 8,  /* a bounded wait inside a kernel ran out (see st_check_status) */
-    ST_ERR_DEV_BOUNDS = 9    /* a kernel-side consistency check failed */
+    ST_ERR_DEV_BOUNDS = 9,   /* a kernel-side consistency check failed */
+    ST_ERR_STATIC_SCRATCH = 10 /* st_sym_moment3_static: the request needs more scratch than the
+                                  built-in ST_STATIC_SCRATCH_BYTES */
 } st_status;
 
 typedef enum { ST_F32 = 0, ST_BF16 = 1, ST_F64 = 2 } st_dtype;
@@ -135,6 +137,32 @@ st_status st_sym_moment2(const void *X, st_dtype xdt, int64_t N, int64_t d, int6
 st_status st_sym_moment3(const float *X, int64_t N, int64_t d, int64_t ldx,
                          float *out_packed, void *ws, size_t ws_bytes, unsigned flags,
                          void *stream);
+
+/* Size of the scratch array built into the library image for st_sym_moment3_static. */
+#define ST_STATIC_SCRATCH_BYTES (16u << 20)
+
+/* st_sym_moment3 for callers that cannot allocate device memory.  (The paper has no
+ * counterpart: this is a property of the calling environment, not of the method.)
+ *
+ * Same operation, same arguments and same result as st_sym_moment3, but without the `ws`
+ * pair: the per-slice partial sums go to a 16 MiB array that is part of the library
+ * (ST_STATIC_SCRATCH_BYTES; every GPU that loads the library holds it until the process
+ * exits).  Meant for code that runs where cudaMalloc is off limits -- inside a framework's
+ * hot loop that owns the allocator, in a plug-in that is handed nothing but its input and
+ * output buffers, or in a process whose device-memory budget was fixed at start-up.  The
+ * call itself allocates and frees nothing, on the device or through any library.
+ *
+ *   - A request whose partial sums do not fit (st_workspace_bytes(ST_OP_SYM_MOMENT3, N, d)
+ *     > ST_STATIC_SCRATCH_BYTES) returns ST_ERR_STATIC_SCRATCH and launches nothing.  All
+ *     supported d (<= 64) fit on a GPU with up to 160 SMs.
+ *   - The first call on each device looks up the device address of the array (one runtime
+ *     query, no allocation); make that first call before any stream capture begins.
+ *   - All calls on a device share the one array.  Nothing in it has to be cleared between
+ *     calls (each call overwrites every partial sum it later reads), but two calls that
+ *     overlap on the GPU -- different streams, or different host threads without ordering --
+ *     race on it and give wrong results.  Order them on one stream or with events. */
+st_status st_sym_moment3_static(const float *X, int64_t N, int64_t d, int64_t ldx,
+                                float *out_packed, unsigned flags, void *stream);
 
 /* MTTKRP (Table 1) on a tensor whose unique set is the "upper half cube" of Table 1,
  * B_U(i,j,k) = (0<=i<I)*(i<=j<I)*(0<=k<K):

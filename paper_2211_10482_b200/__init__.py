@@ -19,7 +19,8 @@ LIB_PATH = os.path.join(_HERE, "libstructtensor.so")
 
 # st_status
 ST_OK, ST_ERR_NULL, ST_ERR_SHAPE, ST_ERR_ALIGN, ST_ERR_DTYPE, ST_ERR_WORKSPACE, ST_ERR_UNSUPPORTED, \
-    ST_ERR_CUDA, ST_ERR_DEV_TIMEOUT, ST_ERR_DEV_BOUNDS = range(10)
+    ST_ERR_CUDA, ST_ERR_DEV_TIMEOUT, ST_ERR_DEV_BOUNDS, ST_ERR_STATIC_SCRATCH = range(11)
+ST_STATIC_SCRATCH_BYTES = 16 << 20
 # st_dtype
 ST_F32, ST_BF16, ST_F64 = 0, 1, 2
 # st_kind
@@ -34,7 +35,7 @@ ST_FLAG_TC_TF32 = 2
 
 EXPORTS = [
     "st_packed_elems", "st_dense_elems", "st_pack", "st_unpack", "st_workspace_bytes", "st_sym_moment2",
-    "st_sym_moment3", "st_mttkrp_tri", "st_ttm_blockdiag", "st_check_status", "st_status_string",
+    "st_sym_moment3", "st_sym_moment3_static", "st_mttkrp_tri", "st_ttm_blockdiag", "st_check_status", "st_status_string",
     "st_abi_version",
 ]
 
@@ -89,13 +90,14 @@ def lib() -> ctypes.CDLL:
         L.st_workspace_bytes.restype = sz
         L.st_sym_moment2.argtypes = [vp, ci, i64, i64, i64, vp, vp, sz, cu, vp]
         L.st_sym_moment3.argtypes = [vp, i64, i64, i64, vp, vp, sz, cu, vp]
+        L.st_sym_moment3_static.argtypes = [vp, i64, i64, i64, vp, cu, vp]
         L.st_mttkrp_tri.argtypes = [vp, i64, i64, vp, vp, i64, vp, vp, sz, cu, vp]
         L.st_ttm_blockdiag.argtypes = [vp, i64, i64, i64, vp, i64, vp, vp, sz, cu, vp]
         L.st_check_status.argtypes = [vp, vp]
         L.st_status_string.argtypes = [ci]
         L.st_status_string.restype = ctypes.c_char_p
         L.st_abi_version.restype = ci
-        for name in ("st_pack", "st_unpack", "st_sym_moment2", "st_sym_moment3", "st_mttkrp_tri",
+        for name in ("st_pack", "st_unpack", "st_sym_moment2", "st_sym_moment3", "st_sym_moment3_static", "st_mttkrp_tri",
                      "st_ttm_blockdiag", "st_check_status"):
             getattr(L, name).restype = ci
         _lib = L
@@ -207,6 +209,20 @@ def st_sym_moment3(X: torch.Tensor, out: torch.Tensor | None = None, ws: torch.T
     ws = _workspace(st_workspace_bytes(ST_OP_SYM_MOMENT3, N, d, 0, 0, flags), X.device, ws)
     _check(lib().st_sym_moment3(_dev(X, "X"), N, d, X.stride(0), _dev(out, "out"), ws.data_ptr(),
                                 ws.numel() * ws.element_size(), flags, _stream()), "st_sym_moment3")
+    return out
+
+
+def st_sym_moment3_static(X: torch.Tensor, out: torch.Tensor, flags: int = 0) -> torch.Tensor:
+    """st_sym_moment3 with the library's built-in scratch, for callers that must not allocate:
+    the caller passes the input and the output tensor, and nothing is allocated here either.
+    Calls that overlap on the GPU race on the shared scratch; keep them on one stream."""
+    N, d = X.shape
+    if X.dtype != torch.float32 or out.dtype != torch.float32:
+        raise TypeError("X and out must be float32")
+    if out.numel() != d * (d + 1) * (d + 2) // 6:
+        raise ValueError("out must hold d(d+1)(d+2)/6 elements")
+    _check(lib().st_sym_moment3_static(_dev(X, "X"), N, d, X.stride(0), _dev(out, "out"), flags, _stream()),
+           "st_sym_moment3_static")
     return out
 
 

@@ -50,6 +50,7 @@ const char *st_status_string(st_status s)
     case ST_ERR_CUDA: return "CUDA call failed";
     case ST_ERR_DEV_TIMEOUT: return "a bounded wait inside a kernel ran out";
     case ST_ERR_DEV_BOUNDS: return "kernel-side consistency check failed";
+    case ST_ERR_STATIC_SCRATCH: return "request needs more scratch than the built-in static array holds";
     default: return "unknown status";
     }
 }

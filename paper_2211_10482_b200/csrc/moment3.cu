@@ -19,6 +19,7 @@
 #include "st_common.cuh"
 #include "st_index.cuh"
 #include <algorithm>
+#include <mutex>
 #include <vector>
 
 namespace st {
@@ -325,4 +326,64 @@ extern "C" st_status st_sym_moment3(const float *X, int64_t N, int64_t d, int64_
     if (flags & ST_FLAG_DENSE_CONTROL)
         return st::moment3_launch<128>(X, N, d, ldx, out_packed, ws, ws_bytes, flags, (cudaStream_t)stream);
     return st::moment3_launch<32>(X, N, d, ldx, out_packed, ws, ws_bytes, flags, (cudaStream_t)stream);
+}
+
+// ---- st_sym_moment3_static: the same kernels with built-in scratch ---------------------
+//
+// The per-slice partial sums normally live in a workspace the caller allocates.  Some callers
+// cannot allocate device memory at the point where they need the result: code running inside a
+// framework that owns the allocator and forbids cudaMalloc in its hot loop, plug-ins that are
+// handed only input and output buffers, or a process whose memory budget was fixed at start-up.
+// For them the partial sums go to an array that is part of the library image.  It is reserved
+// on every GPU that loads the library, for the lifetime of the process.
+namespace st {
+
+constexpr size_t kStaticScratchBytes = ST_STATIC_SCRATCH_BYTES;
+static __device__ __align__(256) unsigned char g_moment3_scratch[kStaticScratchBytes];
+
+// In host code `g_moment3_scratch` only names the symbol; the device address has to be asked
+// for, once per device and with that device current.
+static st_status moment3_static_scratch(void **ptr)
+{
+    static void *addr[64] = {nullptr};
+    static std::mutex lock;
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return ST_ERR_CUDA;
+    std::lock_guard<std::mutex> guard(lock);
+    if (!addr[dev]) {
+        void *p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_moment3_scratch) != cudaSuccess || !p) {
+            (void)cudaGetLastError();
+            return ST_ERR_CUDA;
+        }
+        addr[dev] = p;
+    }
+    *ptr = addr[dev];
+    return ST_OK;
+}
+
+}  // namespace st
+
+extern "C" st_status st_sym_moment3_static(const float *X, int64_t N, int64_t d, int64_t ldx, float *out_packed,
+                                           unsigned flags, void *stream)
+{
+    if (!X || !out_packed) return ST_ERR_NULL;
+    if (N <= 0 || d <= 0 || ldx < d) return ST_ERR_SHAPE;
+    if (flags & ~(ST_FLAG_DENSE_CONTROL)) return ST_ERR_UNSUPPORTED;
+    if (d < 8 || d > st::M3_MAX_D || d % 8) return ST_ERR_UNSUPPORTED;
+    if (!st::aligned16(X) || !st::aligned16(out_packed) || ldx % 4) return ST_ERR_ALIGN;
+    // the request must fit the built-in array; nothing is launched otherwise
+    const size_t need = st::moment3_workspace(N, d, flags);
+    if (need == 0) return ST_ERR_UNSUPPORTED;
+    if (need > st::kStaticScratchBytes) return ST_ERR_STATIC_SCRATCH;
+    void *scratch = nullptr;
+    const st_status rc = st::moment3_static_scratch(&scratch);
+    if (rc != ST_OK) return rc;
+    // every partial sum that the second kernel reads is written by the first one in the same
+    // call, so nothing in the array has to start at zero
+    if (flags & ST_FLAG_DENSE_CONTROL)
+        return st::moment3_launch<128>(X, N, d, ldx, out_packed, scratch, st::kStaticScratchBytes, flags,
+                                       (cudaStream_t)stream);
+    return st::moment3_launch<32>(X, N, d, ldx, out_packed, scratch, st::kStaticScratchBytes, flags,
+                                  (cudaStream_t)stream);
 }
