@@ -8,9 +8,9 @@
 //   MTTKRP  m = p(i,j) runs over i<=j only; W = D; then A[i,r] += C[j,r] * Y[m,r], the
 //           product with C hoisted out of the k loop (Section 5.5, loop-invariant code motion).
 //
-// A thread block owns tiles of 256 consecutive fibres; 256 threads each keep TM x 8 sums
-// (TM = R/8) in registers.  Fibres are streamed through a 3-stage cp.async pipeline in
-// slices of 32 k-values; work items (tile, k-split) are walked in one flattened loop so the
+// A thread block owns tiles of consecutive fibres (256 for R=64 and R<=16, 512 for R=32); 256
+// threads each keep TM x 8 sums in registers (TM = 8 for R >= 32).  Fibres are streamed through
+// a cp.async pipeline in slices of 32 k-values; work items (tile, k-split) are walked in one flattened loop so the
 // pipeline never drains between tiles.  MTTKRP splits k over work items when that evens out
 // the load (its output is a sum over k anyway) and reduces over j with shared-memory
 // accumulators per tile followed by one global atomic per (i,r).
@@ -23,11 +23,9 @@ st_status ttm_tf32_tc(const float *Bp, int64_t rows, int64_t K, const float *U, 
                       size_t ws_bytes, cudaStream_t stream);
 
 constexpr int RG_THREADS = 256;
-constexpr int RG_ROWS = 256;      // fibres per tile
 constexpr int RG_KC = 32;         // k-values per stage
 constexpr int RG_LD = RG_KC + 4;  // padded row stride (floats) of a stage
-constexpr int RG_STAGES = 3;
-constexpr int RG_NI = 32;         // rows of A accumulated in shared memory per tile
+constexpr int RG_NI = 40;         // rows of A accumulated in shared memory per tile
 
 enum { RG_TTM = 0, RG_MTTKRP_PACKED = 1, RG_MTTKRP_DENSE = 2 };
 
@@ -48,15 +46,16 @@ struct RgArgs {
     int tiles, ksplit, kchunks_per_split, kchunks;
 };
 
-template <int TM, int MODE>
+// TM rows x 8 columns per thread, CT column threads (R = 8*CT), RG_ROWS = 256/CT*TM fibres per tile.
+template <int TM, int CT, int RG_STAGES, int MODE>
 __global__ void __launch_bounds__(RG_THREADS, 1) rowgemm_kernel(const RgArgs a)
 {
+    constexpr int RG_ROWS = RG_THREADS / CT * TM;
     extern __shared__ __align__(16) float smem[];
     float *Ws = smem;                                   // [kchunks*RG_KC][R], rows >= K are zero
     float *Bs = Ws + (size_t)a.kchunks * RG_KC * a.R;   // RG_STAGES x [RG_ROWS][RG_LD]
     float *As = Bs + RG_STAGES * RG_ROWS * RG_LD;       // MTTKRP: [RG_NI][R]
-    constexpr int R_ = TM * 8;
-    constexpr int CT = R_ / 8;                          // column threads
+    constexpr int R_ = CT * 8;
     constexpr int RT = RG_THREADS / CT;                 // row threads; thread rows = tr + a*RT
     const int tid = threadIdx.x;
     const int tc = tid % CT, tr = tid / CT;
@@ -152,25 +151,51 @@ __global__ void __launch_bounds__(RG_THREADS, 1) rowgemm_kernel(const RgArgs a)
                 (void)j_first;
                 for (int e = tid; e < RG_NI * R_; e += RG_THREADS) As[e] = 0.f;
                 __syncthreads();
+                // A warp holds, for each i, 32/CT consecutive fibres (8 columns per lane).  When they
+                // all belong to one row of A (the usual case: a row of A owns I-i consecutive fibres)
+                // they are summed with shuffles and one lane per column group adds the result to the
+                // shared accumulator; otherwise every lane adds its own fibre.
+                const int lane = tid & 31;
 #pragma unroll
                 for (int i = 0; i < TM; ++i) {
                     const int64_t row = row0 + tr + i * RT;
-                    if (row < a.rows) {
-                        int64_t gi, gj;
+                    const bool valid = row < a.rows;
+                    int64_t gi = -1, gj = 0;
+                    if (valid) {
                         if (MODE == RG_MTTKRP_PACKED) tri_decode(a.I, row, gi, gj);
                         else { gi = row / a.I; gj = row - gi * a.I; }
+                    }
+                    float v[8];
+                    if (valid) {
                         const float4 c0 = *reinterpret_cast<const float4 *>(a.C + gj * R_ + tc * 8);
                         const float4 c1 = *reinterpret_cast<const float4 *>(a.C + gj * R_ + tc * 8 + 4);
                         const float cv[8] = {c0.x, c0.y, c0.z, c0.w, c1.x, c1.y, c1.z, c1.w};
+#pragma unroll
+                        for (int j = 0; j < 8; ++j) v[j] = cv[j] * acc[i][j];
+                    } else {
+#pragma unroll
+                        for (int j = 0; j < 8; ++j) v[j] = 0.f;
+                    }
+                    const int gi32 = (int)gi;
+                    const int gi_first = __shfl_sync(0xffffffffu, gi32, 0);
+                    const int gi_last = __shfl_sync(0xffffffffu, gi32, 31);
+                    const bool uniform = (gi_first == gi_last) && gi_first >= 0;
+                    if (uniform) {
+#pragma unroll
+                        for (int off = CT; off < 32; off <<= 1)
+#pragma unroll
+                            for (int j = 0; j < 8; ++j) v[j] += __shfl_xor_sync(0xffffffffu, v[j], off);
+                    }
+                    if (valid && (!uniform || lane < CT)) {
                         const int li = (int)(gi - i_first);
                         if (li < RG_NI) {
                             float *dst = As + li * R_ + tc * 8;
 #pragma unroll
-                            for (int j = 0; j < 8; ++j) atomicAdd(dst + j, cv[j] * acc[i][j]);
+                            for (int j = 0; j < 8; ++j) atomicAdd(dst + j, v[j]);
                         } else {
                             float *dst = a.out + gi * R_ + tc * 8;
 #pragma unroll
-                            for (int j = 0; j < 8; ++j) atomicAdd(dst + j, cv[j] * acc[i][j]);
+                            for (int j = 0; j < 8; ++j) atomicAdd(dst + j, v[j]);
                         }
                     }
                 }
@@ -190,10 +215,21 @@ __global__ void __launch_bounds__(RG_THREADS, 1) rowgemm_kernel(const RgArgs a)
     asm volatile("cp.async.wait_group 0;\n" ::);
 }
 
+// tile shape by R: {TM, stages}; rows per tile = 256 / (R/8) * TM
+static void rowgemm_shape(int64_t R, int &tm, int &stages)
+{
+    if (R == 64) { tm = 8; stages = 3; }
+    else if (R == 32) { tm = 8; stages = 2; }
+    else { tm = (int)R / 8; stages = 3; }
+}
+
 static size_t rowgemm_smem(int64_t K, int64_t R)
 {
+    int tm, stages;
+    rowgemm_shape(R, tm, stages);
+    const size_t rows = (size_t)RG_THREADS / (R / 8) * tm;
     const size_t kpad = (size_t)((K + RG_KC - 1) / RG_KC) * RG_KC;
-    return (kpad * R + (size_t)RG_STAGES * RG_ROWS * RG_LD + (size_t)RG_NI * R) * sizeof(float);
+    return (kpad * R + (size_t)stages * rows * RG_LD + (size_t)RG_NI * R) * sizeof(float);
 }
 
 template <int MODE>
@@ -205,7 +241,10 @@ static st_status rowgemm_launch(const RgArgs &a0, cudaStream_t stream)
     const size_t smem = rowgemm_smem(a.K, a.R);
     if (smem > (size_t)di.max_smem_optin) return ST_ERR_UNSUPPORTED;
     a.kchunks = (a.K + RG_KC - 1) / RG_KC;
-    a.tiles = (int)((a.rows + RG_ROWS - 1) / RG_ROWS);
+    int tm, stages;
+    rowgemm_shape(a.R, tm, stages);
+    const int64_t tile_rows = (int64_t)RG_THREADS / (a.R / 8) * tm;
+    a.tiles = (int)((a.rows + tile_rows - 1) / tile_rows);
     a.ksplit = 1;
     if (MODE != RG_TTM) {
         // pick the k-split that wastes the fewest SM slots in the last wave
@@ -228,10 +267,10 @@ static st_status rowgemm_launch(const RgArgs &a0, cudaStream_t stream)
         return launch_status();
     };
     switch (a.R) {
-    case 8: return run(rowgemm_kernel<1, MODE>);
-    case 16: return run(rowgemm_kernel<2, MODE>);
-    case 32: return run(rowgemm_kernel<4, MODE>);
-    case 64: return run(rowgemm_kernel<8, MODE>);
+    case 8: return run(rowgemm_kernel<1, 1, 3, MODE>);
+    case 16: return run(rowgemm_kernel<2, 2, 3, MODE>);
+    case 32: return run(rowgemm_kernel<8, 4, 2, MODE>);
+    case 64: return run(rowgemm_kernel<8, 8, 3, MODE>);
     default: return ST_ERR_UNSUPPORTED;
     }
 }
@@ -251,7 +290,7 @@ st_status st_ttm_blockdiag(const float *Bp, int64_t nblocks, int64_t bs, int64_t
     if (nblocks > (int64_t(1) << 24) || bs > (int64_t(1) << 15) || K > (1 << 20)) return ST_ERR_UNSUPPORTED;
     const int64_t d = nblocks * bs;
     const int64_t rows = (flags & ST_FLAG_DENSE_CONTROL) ? d * d : nblocks * bs * bs;
-    if (rows / RG_ROWS + 1 > (int64_t(1) << 28)) return ST_ERR_UNSUPPORTED;
+    if (rows / 256 + 1 > (int64_t(1) << 28)) return ST_ERR_UNSUPPORTED;
     if (flags & ST_FLAG_TC_TF32) return ttm_tf32_tc(Bp, rows, K, U, R, Ap, ws, ws_bytes, (cudaStream_t)stream);
     if (K % 4 != 0) return ST_ERR_UNSUPPORTED;
     if (R != 8 && R != 16 && R != 32 && R != 64) return ST_ERR_UNSUPPORTED;

@@ -141,16 +141,28 @@ moment2_f32_kernel(const float *__restrict__ X, int64_t N, int d, int64_t ldx, f
     if (!s_last) return;
     __threadfence();
 
-    // last arrival: fixed-order sum of the partial tiles, written to the packed upper triangle
+    // last arrival: fixed-order sum of the partial tiles, written to the packed upper triangle.
+    // Four columns per thread and eight independent loads in flight hide the L2 latency.
     const float *base = partials + (size_t)tile * nsplit * (M2_T * M2_T);
-    for (int e = tid; e < M2_T * M2_T; e += 256) {
-        const int r = e >> 6, c = e & 63;
+    for (int e4 = tid; e4 < M2_T * M2_T / 4; e4 += 256) {
+        const int r = e4 >> 4, c = (e4 & 15) << 2;
         const int gi = col_a + r, gj = col_b + c;
-        if (gi < d && gj < d && gi <= gj) {
-            float s = 0.f;
-            for (int k = 0; k < nsplit; ++k) s += __ldcg(&base[(size_t)k * (M2_T * M2_T) + e]);
-            out[tri_encode(d, gi, gj)] = s;
+        if (gi >= d || gj >= d || gj + 3 < gi) continue;       // nothing of this group is in i <= j
+        float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
+        const float4 *p4 = reinterpret_cast<const float4 *>(base) + e4;
+        for (int k0 = 0; k0 < nsplit; k0 += 8) {
+            float4 v[8];                                        // eight loads issued before the first add
+#pragma unroll
+            for (int u = 0; u < 8; ++u)
+                v[u] = (k0 + u < nsplit) ? __ldcg(p4 + (size_t)(k0 + u) * (M2_T * M2_T / 4))
+                                         : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+            for (int u = 0; u < 8; ++u) { s.x += v[u].x; s.y += v[u].y; s.z += v[u].z; s.w += v[u].w; }
         }
+        const float sv[4] = {s.x, s.y, s.z, s.w};
+#pragma unroll
+        for (int q = 0; q < 4; ++q)
+            if (gj + q < d && gi <= gj + q) out[tri_encode(d, gi, gj + q)] = sv[q];
     }
 }
 

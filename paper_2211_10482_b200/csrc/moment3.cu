@@ -6,7 +6,8 @@
 // one tile for a slice of the samples and keeps its <= 64 sums in registers; per sample it
 // reads x_i, the 8 x_j and the 8 x_k of the row from shared memory, forms the pair product
 // p = x_i * x_j once per j (loop-invariant code motion of Section 5.5 applied to the k loop)
-// and issues one FMA per unique triple -- nothing outside i<=j<=k is computed:
+// and issues one FMA per unique triple (two per packed f32x2 instruction; on a triangular
+// tile a pair that straddles k = j carries one unused lane) -- no other work outside i<=j<=k:
 //     variant 0        full 8x8 tile            (jb > block(i) or i at a block start, kb > jb)
 //     variant 1        triangular, k >= j       (kb == jb; rows j < i are not stored)
 //     variant 1+s      rows j >= i only, s=i%8  (jb == block(i), kb > jb), s = 1..7
@@ -51,9 +52,29 @@ __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_gr
 // 8b..8b+3 of block b sit at floats 4b.., columns 8b+4..8b+7 at floats 4*nbk+4b.., so that a
 // 128-bit load of "the first (second) half of block b" by lanes with arbitrary b touches
 // each bank once.
+// Packed fp32 pairs: sm_100 executes fma.rn.f32x2 on a 64-bit register pair, which halves the
+// issue slots per FMA and leaves room for the shared-memory loads and the pair products.
+__device__ __forceinline__ uint64_t pack2(float lo, float hi)
+{
+    uint64_t r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+__device__ __forceinline__ void unpack2(uint64_t v, float &lo, float &hi)
+{
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ uint64_t ffma2(uint64_t a, uint64_t b, uint64_t c)
+{
+    uint64_t d;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+    return d;
+}
+
+// One stage of rows for one tile.  acc[a][c] holds the sums for j = a, k = 2c and 2c+1.
 template <int J0, bool DIAG>
 __device__ __forceinline__ void m3_stage(const float *__restrict__ xs, int d, int pi, int oj, int ok, int half,
-                                         float (&acc)[8][8])
+                                         uint64_t (&acc)[8][4])
 {
 #pragma unroll 2
     for (int r = 0; r < M3_STAGE_ROWS; ++r) {
@@ -70,12 +91,13 @@ __device__ __forceinline__ void m3_stage(const float *__restrict__ xs, int d, in
             kb = *reinterpret_cast<const float4 *>(row + ok + half);
         }
         const float xj[8] = {ja.x, ja.y, ja.z, ja.w, jb.x, jb.y, jb.z, jb.w};
-        const float xk[8] = {ka.x, ka.y, ka.z, ka.w, kb.x, kb.y, kb.z, kb.w};
+        const uint64_t xk[4] = {pack2(ka.x, ka.y), pack2(ka.z, ka.w), pack2(kb.x, kb.y), pack2(kb.z, kb.w)};
 #pragma unroll
         for (int a = J0; a < 8; ++a) {
             const float p = xi * xj[a];
+            const uint64_t pp = pack2(p, p);
 #pragma unroll
-            for (int b = (DIAG ? a : 0); b < 8; ++b) acc[a][b] = fmaf(p, xk[b], acc[a][b]);
+            for (int c = (DIAG ? a / 2 : 0); c < 4; ++c) acc[a][c] = ffma2(pp, xk[c], acc[a][c]);
         }
     }
 }
@@ -99,11 +121,11 @@ moment3_kernel(const float *__restrict__ X, int64_t N, int d, int64_t ldx, float
     const int pi = ((ti & 7) < 4) ? 4 * (ti >> 3) + (ti & 3) : half + 4 * (ti >> 3) + (ti & 3);
     const int oj = 4 * tjb, ok = 4 * tkb;
 
-    float acc[8][8];
+    uint64_t acc[8][4];
 #pragma unroll
     for (int a = 0; a < 8; ++a)
 #pragma unroll
-        for (int b = 0; b < 8; ++b) acc[a][b] = 0.f;
+        for (int c = 0; c < 4; ++c) acc[a][c] = 0ull;
 
     const int64_t n_begin = (int64_t)blockIdx.y * rows_per_slice;
     int64_t n_end = n_begin + rows_per_slice;
@@ -159,9 +181,12 @@ moment3_kernel(const float *__restrict__ X, int64_t N, int d, int64_t ldx, float
         if (j < ti) continue;
         const int base = (int)tet_encode(d, ti, j, j);   // row (i,j,*) is contiguous in k
 #pragma unroll
-        for (int b = 0; b < 8; ++b) {
-            const int k = 8 * tkb + b;
-            if (k >= j) mine[base + (k - j)] = acc[a][b];
+        for (int c = 0; c < 4; ++c) {
+            float lo, hi;
+            unpack2(acc[a][c], lo, hi);
+            const int k = 8 * tkb + 2 * c;
+            if (k >= j) mine[base + (k - j)] = lo;
+            if (k + 1 >= j) mine[base + (k + 1 - j)] = hi;
         }
     }
 }
@@ -186,10 +211,11 @@ struct WarpDesc {
 
 static int variant_cost(int v)
 {
-    if (v == 0) return 64 + 8 + 6;
-    if (v == 1) return 36 + 8 + 4;
+    // fp32-pipe cycles per sample row: two per packed FMA, one per pair product, plus loads
+    if (v == 0) return 64 + 8 + 3;
+    if (v == 1) return 40 + 8 + 2;
     const int rows = 8 - (v - 1);
-    return rows * 8 + rows + 6;
+    return rows * 8 + rows + 3;
 }
 
 // Builds the per-thread tile table for side d.  Returns the number of groups.

@@ -2,11 +2,16 @@
 // (T_C = T * T_U, Section 4) and reconstruct the dense tensor from it
 // (T = T_C + T_R * T_C, Section 6, Property 5).  HBM-bound index-decode copies.
 //
-// Both kernels are organised by rows: a row is one position of the structured modes
-// carrying `inner` contiguous elements.  A group of G lanes (G a power of two <= 32) owns
-// one row of the array being WRITTEN, decodes its index tuple once with the closed forms
-// of st_index.cuh, and copies the row in units of U bytes (16 where the row width allows),
-// so stores are always coalesced and loads are coalesced within a row.
+// Two kernels.
+//   slice_copy_kernel (st_pack, st_unpack with zero fill): the dense array is cut into slices
+//   along its last structured index (matrix row i; pair (i,j) of an order-3 tensor).  In every
+//   supported structure the unique positions of a slice are ONE contiguous run of columns
+//   [lo,hi) that is also contiguous in the packed array, so a slice is "zeros, one flat copy,
+//   zeros" and needs no per-element index arithmetic at all: the run and its packed offset come
+//   from the closed forms of st_index.cuh once per slice.  Copies run in units of U bytes (16
+//   where the row width allows); long slices are split into parts over several thread groups.
+//   structured_copy_kernel (st_unpack with symmetric fill): one lane group per dense row
+//   decodes its index tuple, maps it through the redundancy map and copies the row.
 #include "st_common.cuh"
 #include "st_index.cuh"
 
@@ -113,6 +118,74 @@ structured_copy_kernel(const U *__restrict__ src, U *__restrict__ dst, LayoutArg
     }
 }
 
+// Run of unique columns of slice s, in rows of `chunks` units: dense columns [lo,hi) of the
+// slice map to packed rows prow.. (contiguous).  For ST_BAND also the extent of the fixed-width
+// packed row [band0, band1) whose slots outside the run are zero-filled by pack.
+template <int KIND>
+__device__ __forceinline__ void slice_run(const LayoutArgs &a, int64_t s, int64_t &lo, int64_t &hi, int64_t &prow)
+{
+    if (KIND == ST_TRI_UPPER) {
+        lo = s; hi = a.d; prow = tri_row_start(a.d, s);
+    } else if (KIND == ST_TET) {
+        const int64_t i = s / a.d, j = s - i * a.d;
+        if (j < i) { lo = hi = 0; prow = 0; }
+        else { lo = j; hi = a.d; prow = tet_encode(a.d, i, j, j); }
+    } else if (KIND == ST_BAND) {
+        lo = s - a.kl; if (lo < 0) lo = 0;
+        hi = s + a.ku + 1; if (hi > a.d) hi = a.d;
+        if (hi < lo) hi = lo;
+        prow = s * a.width + (lo - (s - a.kl));
+    } else {
+        const int64_t b = s / a.bs;
+        lo = b * a.bs; hi = lo + a.bs; prow = s * a.bs;
+    }
+}
+
+template <int KIND, typename U, bool PACK>
+__global__ void __launch_bounds__(256)
+slice_copy_kernel(const U *__restrict__ src, U *__restrict__ dst, LayoutArgs a, int group_shift, int parts)
+{
+    const int g = 1 << group_shift;
+    const int lane = (int)(threadIdx.x & (g - 1));
+    const int64_t gid = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> group_shift;
+    const int64_t ngroups = ((int64_t)gridDim.x * blockDim.x) >> group_shift;
+    const int64_t nslices = (KIND == ST_TET) ? a.d * a.d : a.d;
+    const int64_t su = a.d * a.chunks;                        // units per dense slice
+    const int64_t part_units = (su + parts - 1) / parts;
+    for (int64_t item = gid; item < nslices * parts; item += ngroups) {
+        const int64_t s = item / parts;
+        const int64_t part = item - s * parts;
+        int64_t lo, hi, prow;
+        slice_run<KIND>(a, s, lo, hi, prow);
+        const int64_t u0 = part * part_units;                 // this part covers dense units [u0, u1) of the slice
+        int64_t u1 = u0 + part_units;
+        if (u1 > su) u1 = su;
+        const int64_t c0 = lo * a.chunks, c1 = hi * a.chunks;  // units of the run inside the slice
+        const int64_t x0 = u0 > c0 ? u0 : c0, x1 = u1 < c1 ? u1 : c1;   // run clipped to this part
+        if (PACK) {
+            const U *in = src + s * su;
+            U *out = dst + prow * a.chunks - c0;                // out[u] for dense unit u of the run
+            for (int64_t u = x0 + lane; u < x1; u += g) out[u] = in[u];
+            if (KIND == ST_BAND && part == 0) {
+                // slots of the fixed-width packed row that fall outside the matrix
+                U *row = dst + s * a.width * a.chunks;
+                const int64_t first = (prow - s * a.width) * a.chunks, last = first + (c1 - c0);
+                const int64_t wu = a.width * a.chunks;
+                for (int64_t u = lane; u < first; u += g) row[u] = zero_unit<U>();
+                for (int64_t u = last + lane; u < wu; u += g) row[u] = zero_unit<U>();
+            }
+        } else {
+            U *out = dst + s * su;
+            const U *in = src + prow * a.chunks - c0;
+            const int64_t z1 = u1 < c0 ? u1 : c0;               // zeros before the run
+            for (int64_t u = u0 + lane; u < z1; u += g) out[u] = zero_unit<U>();
+            for (int64_t u = x0 + lane; u < x1; u += g) out[u] = in[u];
+            const int64_t z2 = u0 > c1 ? u0 : c1;               // zeros after the run
+            for (int64_t u = z2 + lane; u < u1; u += g) out[u] = zero_unit<U>();
+        }
+    }
+}
+
 static bool layout_ok(const st_layout *L)
 {
     if (!L) return false;
@@ -156,14 +229,29 @@ static int dtype_bytes(st_dtype t)
 template <int KIND, typename U, bool PACK>
 static st_status launch_copy(const void *src, void *dst, const LayoutArgs &a, cudaStream_t s)
 {
-    const int64_t rows = PACK ? a.packed_rows : a.dense_rows;
-    int shift = 0;
-    while ((1 << shift) < 32 && (int64_t(1) << shift) < a.chunks) ++shift;
-    const int64_t threads = rows << shift;
-    const int64_t want = (threads + 255) / 256;
     const int64_t cap = (int64_t)sm_count_or_default() * 16;
+    if (!PACK && a.fill == ST_FILL_SYMMETRIC) {
+        // redundancy map: one lane group per dense row
+        int shift = 0;
+        while ((1 << shift) < 32 && (int64_t(1) << shift) < a.chunks) ++shift;
+        const int64_t threads = a.dense_rows << shift;
+        const int64_t want = (threads + 255) / 256;
+        const int grid = (int)(want < cap ? (want < 1 ? 1 : want) : cap);
+        structured_copy_kernel<KIND, U, PACK><<<grid, 256, 0, s>>>((const U *)src, (U *)dst, a, shift);
+        return launch_status();
+    }
+    // slices: about 8 units per thread, at most 8192 units per (slice, part)
+    const int64_t su = a.d * a.chunks;
+    int parts = (int)((su + 8191) / 8192);
+    if (parts < 1) parts = 1;
+    const int64_t pu = (su + parts - 1) / parts;
+    int shift = 0;
+    while ((1 << shift) < 256 && (int64_t(8) << shift) < pu) ++shift;
+    const int64_t nslices = (KIND == ST_TET) ? a.d * a.d : a.d;
+    const int64_t threads = (nslices * parts) << shift;
+    const int64_t want = (threads + 255) / 256;
     const int grid = (int)(want < cap ? (want < 1 ? 1 : want) : cap);
-    structured_copy_kernel<KIND, U, PACK><<<grid, 256, 0, s>>>((const U *)src, (U *)dst, a, shift);
+    slice_copy_kernel<KIND, U, PACK><<<grid, 256, 0, s>>>((const U *)src, (U *)dst, a, shift, parts);
     return launch_status();
 }
 

@@ -368,3 +368,20 @@ def test_ttm_tf32_config(st):
     A, S = oracle.ttm(Bp.reshape(-1, 256)[rows], U)
     assert oracle.rel_err(got[rows], A, S) <= TOL_TC
     assert st.st_check_status() == st.ST_OK
+
+
+def test_moment2_bf16_all_tiles_midsize(st):
+    """d = 1024 (all 20 launched tiles, both diagonal and off-diagonal kinds) at a sample count
+    the oracle can still check on sampled entries quickly; input 256 MiB, larger than L2."""
+    N, d = 131072, 1024
+    bits = workloads.draw_rows_bf16(N, d, "normal", 4242)
+    got = st.st_sym_moment2(bf16_dev(bits)).cpu().numpy()
+    Xb = workloads.bf16_bits_to_f32(bits).reshape(N, d)
+    rng = np.random.default_rng(9)
+    pairs = [(i, i) for i in range(0, d, 61)] + [(r * 128 + a, c * 256 + b) for r in range(8) for c in range(4)
+                                                 for a, b in ((0, 0), (127, 255), (5, 200)) if r * 128 + a <= c * 256 + b]
+    pairs += [tuple(sorted(int(v) for v in rng.integers(0, d, 2))) for _ in range(200)]
+    ii, jj = (np.array(v) for v in zip(*pairs))
+    T, S = oracle.moment2_at(Xb, ii, jj)
+    pos = ii * (2 * d - ii + 1) // 2 + (jj - ii)
+    assert oracle.rel_err(got[pos], T, S) <= TOL_F32
