@@ -27,8 +27,9 @@ namespace st {
 
 constexpr int M3_THREADS = 512;            // 16 warps per block
 constexpr int M3_WPB = M3_THREADS / 32;
-constexpr int M3_STAGE_ROWS = 64;          // sample rows per shared-memory stage
+constexpr int M3_STAGE_ROWS = 128;         // sample rows per shared-memory stage
 constexpr int M3_MAX_D = 64;
+constexpr int M3_BUFFERS = 3;               // shared-memory stages in flight
 
 template <int WARPS>
 struct M3Table {
@@ -107,7 +108,7 @@ __global__ void __launch_bounds__(M3_THREADS, 1)
 moment3_kernel(const float *__restrict__ X, int64_t N, int d, int64_t ldx, float *__restrict__ partials,
                int64_t rows_per_slice, int out_elems, const __grid_constant__ M3Table<WARPS> tab)
 {
-    extern __shared__ __align__(16) float smem[];   // 2 stages of M3_STAGE_ROWS x d floats
+    extern __shared__ __align__(16) float smem[];   // M3_BUFFERS stages of M3_STAGE_ROWS x d floats
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int group = blockIdx.x;
     const int slot = group * M3_WPB + warp;
@@ -147,17 +148,20 @@ moment3_kernel(const float *__restrict__ X, int64_t N, int d, int64_t ldx, float
     };
 
     const int64_t nstages = (n_end > n_begin) ? (n_end - n_begin + M3_STAGE_ROWS - 1) / M3_STAGE_ROWS : 0;
-    if (nstages > 0) load_stage(0, n_begin);
+    // three buffers, one barrier per stage: stage s+2 is issued after the barrier of stage s, which
+    // every warp passes only after it has finished stage s-1 (the previous user of that buffer)
+    for (int s = 0; s < M3_BUFFERS - 1; ++s) {
+        if (s < nstages) load_stage(s, n_begin + (int64_t)s * M3_STAGE_ROWS);
+        else cp_async_commit();
+    }
     for (int64_t s = 0; s < nstages; ++s) {
-        const int buf = (int)(s & 1);
-        if (s + 1 < nstages) {
-            load_stage(buf ^ 1, n_begin + (s + 1) * M3_STAGE_ROWS);
-            cp_async_wait<1>();
-        } else {
-            cp_async_wait<0>();
-        }
+        cp_async_wait<M3_BUFFERS - 2>();
         __syncthreads();
-        const float *xs = smem + buf * stage_floats;
+        if (s + M3_BUFFERS - 1 < nstages)
+            load_stage((int)((s + M3_BUFFERS - 1) % M3_BUFFERS), n_begin + (s + M3_BUFFERS - 1) * M3_STAGE_ROWS);
+        else
+            cp_async_commit();
+        const float *xs = smem + (int)(s % M3_BUFFERS) * stage_floats;
         switch (variant) {
         case 0: m3_stage<0, false>(xs, d, pi, oj, ok, half, acc); break;
         case 1: m3_stage<0, true>(xs, d, pi, oj, ok, half, acc); break;
@@ -170,8 +174,8 @@ moment3_kernel(const float *__restrict__ X, int64_t N, int d, int64_t ldx, float
         case 8: m3_stage<7, false>(xs, d, pi, oj, ok, half, acc); break;
         default: break;
         }
-        __syncthreads();
     }
+    cp_async_wait<0>();
 
     if (!valid || variant == 255) return;
     float *mine = partials + (size_t)blockIdx.y * out_elems;
@@ -197,7 +201,13 @@ sum_slices_kernel(const float *__restrict__ partials, float *__restrict__ out, i
     const int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (e >= elems) return;
     float s = 0.f;
-    for (int k = 0; k < slices; ++k) s += __ldcg(&partials[(size_t)k * elems + e]);
+    for (int k0 = 0; k0 < slices; k0 += 8) {
+        float v[8];                       // eight loads in flight before the first add
+#pragma unroll
+        for (int u = 0; u < 8; ++u) v[u] = (k0 + u < slices) ? __ldcg(&partials[(size_t)(k0 + u) * elems + e]) : 0.f;
+#pragma unroll
+        for (int u = 0; u < 8; ++u) s += v[u];
+    }
     out[e] = s;
 }
 
@@ -211,11 +221,11 @@ struct WarpDesc {
 
 static int variant_cost(int v)
 {
-    // fp32-pipe cycles per sample row: two per packed FMA, one per pair product, plus loads
-    if (v == 0) return 64 + 8 + 3;
-    if (v == 1) return 40 + 8 + 2;
+    // fp32-pipe cycles per sample row: two per packed FMA, one per pair product, one per pair move
+    if (v == 0) return 64 + 16;
+    if (v == 1) return 40 + 16;
     const int rows = 8 - (v - 1);
-    return rows * 8 + rows + 3;
+    return rows * 8 + 2 * rows;
 }
 
 // Builds the per-thread tile table for side d.  Returns the number of groups.
@@ -249,25 +259,63 @@ static bool build_table(int d, bool dense, M3Table<WARPS> &tab)
     const int nw = (int)warps.size();
     const int groups = (nw + M3_WPB - 1) / M3_WPB;
     if (groups * M3_WPB > WARPS) return false;
-    // deal warps, most expensive first, to the scheduler bin (group, warp%4) with the least load
+    // deal warps, most expensive first, to the scheduler bin (group, warp%4) with the least load,
+    // then swap warps between the fullest bin and the others while that lowers the maximum
     std::stable_sort(warps.begin(), warps.end(), [](const WarpDesc &a, const WarpDesc &b) { return a.cost > b.cost; });
     const int bins = groups * 4;
-    std::vector<int> load(bins, 0), count(bins, 0);
+    const int cap = M3_WPB / 4;
+    std::vector<int> load(bins, 0);
+    std::vector<std::vector<int>> members(bins);
+    for (int w = 0; w < nw; ++w) {
+        int best = -1;
+        for (int b = 0; b < bins; ++b)
+            if ((int)members[b].size() < cap && (best < 0 || load[b] < load[best])) best = b;
+        if (best < 0) return false;
+        members[best].push_back(w);
+        load[best] += warps[w].cost;
+    }
+    for (int iter = 0; iter < 200; ++iter) {
+        int hi = 0;
+        for (int b = 1; b < bins; ++b)
+            if (load[b] > load[hi]) hi = b;
+        bool improved = false;
+        for (int b = 0; b < bins && !improved; ++b) {
+            if (b == hi) continue;
+            for (size_t x = 0; x < members[hi].size() && !improved; ++x) {
+                const int cx = warps[members[hi][x]].cost;
+                // move x to b
+                if ((int)members[b].size() < cap && load[b] + cx < load[hi]) {
+                    load[b] += cx; load[hi] -= cx;
+                    members[b].push_back(members[hi][x]);
+                    members[hi].erase(members[hi].begin() + x);
+                    improved = true;
+                    break;
+                }
+                for (size_t y = 0; y < members[b].size(); ++y) {
+                    const int cy = warps[members[b][y]].cost;
+                    if (cy < cx && load[b] - cy + cx < load[hi]) {
+                        load[b] += cx - cy; load[hi] -= cx - cy;
+                        std::swap(members[hi][x], members[b][y]);
+                        improved = true;
+                        break;
+                    }
+                }
+            }
+        }
+        if (!improved) break;
+    }
     tab.groups = groups;
     tab.nbk = nbk;
     for (int w = 0; w < WARPS; ++w) tab.variant[w] = 255;
     for (int e = 0; e < WARPS * 32; ++e) tab.tile[e] = 0;
-    for (const WarpDesc &w : warps) {
-        int best = -1;
-        for (int b = 0; b < bins; ++b)
-            if (count[b] < M3_WPB / 4 && (best < 0 || load[b] < load[best])) best = b;
-        if (best < 0) return false;
-        const int g = best / 4, sched = best % 4;
-        const int slot = g * M3_WPB + sched + 4 * count[best];   // warp index % 4 = scheduler
-        load[best] += w.cost;
-        count[best] += 1;
-        tab.variant[slot] = (unsigned char)w.variant;
-        for (size_t l = 0; l < w.tiles.size(); ++l) tab.tile[slot * 32 + l] = w.tiles[l];
+    for (int b = 0; b < bins; ++b) {
+        const int g = b / 4, sched = b % 4;
+        for (size_t k = 0; k < members[b].size(); ++k) {
+            const WarpDesc &w = warps[members[b][k]];
+            const int slot = g * M3_WPB + sched + 4 * (int)k;   // warp index % 4 = scheduler
+            tab.variant[slot] = (unsigned char)w.variant;
+            for (size_t l = 0; l < w.tiles.size(); ++l) tab.tile[slot * 32 + l] = w.tiles[l];
+        }
     }
     return true;
 }
@@ -305,7 +353,7 @@ static st_status moment3_launch(const float *X, int64_t N, int64_t d, int64_t ld
     if (!ws || ws_bytes < need) return ST_ERR_WORKSPACE;
     if (!aligned256(ws)) return ST_ERR_ALIGN;
     float *partials = (float *)((unsigned char *)ws + kWsHeaderBytes);
-    const size_t smem = 2 * (size_t)M3_STAGE_ROWS * d * sizeof(float);
+    const size_t smem = (size_t)M3_BUFFERS * M3_STAGE_ROWS * d * sizeof(float);
     if (smem > 48 * 1024) {
         if (cudaFuncSetAttribute(moment3_kernel<WARPS>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
             cudaSuccess)
