@@ -233,6 +233,246 @@ moment2_tc_reduce_kernel(const float *__restrict__ partials, float *__restrict__
     }
 }
 
+// ---------------------------------------------------------------------------------------------
+// Two-block variant (d >= 512): a cluster of two blocks owns a 256 x 256 tile.  Block r stages
+// columns 256*TM+128r.. (its 128 rows of the A operand) and columns 256*TN+128r.. (its half of
+// the B operand); on diagonal tiles the two coincide and are loaded once.  The leader block
+// issues one MMA of M = 256, N = 256 for the pair; each block keeps the accumulator of its 128
+// rows in its own tensor memory.  Per MMA cycle a block now fetches a third less from L2 than in
+// the one-block kernel and has six stages in flight, which is what that kernel was short of
+// (its tensor pipe idled ~30% of the time waiting for operands).
+namespace m2tc2 {
+constexpr int BM = 256, BN = 256;               // tile of the pair
+constexpr int HALF = 128;                       // rows / B columns staged per block
+constexpr int KROWS = m2tc::KROWS, BOXC = m2tc::BOXC, BOX_BYTES = m2tc::BOX_BYTES;
+constexpr int NBOX = HALF / BOXC;               // 2 boxes per operand per block
+constexpr int STAGE_BYTES = 2 * NBOX * BOX_BYTES;   // 32 KiB
+constexpr int STAGES = 6;
+constexpr int THREADS = 192;
+constexpr int MAX_TILES = 160;
+constexpr uint32_t TMEM_COLS = 512;
+constexpr int FLUSH_CHUNKS = 64;
+constexpr size_t SMEM_BYTES = (size_t)STAGES * STAGE_BYTES + 1024 + 256;
+
+struct TileTable {
+    int ntiles, nsplit;
+    unsigned char tm[MAX_TILES];   // units of 256
+    unsigned char tn[MAX_TILES];
+};
+}  // namespace m2tc2
+
+__global__ void __launch_bounds__(m2tc2::THREADS, 1)
+moment2_tc_pair_kernel(const __grid_constant__ CUtensorMap tmap, float *__restrict__ partials, unsigned *status,
+                       int chunks_total, const __grid_constant__ m2tc2::TileTable tab)
+{
+    using namespace m2tc2;
+    using namespace tc;
+    extern __shared__ unsigned char smem_raw[];
+    unsigned char *smem = (unsigned char *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+    uint64_t *bars = (uint64_t *)(smem + (size_t)STAGES * STAGE_BYTES);
+    uint64_t *full = bars, *empty = bars + STAGES, *acc_full = bars + 2 * STAGES, *acc_empty = bars + 2 * STAGES + 2;
+    uint32_t *tmem_slot = (uint32_t *)(bars + 2 * STAGES + 4);
+    volatile int *abort_flag = (volatile int *)(tmem_slot + 1);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t rank = cluster_ctarank();            // 0 = leader
+    const int cluster = blockIdx.x >> 1;
+    const int tile = cluster / tab.nsplit, split = cluster - tile * tab.nsplit;
+    const int tm = tab.tm[tile], tn = tab.tn[tile];
+    const bool diag = (tm == tn);                       // A columns == B columns in every block
+    const int chunks_per_split = (chunks_total + tab.nsplit - 1) / tab.nsplit;
+    const int c_begin = split * chunks_per_split;
+    int c_end = c_begin + chunks_per_split;
+    if (c_end > chunks_total) c_end = chunks_total;
+    const int nchunks = c_end > c_begin ? c_end - c_begin : 0;
+    const int nphases = (nchunks + FLUSH_CHUNKS - 1) / FLUSH_CHUNKS;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < STAGES; ++s) {
+            mbar_init(&full[s], 1);          // leader's producer arrives once and announces the bytes of both blocks
+            mbar_init(&empty[s], 1);         // one commit per use, delivered to both blocks
+        }
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(&acc_full[b], 1);
+            mbar_init(&acc_empty[b], 8);     // four epilogue warps in each of the two blocks (leader's copy is used)
+        }
+        *abort_flag = 0;
+        fence_barrier_init();
+    }
+    if (warp == 1) {
+        tmem_alloc_pair(tmem_slot, TMEM_COLS);
+        tmem_relinquish_pair();
+    }
+    tc_fence_before();
+    __syncthreads();
+    cluster_sync_all();                      // both blocks' barriers exist before anything is signalled across
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    if (warp == 0) {
+        // ---------------- TMA producer (both blocks): own boxes, completion counted on the leader's barrier
+        if (elect_one()) {
+            prefetch_tmap(&tmap);
+            const uint32_t own_tx = (uint32_t)((diag ? NBOX : 2 * NBOX) * BOX_BYTES);
+            for (int c = 0; c < nchunks; ++c) {
+                const int s = c % STAGES;
+                if (c >= STAGES && !mbar_wait(&empty[s], ((c / STAGES) - 1) & 1, abort_flag, status, 1)) break;
+                unsigned char *st_base = smem + (size_t)s * STAGE_BYTES;
+                if (rank == 0) mbar_expect_tx(&full[s], 2 * own_tx);
+                const uint32_t bar = map_to_cta(smem_u32(&full[s]), 0);
+                const int row = (c_begin + c) * KROWS;
+                for (int b = 0; b < NBOX; ++b)          // B half (and A on diagonal tiles)
+                    tma_load_2d_pair(st_base + b * BOX_BYTES, &tmap, bar, tn * BN + (int)rank * HALF + b * BOXC, row);
+                if (!diag)
+                    for (int b = 0; b < NBOX; ++b)      // A rows of this block
+                        tma_load_2d_pair(st_base + (NBOX + b) * BOX_BYTES, &tmap, bar, tm * BM + (int)rank * HALF + b * BOXC, row);
+            }
+        }
+    } else if (warp == 1) {
+        // ---------------- MMA issuer (leader only)
+        if (rank == 0 && elect_one()) {
+            constexpr uint32_t idesc = make_idesc(1, 1, 1, BM, BN);
+            const uint32_t a_off = diag ? 0u : (uint32_t)(NBOX * BOX_BYTES);
+            const uint32_t sb0 = smem_u32(smem);
+            const uint64_t adesc_base = make_smem_desc(sb0 + a_off, BOX_BYTES, 1024);
+            const uint64_t bdesc_base = make_smem_desc(sb0, BOX_BYTES, 1024);
+            bool ok = true;
+            int c = 0;
+            for (int ph = 0; ph < nphases && ok; ++ph) {
+                const int buf = ph & 1;
+                if (ph >= 2 && !mbar_wait(&acc_empty[buf], (uint32_t)(((ph >> 1) - 1) & 1), abort_flag, status, 4)) break;
+                tc_fence_after();
+                const uint32_t d_tmem = tmem_base + (uint32_t)(buf * BN);
+                const int ce = (c + FLUSH_CHUNKS < nchunks) ? c + FLUSH_CHUNKS : nchunks;
+                uint32_t accumulate = 0;
+                for (; c < ce; ++c) {
+                    const int s = c % STAGES;
+                    if (!mbar_wait(&full[s], (c / STAGES) & 1, abort_flag, status, 2)) {
+                        ok = false;
+                        break;
+                    }
+                    tc_fence_after();
+                    const uint64_t ad = adesc_base + (uint64_t)(s * (STAGE_BYTES >> 4));
+                    const uint64_t bd = bdesc_base + (uint64_t)(s * (STAGE_BYTES >> 4));
+#pragma unroll
+                    for (int k = 0; k < KROWS / 16; ++k) {
+                        mma_bf16_pair(d_tmem, ad + (uint64_t)(k * 128), bd + (uint64_t)(k * 128), idesc, accumulate);
+                        accumulate = 1;
+                    }
+                    tc_commit_pair(&empty[s]);
+                }
+                tc_commit_pair(&acc_full[buf]);
+            }
+        }
+    } else {
+        // ---------------- epilogue (both blocks): own 128 rows of the tile
+        const int q = warp & 3;
+        float *dst = partials + ((size_t)blockIdx.x * HALF + (q * 32 + lane)) * BN;
+        const uint32_t leader_acc_empty0 = map_to_cta(smem_u32(&acc_empty[0]), 0);
+        if (nphases == 0) {
+            for (int c0 = 0; c0 < BN; c0 += 4) *reinterpret_cast<float4 *>(dst + c0) = make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+        for (int ph = 0; ph < nphases; ++ph) {
+            const int buf = ph & 1;
+            if (!mbar_wait(&acc_full[buf], (uint32_t)((ph >> 1) & 1), abort_flag, status, 3)) break;
+            tc_fence_after();
+#pragma unroll 1
+            for (int c0 = 0; c0 < BN; c0 += 32) {
+                uint32_t r[32];
+                tmem_ld_32x32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * BN + c0), r);
+                tmem_ld_wait();
+#pragma unroll
+                for (int e = 0; e < 32; e += 4) {
+                    float4 v = make_float4(__uint_as_float(r[e]), __uint_as_float(r[e + 1]), __uint_as_float(r[e + 2]),
+                                           __uint_as_float(r[e + 3]));
+                    float4 *p = reinterpret_cast<float4 *>(dst + c0 + e);
+                    if (ph > 0) {
+                        const float4 o = *p;
+                        v.x += o.x; v.y += o.y; v.z += o.z; v.w += o.w;
+                    }
+                    *p = v;
+                }
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive_cluster(leader_acc_empty0 + (uint32_t)(buf * sizeof(uint64_t)));
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    cluster_sync_all();                      // no block leaves while its peer may still signal it
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc_pair(tmem_base, TMEM_COLS);
+    }
+}
+
+__global__ void __launch_bounds__(256)
+moment2_tc_pair_reduce_kernel(const float *__restrict__ partials, float *__restrict__ out, int d,
+                              const __grid_constant__ m2tc2::TileTable tab)
+{
+    using namespace m2tc2;
+    const int tile = blockIdx.x;
+    const int tm = tab.tm[tile], tn = tab.tn[tile], nsplit = tab.nsplit;
+    // partial of (tile, split, block r) lives in slot 2*(tile*nsplit+split)+r, a [128][256] array
+    for (int e = blockIdx.y * 256 + threadIdx.x; e < BM * BN; e += gridDim.y * 256) {
+        const int r = e / BN, c = e - r * BN;
+        const int gi = tm * BM + r, gj = tn * BN + c;
+        if (gi < d && gj < d && gi <= gj) {
+            const float *base = partials + ((size_t)(2 * tile * nsplit + (r >> 7)) * HALF + (r & 127)) * BN + c;
+            const size_t stride = (size_t)2 * HALF * BN;
+            float s = 0.f;
+            for (int k0 = 0; k0 < nsplit; k0 += 8) {
+                float v[8];
+#pragma unroll
+                for (int u = 0; u < 8; ++u) v[u] = (k0 + u < nsplit) ? __ldcg(base + (size_t)(k0 + u) * stride) : 0.f;
+#pragma unroll
+                for (int u = 0; u < 8; ++u) s += v[u];
+            }
+            out[tri_encode(d, gi, gj)] = s;
+        }
+    }
+}
+
+struct M2Tc2Plan {
+    m2tc2::TileTable tab;
+    int chunks_total;
+    size_t partial_bytes;
+    bool ok;
+};
+
+static M2Tc2Plan m2tc2_plan(int64_t N, int64_t d, unsigned flags)
+{
+    using namespace m2tc2;
+    M2Tc2Plan p;
+    p.ok = false;
+    const bool dense = (flags & ST_FLAG_DENSE_CONTROL) != 0;
+    const int nt = (int)((d + BM - 1) / BM);
+    int n = 0;
+    for (int tn = 0; tn < nt; ++tn)
+        for (int tm = 0; tm < nt; ++tm) {
+            if (tm > tn && !dense) continue;
+            if (n >= MAX_TILES) return p;
+            p.tab.tm[n] = (unsigned char)tm;
+            p.tab.tn[n] = (unsigned char)tn;
+            ++n;
+        }
+    for (int i = n; i < MAX_TILES; ++i) p.tab.tm[i] = p.tab.tn[i] = 0;
+    p.tab.ntiles = n;
+    const int64_t chunks = (N + KROWS - 1) / KROWS;
+    if (chunks > (int64_t(1) << 30)) return p;
+    p.chunks_total = (int)chunks;
+    int64_t per = (sm_count_or_default() / 2) / n;   // clusters per tile: equal, so that sample ranges run in step
+    if (per < 1) per = 1;
+    if (per > chunks) per = chunks;
+    p.tab.nsplit = (int)per;
+    p.partial_bytes = (size_t)2 * n * per * HALF * BN * sizeof(float);
+    p.ok = true;
+    return p;
+}
+
+static bool m2_use_pair(int64_t d) { return d >= 512; }
+
 struct M2TcPlan {
     m2tc::TileTable tab;
     int chunks_total;
@@ -293,6 +533,10 @@ static M2TcPlan m2tc_plan(int64_t N, int64_t d, unsigned flags)
 size_t moment2_bf16_tc_workspace(int64_t N, int64_t d, unsigned flags)
 {
     if (N <= 0 || d <= 0 || d % 8 != 0 || d > 4096 || N > (int64_t(1) << 31) - 64) return 0;
+    if (m2_use_pair(d)) {
+        const M2Tc2Plan q = m2tc2_plan(N, d, flags);
+        return q.ok ? kWsHeaderBytes + q.partial_bytes : 0;
+    }
     const M2TcPlan p = m2tc_plan(N, d, flags);
     return p.ok ? kWsHeaderBytes + p.partial_bytes : 0;
 }
@@ -303,6 +547,40 @@ st_status moment2_bf16_tc(const void *X, int64_t N, int64_t d, int64_t ldx, floa
     using namespace m2tc;
     if (d % 8 != 0 || ldx % 8 != 0) return ST_ERR_ALIGN;
     if (d > 4096 || N > (int64_t(1) << 31) - 64) return ST_ERR_UNSUPPORTED;
+    if (m2_use_pair(d)) {
+        const M2Tc2Plan q = m2tc2_plan(N, d, flags);
+        if (!q.ok) return ST_ERR_UNSUPPORTED;
+        if (!ws || ws_bytes < kWsHeaderBytes + q.partial_bytes) return ST_ERR_WORKSPACE;
+        if (!aligned256(ws)) return ST_ERR_ALIGN;
+        CUtensorMap tm2;
+        if (!tc::make_tmap_2d(&tm2, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, X, (uint64_t)N, (uint64_t)d, (uint64_t)ldx * 2,
+                              BOXC, KROWS))
+            return ST_ERR_CUDA;
+        if (cudaMemsetAsync(ws, 0, kWsHeaderBytes, stream) != cudaSuccess) return ST_ERR_CUDA;
+        float *part2 = (float *)((unsigned char *)ws + kWsHeaderBytes);
+        if (cudaFuncSetAttribute(moment2_tc_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 (int)m2tc2::SMEM_BYTES) != cudaSuccess)
+            return ST_ERR_CUDA;
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(2 * q.tab.ntiles * q.tab.nsplit);
+        cfg.blockDim = dim3(m2tc2::THREADS);
+        cfg.dynamicSmemBytes = m2tc2::SMEM_BYTES;
+        cfg.stream = stream;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeClusterDimension;
+        attr[0].val.clusterDim.x = 2;
+        attr[0].val.clusterDim.y = 1;
+        attr[0].val.clusterDim.z = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        if (cudaLaunchKernelEx(&cfg, moment2_tc_pair_kernel, tm2, part2, (unsigned *)ws, q.chunks_total, q.tab) !=
+            cudaSuccess) {
+            (void)cudaGetLastError();
+            return ST_ERR_CUDA;
+        }
+        moment2_tc_pair_reduce_kernel<<<dim3(q.tab.ntiles, 16), 256, 0, stream>>>(part2, out, (int)d, q.tab);
+        return launch_status();
+    }
     const M2TcPlan p = m2tc_plan(N, d, flags);
     if (!p.ok) return ST_ERR_UNSUPPORTED;
     const size_t need = kWsHeaderBytes + p.partial_bytes;
