@@ -18,7 +18,7 @@ constexpr int BM = 128;                    // fibres per tile
 constexpr int KC = 32;                     // floats per k-slice (128 bytes)
 constexpr int STAGE_BYTES = BM * KC * 4;   // 16 KiB
 constexpr int THREADS = 192;
-constexpr int MAX_STAGES = 6;
+constexpr int MAX_STAGES = 10;
 }  // namespace ttmtc
 
 struct TtmTcArgs {
@@ -64,22 +64,47 @@ ttm_tc_kernel(const __grid_constant__ CUtensorMap tmap, const TtmTcArgs a)
         tmem_alloc(tmem_slot, a.tmem_cols);
         tmem_relinquish();
     }
-    // U^T, rounded to TF32, K-major with the 128-byte swizzle: element (r, k) of slice k/32
-    // goes to byte r*128 + ((k%32/4) ^ (r%8))*16 + (k%4)*4 of that slice's region
-    for (int e = threadIdx.x; e < a.kchunks * KC * a.R; e += THREADS) {
-        const int k = e / a.R, r = e - k * a.R;                      // consecutive threads: consecutive r (coalesced)
-        const float v = (k < a.K) ? a.U[(size_t)k * a.R + r] : 0.f;
-        uint32_t t;
-        asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(t) : "f"(v));
-        const int kc = k >> 5, kk = k & 31;
-        const int off = r * 128 + (((kk >> 2) ^ (r & 7)) << 4) + ((kk & 3) << 2);
-        *reinterpret_cast<uint32_t *>(u_smem + (size_t)kc * u_region + off) = t;
-    }
-    fence_proxy_async();      // make the generic-proxy writes of U visible to the tensor core
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
+
+    if (warp != 0) {
+        // Warps 1..5 build U^T while warp 0 already streams fibres: U rounded to TF32, K-major with
+        // the 128-byte swizzle; element (r, k) of slice k/32 goes to byte
+        // r*128 + ((k%32/4) ^ (r%8))*16 + (k%4)*4 of that slice's region.
+        const int nthr = THREADS - 32, t0 = threadIdx.x - 32;
+        const int r4 = a.R >> 2;                                      // float4 groups per row of U
+        const int total4 = a.kchunks * KC * r4;
+        for (int e0 = t0; e0 < total4; e0 += 4 * nthr) {
+            float4 v[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {                             // four independent loads in flight
+                const int e = e0 + u * nthr;
+                const int k = e / r4;
+                v[u] = (e < total4 && k < a.K) ? __ldg(reinterpret_cast<const float4 *>(a.U) + e)
+                                               : make_float4(0.f, 0.f, 0.f, 0.f);
+            }
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const int e = e0 + u * nthr;
+                if (e >= total4) continue;
+                const int k = e / r4, rb = (e - k * r4) << 2;
+                const int kc = k >> 5, kk = k & 31;
+                const float vv[4] = {v[u].x, v[u].y, v[u].z, v[u].w};
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const int r = rb + j;
+                    uint32_t t;
+                    asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(t) : "f"(vv[j]));
+                    const int off = r * 128 + (((kk >> 2) ^ (r & 7)) << 4) + ((kk & 3) << 2);
+                    *reinterpret_cast<uint32_t *>(u_smem + (size_t)kc * u_region + off) = t;
+                }
+            }
+        }
+        fence_proxy_async();      // make the generic-proxy writes of U visible to the tensor core
+        asm volatile("bar.sync 1, %0;" ::"n"(THREADS - 32) : "memory");
+    }
 
     const int my_tiles = (a.ntiles > (int)blockIdx.x) ? (a.ntiles - 1 - (int)blockIdx.x) / (int)gridDim.x + 1 : 0;
 
