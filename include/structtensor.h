@@ -70,7 +70,7 @@ typedef enum { ST_OP_SYM_MOMENT2 = 0, ST_OP_SYM_MOMENT3 = 1, ST_OP_MTTKRP_TRI = 
 /* flags (bit mask) */
 #define ST_FLAG_DENSE_CONTROL 1u /* run the same kernel over the dense, unstructured iteration
                                     space (a control for measurements; see each call) */
-#define ST_FLAG_TC_TF32       2u /* st_ttm_blockdiag: tensor cores, operands read as TF32 */
+#define ST_FLAG_TC_TF32       2u /* st_ttm_blockdiag, st_mttkrp_tri: tensor cores, operands read as TF32 */
 
 typedef struct {
     int32_t kind;      /* st_kind */
@@ -168,7 +168,9 @@ st_status st_sym_moment3_static(const float *X, int64_t N, int64_t d, int64_t ld
  * B_U(i,j,k) = (0<=i<I)*(i<=j<I)*(0<=k<K):
  *     A[i,r] = sum_{j>=i} sum_k Bp[p(i,j), k] * C[j,r] * D[k,r]
  * Bp: packed [I(I+1)/2, K] fp32 (ST_TRI_UPPER with inner=K); C: [I,R]; D: [K,R];
- * A: [I,R] fp32 (dense: its unique set is every (i,r)).  Needs K % 4 == 0, R in {8,16,32,64}.
+ * A: [I,R] fp32 (dense: its unique set is every (i,r)).  Needs K % 4 == 0, R in {8,16,32,64},
+ * I <= 32768.  ST_FLAG_TC_TF32 selects the tensor-core path (Bp truncated and D rounded to TF32,
+ * fp32 accumulation, the product with C in fp32; 5e-3 tolerance; needs R % 32 == 0, R <= 256).
  * ST_FLAG_DENSE_CONTROL: Bp is instead a dense [I,I,K] tensor and all j are visited. */
 st_status st_mttkrp_tri(const float *Bp, int64_t I, int64_t K, const float *C, const float *D,
                         int64_t R, float *A, void *ws, size_t ws_bytes, unsigned flags,

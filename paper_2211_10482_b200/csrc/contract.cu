@@ -21,6 +21,8 @@ namespace st {
 
 st_status ttm_tf32_tc(const float *Bp, int64_t rows, int64_t K, const float *U, int64_t R, float *Ap, void *ws,
                       size_t ws_bytes, cudaStream_t stream);
+st_status mttkrp_tf32_tc(const float *Bp, int64_t I, int64_t K, const float *C, const float *D, int64_t R, float *A,
+                         bool dense, void *ws, size_t ws_bytes, cudaStream_t stream);
 
 constexpr int RG_THREADS = 256;
 constexpr int RG_KC = 32;         // k-values per stage
@@ -303,12 +305,14 @@ st_status st_mttkrp_tri(const float *Bp, int64_t I, int64_t K, const float *C, c
                         float *A, void *ws, size_t ws_bytes, unsigned flags, void *stream)
 {
     using namespace st;
-    (void)ws; (void)ws_bytes;
     if (!Bp || !C || !D || !A) return ST_ERR_NULL;
     if (I <= 0 || K <= 0 || R <= 0) return ST_ERR_SHAPE;
-    if (flags & ~(ST_FLAG_DENSE_CONTROL)) return ST_ERR_UNSUPPORTED;
+    if (flags & ~(ST_FLAG_DENSE_CONTROL | ST_FLAG_TC_TF32)) return ST_ERR_UNSUPPORTED;
     if (!aligned16(Bp) || !aligned16(C) || !aligned16(D) || !aligned16(A)) return ST_ERR_ALIGN;
-    if (I > (1 << 20) || K > (1 << 20) || K % 4 != 0) return ST_ERR_UNSUPPORTED;
+    if (I > (1 << 15) || K > (1 << 20) || K % 4 != 0) return ST_ERR_UNSUPPORTED;
+    if (flags & ST_FLAG_TC_TF32)
+        return mttkrp_tf32_tc(Bp, I, K, C, D, R, A, (flags & ST_FLAG_DENSE_CONTROL) != 0, ws, ws_bytes,
+                              (cudaStream_t)stream);
     if (R != 8 && R != 16 && R != 32 && R != 64) return ST_ERR_UNSUPPORTED;
     const bool dense = (flags & ST_FLAG_DENSE_CONTROL) != 0;
     RgArgs a{};

@@ -10,6 +10,7 @@
 // in tensor memory, double buffered so that the epilogue of one tile overlaps the MMAs of the
 // next.  Warp roles: warp 0 TMA producer, warp 1 MMA issuer / TMEM owner, warps 2..5 epilogue.
 #include "tc_common.cuh"
+#include "st_index.cuh"
 
 namespace st {
 
@@ -21,8 +22,12 @@ constexpr int THREADS = 192;
 constexpr int MAX_STAGES = 10;
 }  // namespace ttmtc
 
+enum { TC_TTM = 0, TC_MTTKRP_PACKED = 1, TC_MTTKRP_DENSE = 2 };
+
 struct TtmTcArgs {
     const float *U;
+    const float *C;      // MTTKRP: [I, R]
+    int I, mode;
     float *out;
     unsigned *status;
     int64_t rows;
@@ -166,16 +171,69 @@ ttm_tc_kernel(const __grid_constant__ CUtensorMap tmap, const TtmTcArgs a)
             if (!mbar_wait(&acc_full[buf], (uint32_t)((t >> 1) & 1), abort_flag, a.status, 4)) break;
             tc_fence_after();
             const int64_t row = tile * BM + q * 32 + lane;
-            float *dst = a.out + row * a.R;
-            for (int c0 = 0; c0 < a.R; c0 += 32) {
-                uint32_t r[32];
-                tmem_ld_32x32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * a.R + c0), r);
-                tmem_ld_wait();
-                if (row < a.rows) {
+            if (a.mode == TC_TTM) {
+                float *dst = a.out + row * a.R;
+                for (int c0 = 0; c0 < a.R; c0 += 32) {
+                    uint32_t r[32];
+                    tmem_ld_32x32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * a.R + c0), r);
+                    tmem_ld_wait();
+                    if (row < a.rows) {
 #pragma unroll
-                    for (int e = 0; e < 32; e += 4)
-                        if (c0 + e < a.R)
-                            *reinterpret_cast<uint4 *>(dst + c0 + e) = make_uint4(r[e], r[e + 1], r[e + 2], r[e + 3]);
+                        for (int e = 0; e < 32; e += 4)
+                            if (c0 + e < a.R)
+                                *reinterpret_cast<uint4 *>(dst + c0 + e) = make_uint4(r[e], r[e + 1], r[e + 2], r[e + 3]);
+                    }
+                }
+            } else {
+                // MTTKRP: this lane's fibre is packed row p(i,j); scale by C[j,:] and add into A[i,:].
+                // The 32 fibres of a warp are consecutive, so they usually share i: then the warp sums
+                // them with a transposing shuffle reduction and issues one atomic per column.
+                const bool valid = row < a.rows;
+                int64_t gi = -1, gj = 0;
+                if (valid) {
+                    if (a.mode == TC_MTTKRP_PACKED) tri_decode(a.I, row, gi, gj);
+                    else { gi = row / a.I; gj = row - gi * a.I; }
+                }
+                const int gi32 = (int)gi;
+                const bool uniform = __shfl_sync(0xffffffffu, gi32, 0) == __shfl_sync(0xffffffffu, gi32, 31) && gi32 >= 0;
+                for (int c0 = 0; c0 < a.R; c0 += 32) {
+                    uint32_t r[32];
+                    tmem_ld_32x32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * a.R + c0), r);
+                    tmem_ld_wait();
+                    float v[32];
+                    if (valid) {
+                        const float4 *crow = reinterpret_cast<const float4 *>(a.C + gj * a.R + c0);
+#pragma unroll
+                        for (int e = 0; e < 8; ++e) {
+                            const float4 c = __ldg(crow + e);
+                            v[4 * e + 0] = c.x * __uint_as_float(r[4 * e + 0]);
+                            v[4 * e + 1] = c.y * __uint_as_float(r[4 * e + 1]);
+                            v[4 * e + 2] = c.z * __uint_as_float(r[4 * e + 2]);
+                            v[4 * e + 3] = c.w * __uint_as_float(r[4 * e + 3]);
+                        }
+                    } else {
+#pragma unroll
+                        for (int e = 0; e < 32; ++e) v[e] = 0.f;
+                    }
+                    if (uniform) {
+                        // after the step with offset o a lane keeps the half of its columns selected by
+                        // bit o of its lane index; at the end lane l holds the sum of column l
+#define ST_TR_STEP(OFF)                                                                       \
+    {                                                                                         \
+        const bool up = (lane & OFF) != 0;                                                    \
+        _Pragma("unroll") for (int j = 0; j < OFF; ++j) {                                     \
+            const float send = up ? v[j] : v[j + OFF];                                        \
+            const float keep = up ? v[j + OFF] : v[j];                                        \
+            v[j] = keep + __shfl_xor_sync(0xffffffffu, send, OFF);                            \
+        }                                                                                     \
+    }
+                        ST_TR_STEP(16) ST_TR_STEP(8) ST_TR_STEP(4) ST_TR_STEP(2) ST_TR_STEP(1)
+#undef ST_TR_STEP
+                        atomicAdd(a.out + (int64_t)gi32 * a.R + c0 + lane, v[0]);
+                    } else if (valid) {
+#pragma unroll
+                        for (int e = 0; e < 32; ++e) atomicAdd(a.out + gi * a.R + c0 + e, v[e]);
+                    }
                 }
             }
             tc_fence_before();
@@ -226,8 +284,28 @@ size_t ttm_tf32_tc_workspace(int64_t rows, int64_t K, int64_t R)
     return ttm_tc_plan(K, R).ok ? kWsHeaderBytes : 0;
 }
 
+static st_status tc_rows_launch(const float *Bp, int64_t rows, int64_t K, const float *U, int64_t R, float *Ap,
+                                const float *C, int64_t I, int mode, void *ws, size_t ws_bytes, cudaStream_t stream);
+
 st_status ttm_tf32_tc(const float *Bp, int64_t rows, int64_t K, const float *U, int64_t R, float *Ap, void *ws,
                       size_t ws_bytes, cudaStream_t stream)
+{
+    return tc_rows_launch(Bp, rows, K, U, R, Ap, nullptr, 0, TC_TTM, ws, ws_bytes, stream);
+}
+
+// MTTKRP on tensor cores: the same streaming kernel with W = D; the epilogue scales every fibre's
+// result by C[j,:] and adds it into A[i,:] (A is zeroed first).  TF32 operands, 5e-3 tolerance.
+st_status mttkrp_tf32_tc(const float *Bp, int64_t I, int64_t K, const float *C, const float *D, int64_t R, float *A,
+                         bool dense, void *ws, size_t ws_bytes, cudaStream_t stream)
+{
+    if (R % 32 != 0) return ST_ERR_UNSUPPORTED;
+    if (cudaMemsetAsync(A, 0, (size_t)I * R * sizeof(float), stream) != cudaSuccess) return ST_ERR_CUDA;
+    const int64_t rows = dense ? I * I : tri_rows(I);
+    return tc_rows_launch(Bp, rows, K, D, R, A, C, I, dense ? TC_MTTKRP_DENSE : TC_MTTKRP_PACKED, ws, ws_bytes, stream);
+}
+
+static st_status tc_rows_launch(const float *Bp, int64_t rows, int64_t K, const float *U, int64_t R, float *Ap,
+                                const float *C, int64_t I, int mode, void *ws, size_t ws_bytes, cudaStream_t stream)
 {
     using namespace ttmtc;
     const TtmTcPlan p = ttm_tc_plan(K, R);
@@ -244,7 +322,7 @@ st_status ttm_tf32_tc(const float *Bp, int64_t rows, int64_t K, const float *U, 
         return ST_ERR_CUDA;
     if (cudaMemsetAsync(ws, 0, kWsHeaderBytes, stream) != cudaSuccess) return ST_ERR_CUDA;
     TtmTcArgs a;
-    a.U = U; a.out = Ap; a.status = (unsigned *)ws; a.rows = rows; a.K = (int)K; a.R = (int)R;
+    a.U = U; a.C = C; a.I = (int)I; a.mode = mode; a.out = Ap; a.status = (unsigned *)ws; a.rows = rows; a.K = (int)K; a.R = (int)R;
     a.kchunks = p.kchunks; a.stages = p.stages; a.tmem_cols = p.tmem_cols;
     a.ntiles = (int)((rows + BM - 1) / BM);
     if (cudaFuncSetAttribute(ttm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)p.smem) != cudaSuccess)

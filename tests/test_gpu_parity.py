@@ -385,3 +385,23 @@ def test_moment2_bf16_all_tiles_midsize(st):
     T, S = oracle.moment2_at(Xb, ii, jj)
     pos = ii * (2 * d - ii + 1) // 2 + (jj - ii)
     assert oracle.rel_err(got[pos], T, S) <= TOL_F32
+
+
+@pytest.mark.parametrize("I,K,R", [(1, 4, 32), (5, 36, 32), (16, 64, 64), (40, 100, 32), (70, 32, 96), (33, 68, 64)])
+def test_mttkrp_tf32_tensor_core_small(st, I, K, R):
+    Bp, C, D = workloads.mttkrp_inputs(I, K, R)
+    Bd = oracle.unpack(Bp.reshape(-1), oracle.KIND_TRI, I, inner=K)
+    A, S = oracle.mttkrp(Bd, C, D)
+    got = st.st_mttkrp_tri(dev(Bp), dev(C), dev(D), flags=st.ST_FLAG_TC_TF32).cpu().numpy()
+    assert oracle.rel_err(got, A, S) <= TOL_TC
+    ctl = st.st_mttkrp_tri(dev(Bd), dev(C), dev(D), flags=st.ST_FLAG_TC_TF32 | st.ST_FLAG_DENSE_CONTROL).cpu().numpy()
+    assert oracle.rel_err(ctl, A, S) <= TOL_TC
+
+
+def test_mttkrp_tf32_config(st):
+    Bp, C, D = workloads.mttkrp_inputs()
+    got = st.st_mttkrp_tri(dev(Bp), dev(C), dev(D), flags=st.ST_FLAG_TC_TF32).cpu().numpy()
+    Bd = oracle.unpack(Bp.reshape(-1), oracle.KIND_TRI, 512, inner=512)
+    for i0 in (0, 1, 255, 256, 300, 480, 510, 511):
+        A, S = oracle.mttkrp(Bd, C, D, i0, i0 + 1)
+        assert oracle.rel_err(got[i0:i0 + 1], A, S) <= TOL_TC, i0
