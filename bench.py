@@ -76,7 +76,8 @@ def step_table(cfg):
     nnz3 = tri(c3["I"]) * c3["K"]
     t["pack_tri_x_k"] = dict(flops=0, bytes=2 * 4 * nnz3, bound="hbm", launches=1)
     t["mttkrp_tri"] = dict(flops=2 * c3["R"] * nnz3 + 2 * c3["R"] * tri(c3["I"]),
-                           bytes=4 * (nnz3 + (2 * c3["I"] + c3["K"]) * c3["R"]), bound="alu", launches=1)
+                           bytes=4 * (nnz3 + (2 * c3["I"] + c3["K"]) * c3["R"]),
+                           bound=("hbm" if cfg["mttkrp_tc"] else "alu"), launches=1)
     rows4 = c4["nb"] * c4["bs"] ** 2
     t["ttm_blockdiag"] = dict(flops=2 * rows4 * c4["K"] * c4["R"],
                               bytes=4 * (rows4 * (c4["K"] + c4["R"]) + c4["K"] * c4["R"]),
@@ -171,6 +172,7 @@ def bench_config():
     cfg["band"] = dict(d=2048, kl=64, ku=63, inner=16)
     cfg["m2_large_dtype"] = "bf16"
     cfg["ttm_tc"] = True
+    cfg["mttkrp_tc"] = True
     return cfg
 
 
@@ -220,6 +222,7 @@ class Workload:
             "m2l": torch.empty(tri(c5["d"]), **f32), "m2l_dense": torch.empty(c5["d"] ** 2, **f32),
         }
         self.ttm_flags = st.ST_FLAG_TC_TF32 if cfg["ttm_tc"] else 0
+        self.mttkrp_flags = st.ST_FLAG_TC_TF32 if cfg["mttkrp_tc"] else 0
         x5dt = st.ST_BF16 if cfg["m2_large_dtype"] == "bf16" else st.ST_F32
         wsb = max(
             st.st_workspace_bytes(st.ST_OP_SYM_MOMENT2, c1["N"], c1["d"], st.ST_F32),
@@ -242,7 +245,8 @@ class Workload:
             ("sym_moment3", lambda: st.st_sym_moment3(d["X2"], out=o["m3"], ws=self.ws)),
             ("unpack_tet_sym", lambda: st.st_unpack(o["m3"], self.lay2, st.ST_FILL_SYMMETRIC, out=o["m3_dense"])),
             ("pack_tri_x_k", lambda: st.st_pack(d["B3"], self.lay3, out=o["Bp3"])),
-            ("mttkrp_tri", lambda: st.st_mttkrp_tri(o["Bp3"], d["C3"], d["D3"], out=o["A3"], ws=self.ws)),
+            ("mttkrp_tri", lambda: st.st_mttkrp_tri(o["Bp3"], d["C3"], d["D3"], out=o["A3"], ws=self.ws,
+                                                       flags=self.mttkrp_flags)),
             ("ttm_blockdiag", lambda: st.st_ttm_blockdiag(d["Bp4"], d["U4"], c4["nb"], c4["bs"], out=o["Ap4"],
                                                           ws=self.ws, flags=self.ttm_flags)),
             ("unpack_blockdiag", lambda: st.st_unpack(o["Ap4"].view(-1), self.lay4, out=o["A4_dense"])),
@@ -283,6 +287,8 @@ def run_ours(args):
         cfg["m2_large_dtype"] = "f32"
     if st.st_workspace_bytes(st.ST_OP_TTM_BLOCKDIAG, 64, 64, 256, 64, st.ST_FLAG_TC_TF32) == 0 or args.ttm == "f32":
         cfg["ttm_tc"] = False
+    if args.mttkrp == "f32":
+        cfg["mttkrp_tc"] = False
     w = Workload(cfg, device, st, torch)
     table = step_table(cfg)
     calls = w.calls()
@@ -322,7 +328,6 @@ def run_ours(args):
     t1.record()
     barrier()
     total_ms = t0.elapsed_time(t1)
-    clocks = sampler.stop() if rank == 0 else None
     per_call_us = {n: float(np.mean([ev[s][i][0].elapsed_time(ev[s][i][1]) for s in range(args.steps)])) * 1e3
                    for i, n in enumerate(names)}
 
@@ -339,6 +344,7 @@ def run_ours(args):
     e1.record()
     barrier()
     e2e_ms = e0.elapsed_time(e1)
+    clocks = sampler.stop() if rank == 0 else None   # sampled over both timed regions
 
     if world > 1:
         tt = torch.tensor([total_ms, e2e_ms], device=device, dtype=torch.float64)
@@ -375,12 +381,13 @@ def run_ours(args):
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-        "dtype": "f32" + ("+bf16" if cfg["m2_large_dtype"] == "bf16" else "") + ("+tf32" if cfg["ttm_tc"] else ""),
+        "dtype": "f32" + ("+bf16" if cfg["m2_large_dtype"] == "bf16" else "") + ("+tf32" if (cfg["ttm_tc"] or cfg["mttkrp_tc"]) else ""),
         "data": "synthetic",
         "config": {"workload": "all five named configurations in one step: sym_moment2 [4096,64], sym_moment3 "
-                               "[65536,64], mttkrp_tri I=K=512 R=32, ttm_blockdiag 64x(64x64) K=256 R=64, "
+                               "[65536,64], mttkrp_tri I=K=512 R=32 (%s), ttm_blockdiag 64x(64x64) K=256 R=64 (%s), "
                                "sym_moment2 large [1048576,1024] %s; plus pack/unpack of their operands"
-                               % cfg["m2_large_dtype"],
+                               % ("tf32" if cfg["mttkrp_tc"] else "f32", "tf32" if cfg["ttm_tc"] else "f32",
+                                  cfg["m2_large_dtype"]),
                    "l2": "inputs larger than L2 (each step streams >2.5 GB between two uses of any buffer)",
                    "replicas": "independent replicas, no collective" if world > 1 else "single GPU"},
         "roofline": roof,
@@ -499,6 +506,7 @@ def main():
     ap.add_argument("--cpu-budget", type=float, default=15.0)
     ap.add_argument("--m2-large", default="bf16", choices=["bf16", "f32"])
     ap.add_argument("--ttm", default="tf32", choices=["tf32", "f32"])
+    ap.add_argument("--mttkrp", default="tf32", choices=["tf32", "f32"])
     args = ap.parse_args()
     if args.warmup < 3 and args.impl == "ours":
         args.warmup = 3
