@@ -74,7 +74,7 @@ def step_table(cfg):
     c1, c2, c3, c4, c5 = (cfg[k] for k in ("moment2", "moment3", "mttkrp", "ttm", "moment2_large"))
     t = {}
     t["sym_moment2"] = dict(flops=2 * c1["N"] * tri(c1["d"]), bytes=4 * (c1["N"] * c1["d"] + tri(c1["d"])),
-                            bound="alu", launches=1)
+                            bound="alu", launches=2)
     t["unpack_tri_sym"] = dict(flops=0, bytes=4 * (tri(c1["d"]) + c1["d"] ** 2), bound="hbm", launches=1)
     t["sym_moment3"] = dict(flops=2 * c2["N"] * tet(c2["d"]) + c2["N"] * tri(c2["d"]),
                             bytes=4 * (c2["N"] * c2["d"] + tet(c2["d"])), bound="alu", launches=2)

@@ -5,8 +5,8 @@
 // never launched, and on diagonal tiles only the 136 of 256 4x4 register blocks that touch
 // i<=j are computed.  The samples are split over gridDim.y; every CTA stages 32-row slices
 // of its two column panels in shared memory, accumulates a 4x4 block per thread, and
-// writes a partial tile to the workspace.  The CTA that arrives last at a tile's counter
-// adds the partials in a fixed order (deterministic result) and writes the packed output.
+// writes a partial tile to the workspace.  A second kernel adds the partials of every tile in
+// a fixed order (deterministic result) and writes the packed output.
 #include "st_common.cuh"
 #include "st_index.cuh"
 
@@ -17,7 +17,7 @@ st_status moment2_bf16_tc(const void *X, int64_t N, int64_t d, int64_t ldx, floa
 size_t moment2_bf16_tc_workspace(int64_t N, int64_t d, unsigned flags);
 
 constexpr int M2_T = 64;    // output tile edge
-constexpr int M2_KC = 32;   // sample rows staged per step
+constexpr int M2_KC = 64;   // sample rows staged per step
 
 struct M2Plan {
     int nt;          // tiles per edge
@@ -34,9 +34,9 @@ static M2Plan moment2_plan(int64_t N, int64_t d, unsigned flags)
     p.ntiles = (flags & ST_FLAG_DENSE_CONTROL) ? p.nt * p.nt : p.nt * (p.nt + 1) / 2;
     const int sms = sm_count_or_default();
     int64_t want = (2 * (int64_t)sms + p.ntiles - 1) / p.ntiles;   // about two CTAs per SM
-    int64_t max_split = (N + 4 * M2_KC - 1) / (4 * M2_KC);         // at least 128 rows per split
+    int64_t max_split = (N + M2_KC - 1) / M2_KC;                   // at least one stage of rows per split
     if (want > max_split) want = max_split;
-    if (want > 64) want = 64;
+    if (want > 128) want = 128;
     if (want < 1) want = 1;
     int64_t rows = (N + want - 1) / want;
     rows = (rows + M2_KC - 1) / M2_KC * M2_KC;
@@ -50,12 +50,10 @@ static M2Plan moment2_plan(int64_t N, int64_t d, unsigned flags)
 template <bool DENSE>
 __global__ void __launch_bounds__(256)
 moment2_f32_kernel(const float *__restrict__ X, int64_t N, int d, int64_t ldx, float *__restrict__ out,
-                   float *__restrict__ partials, unsigned *__restrict__ tickets, int nt, int nsplit,
-                   int64_t rows_per_split)
+                   float *__restrict__ partials, int nt, int nsplit, int64_t rows_per_split)
 {
     __shared__ __align__(16) float As[M2_KC][M2_T];
     __shared__ __align__(16) float Bs[M2_KC][M2_T];
-    __shared__ int s_last;
 
     const int tile = blockIdx.x;
     int bi, bj;
@@ -104,7 +102,7 @@ moment2_f32_kernel(const float *__restrict__ X, int64_t N, int d, int64_t ldx, f
     for (int64_t n0 = n_begin; n0 < n_end; n0 += M2_KC) {
         // stage rows n0..n0+31 of both column panels (zero beyond N and beyond d)
         for (int e = tid; e < M2_KC * M2_T; e += 256) {
-            const int r = e >> 6, c = e & 63;
+            const int r = e >> 6, c = e & 63;   // M2_T == 64
             const int64_t n = n0 + r;
             const bool row_ok = n < n_end;
             As[r][c] = (row_ok && col_a + c < d) ? X[n * ldx + col_a + c] : 0.f;
@@ -134,35 +132,43 @@ moment2_f32_kernel(const float *__restrict__ X, int64_t N, int d, int64_t ldx, f
             *reinterpret_cast<float4 *>(&mine[(ty * 4 + r) * M2_T + tx * 4]) =
                 make_float4(acc[r][0], acc[r][1], acc[r][2], acc[r][3]);
     }
-    __threadfence();
-    __syncthreads();
-    if (tid == 0) s_last = (atomicAdd(&tickets[tile], 1u) == (unsigned)(nsplit - 1));
-    __syncthreads();
-    if (!s_last) return;
-    __threadfence();
+}
 
-    // last arrival: fixed-order sum of the partial tiles, written to the packed upper triangle.
-    // Four columns per thread and eight independent loads in flight hide the L2 latency.
+// out[p(i,j)] = sum over the splits of a tile, in split order; i <= j only.
+__global__ void __launch_bounds__(256)
+moment2_f32_reduce_kernel(const float *__restrict__ partials, float *__restrict__ out, int d, int nt, int nsplit,
+                          int dense)
+{
+    const int tile = blockIdx.x;
+    int bi, bj;
+    if (dense) {
+        bi = tile / nt;
+        bj = tile - bi * nt;
+    } else {
+        int64_t a, b;
+        tri_decode(nt, tile, a, b);
+        bi = (int)a;
+        bj = (int)b;
+    }
+    if (bi > bj) return;                                        // dense control: lower tiles are discarded
+    const int col_a = bi * M2_T, col_b = bj * M2_T;
     const float *base = partials + (size_t)tile * nsplit * (M2_T * M2_T);
-    for (int e4 = tid; e4 < M2_T * M2_T / 4; e4 += 256) {
-        const int r = e4 >> 4, c = (e4 & 15) << 2;
+    // one output per thread and up to 32 independent loads in flight: after the other kernels of
+    // a pipeline have streamed gigabytes, every dependent round trip to memory costs microseconds
+    for (int e = blockIdx.y * 256 + threadIdx.x; e < M2_T * M2_T; e += gridDim.y * 256) {
+        const int r = e >> 6, c = e & 63;
         const int gi = col_a + r, gj = col_b + c;
-        if (gi >= d || gj >= d || gj + 3 < gi) continue;       // nothing of this group is in i <= j
-        float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
-        const float4 *p4 = reinterpret_cast<const float4 *>(base) + e4;
-        for (int k0 = 0; k0 < nsplit; k0 += 8) {
-            float4 v[8];                                        // eight loads issued before the first add
+        if (gi >= d || gj >= d || gi > gj) continue;
+        float s = 0.f;
+        const float *p1 = base + e;
+        for (int k0 = 0; k0 < nsplit; k0 += 32) {
+            float v[32];
 #pragma unroll
-            for (int u = 0; u < 8; ++u)
-                v[u] = (k0 + u < nsplit) ? __ldcg(p4 + (size_t)(k0 + u) * (M2_T * M2_T / 4))
-                                         : make_float4(0.f, 0.f, 0.f, 0.f);
+            for (int u = 0; u < 32; ++u) v[u] = (k0 + u < nsplit) ? __ldcg(p1 + (size_t)(k0 + u) * (M2_T * M2_T)) : 0.f;
 #pragma unroll
-            for (int u = 0; u < 8; ++u) { s.x += v[u].x; s.y += v[u].y; s.z += v[u].z; s.w += v[u].w; }
+            for (int u = 0; u < 32; ++u) s += v[u];
         }
-        const float sv[4] = {s.x, s.y, s.z, s.w};
-#pragma unroll
-        for (int q = 0; q < 4; ++q)
-            if (gj + q < d && gi <= gj + q) out[tri_encode(d, gi, gj + q)] = sv[q];
+        out[tri_encode(d, gi, gj)] = s;
     }
 }
 
@@ -175,16 +181,17 @@ static st_status moment2_f32(const float *X, int64_t N, int64_t d, int64_t ldx, 
     if (!ws || ws_bytes < need) return ST_ERR_WORKSPACE;
     if (!aligned256(ws)) return ST_ERR_ALIGN;
     unsigned char *w = (unsigned char *)ws;
-    if (cudaMemsetAsync(w, 0, kWsHeaderBytes + p.ticket_bytes, stream) != cudaSuccess) return ST_ERR_CUDA;
-    unsigned *tickets = (unsigned *)(w + kWsHeaderBytes);
     float *partials = (float *)(w + kWsHeaderBytes + p.ticket_bytes);
     dim3 grid(p.ntiles, p.nsplit);
-    if (flags & ST_FLAG_DENSE_CONTROL)
-        moment2_f32_kernel<true><<<grid, 256, 0, stream>>>(X, N, (int)d, ldx, out, partials, tickets, p.nt,
-                                                           p.nsplit, p.rows_per_split);
+    const int dense = (flags & ST_FLAG_DENSE_CONTROL) ? 1 : 0;
+    if (dense)
+        moment2_f32_kernel<true><<<grid, 256, 0, stream>>>(X, N, (int)d, ldx, out, partials, p.nt, p.nsplit,
+                                                           p.rows_per_split);
     else
-        moment2_f32_kernel<false><<<grid, 256, 0, stream>>>(X, N, (int)d, ldx, out, partials, tickets, p.nt,
-                                                            p.nsplit, p.rows_per_split);
+        moment2_f32_kernel<false><<<grid, 256, 0, stream>>>(X, N, (int)d, ldx, out, partials, p.nt, p.nsplit,
+                                                            p.rows_per_split);
+    if (cudaGetLastError() != cudaSuccess) return ST_ERR_CUDA;
+    moment2_f32_reduce_kernel<<<dim3(p.ntiles, 16), 256, 0, stream>>>(partials, out, (int)d, p.nt, p.nsplit, dense);
     return launch_status();
 }
 

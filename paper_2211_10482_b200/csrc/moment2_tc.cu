@@ -95,6 +95,12 @@ moment2_tc_kernel(const __grid_constant__ CUtensorMap tmap, float *__restrict__ 
             mbar_init(&acc_empty[b], 4);     // one arrival per epilogue warp
         }
         *abort_flag = 0;
+        if (blockIdx.x == 0) {
+            // the status words are cleared here instead of by a separate memset; a time-out
+            // report can only be written 2^24 failed polls later
+            status[kWsStatusWord] = 0;
+            status[kWsDetailWord] = 0;
+        }
         fence_barrier_init();
     }
     if (warp == 1) {
@@ -297,6 +303,12 @@ moment2_tc_pair_kernel(const __grid_constant__ CUtensorMap tmap, float *__restri
             mbar_init(&acc_empty[b], 8);     // four epilogue warps in each of the two blocks (leader's copy is used)
         }
         *abort_flag = 0;
+        if (blockIdx.x == 0) {
+            // the status words are cleared here instead of by a separate memset; a time-out
+            // report can only be written 2^24 failed polls later
+            status[kWsStatusWord] = 0;
+            status[kWsDetailWord] = 0;
+        }
         fence_barrier_init();
     }
     if (warp == 1) {
@@ -556,7 +568,6 @@ st_status moment2_bf16_tc(const void *X, int64_t N, int64_t d, int64_t ldx, floa
         if (!tc::make_tmap_2d(&tm2, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, X, (uint64_t)N, (uint64_t)d, (uint64_t)ldx * 2,
                               BOXC, KROWS))
             return ST_ERR_CUDA;
-        if (cudaMemsetAsync(ws, 0, kWsHeaderBytes, stream) != cudaSuccess) return ST_ERR_CUDA;
         float *part2 = (float *)((unsigned char *)ws + kWsHeaderBytes);
         if (cudaFuncSetAttribute(moment2_tc_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  (int)m2tc2::SMEM_BYTES) != cudaSuccess)
@@ -590,7 +601,6 @@ st_status moment2_bf16_tc(const void *X, int64_t N, int64_t d, int64_t ldx, floa
     if (!tc::make_tmap_2d(&tmap, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, X, (uint64_t)N, (uint64_t)d, (uint64_t)ldx * 2,
                           BOXC, KROWS))
         return ST_ERR_CUDA;
-    if (cudaMemsetAsync(ws, 0, kWsHeaderBytes, stream) != cudaSuccess) return ST_ERR_CUDA;
     float *partials = (float *)((unsigned char *)ws + kWsHeaderBytes);
     if (cudaFuncSetAttribute(moment2_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES) !=
         cudaSuccess)

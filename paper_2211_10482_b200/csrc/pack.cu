@@ -143,7 +143,8 @@ __device__ __forceinline__ void slice_run(const LayoutArgs &a, int64_t s, int64_
 
 template <int KIND, typename U, bool PACK>
 __global__ void __launch_bounds__(256)
-slice_copy_kernel(const U *__restrict__ src, U *__restrict__ dst, LayoutArgs a, int group_shift, int parts)
+slice_copy_kernel(const U *__restrict__ src, U *__restrict__ dst, LayoutArgs a, int group_shift, int parts,
+                  int64_t part_units)
 {
     const int g = 1 << group_shift;
     const int lane = (int)(threadIdx.x & (g - 1));
@@ -151,16 +152,18 @@ slice_copy_kernel(const U *__restrict__ src, U *__restrict__ dst, LayoutArgs a, 
     const int64_t ngroups = ((int64_t)gridDim.x * blockDim.x) >> group_shift;
     const int64_t nslices = (KIND == ST_TET) ? a.d * a.d : a.d;
     const int64_t su = a.d * a.chunks;                        // units per dense slice
-    const int64_t part_units = (su + parts - 1) / parts;
     for (int64_t item = gid; item < nslices * parts; item += ngroups) {
         const int64_t s = item / parts;
         const int64_t part = item - s * parts;
         int64_t lo, hi, prow;
         slice_run<KIND>(a, s, lo, hi, prow);
-        const int64_t u0 = part * part_units;                 // this part covers dense units [u0, u1) of the slice
-        int64_t u1 = u0 + part_units;
-        if (u1 > su) u1 = su;
         const int64_t c0 = lo * a.chunks, c1 = hi * a.chunks;  // units of the run inside the slice
+        // pack splits the run itself into parts, unpack the whole dense slice (it writes all of it)
+        const int64_t r0 = PACK ? c0 : 0, r1 = PACK ? c1 : su;
+        int64_t u0 = r0 + part * part_units;                  // this part covers dense units [u0, u1) of the slice
+        int64_t u1 = u0 + part_units;
+        if (u0 > r1) u0 = r1;
+        if (u1 > r1) u1 = r1;
         const int64_t x0 = u0 > c0 ? u0 : c0, x1 = u1 < c1 ? u1 : c1;   // run clipped to this part
         if (PACK) {
             const U *in = src + s * su;
@@ -240,8 +243,12 @@ static st_status launch_copy(const void *src, void *dst, const LayoutArgs &a, cu
         structured_copy_kernel<KIND, U, PACK><<<grid, 256, 0, s>>>((const U *)src, (U *)dst, a, shift);
         return launch_status();
     }
-    // slices: about 8 units per thread, at most 8192 units per (slice, part)
-    const int64_t su = a.d * a.chunks;
+    // slices: about 8 units per thread, at most 8192 units per (slice, part).  Pack splits the
+    // longest run of unique columns, unpack the whole dense slice.
+    int64_t run_rows = a.d;
+    if (KIND == ST_BAND) run_rows = a.width < a.d ? a.width : a.d;
+    if (KIND == ST_BLOCKDIAG) run_rows = a.bs;
+    const int64_t su = (PACK ? run_rows : a.d) * a.chunks;
     int parts = (int)((su + 8191) / 8192);
     if (parts < 1) parts = 1;
     const int64_t pu = (su + parts - 1) / parts;
@@ -251,7 +258,7 @@ static st_status launch_copy(const void *src, void *dst, const LayoutArgs &a, cu
     const int64_t threads = (nslices * parts) << shift;
     const int64_t want = (threads + 255) / 256;
     const int grid = (int)(want < cap ? (want < 1 ? 1 : want) : cap);
-    slice_copy_kernel<KIND, U, PACK><<<grid, 256, 0, s>>>((const U *)src, (U *)dst, a, shift, parts);
+    slice_copy_kernel<KIND, U, PACK><<<grid, 256, 0, s>>>((const U *)src, (U *)dst, a, shift, parts, pu);
     return launch_status();
 }
 

@@ -63,6 +63,12 @@ ttm_tc_kernel(const __grid_constant__ CUtensorMap tmap, const TtmTcArgs a)
             mbar_init(&acc_empty[b], 4);     // one arrival per epilogue warp
         }
         *abort_flag = 0;
+        if (blockIdx.x == 0) {
+            // the status words are cleared here instead of by a separate memset; a time-out
+            // report can only be written 2^24 failed polls later
+            a.status[kWsStatusWord] = 0;
+            a.status[kWsDetailWord] = 0;
+        }
         fence_barrier_init();
     }
     if (warp == 1) {
@@ -81,17 +87,18 @@ ttm_tc_kernel(const __grid_constant__ CUtensorMap tmap, const TtmTcArgs a)
         const int nthr = THREADS - 32, t0 = threadIdx.x - 32;
         const int r4 = a.R >> 2;                                      // float4 groups per row of U
         const int total4 = a.kchunks * KC * r4;
-        for (int e0 = t0; e0 < total4; e0 += 4 * nthr) {
-            float4 v[4];
+        constexpr int UB = 8;
+        for (int e0 = t0; e0 < total4; e0 += UB * nthr) {
+            float4 v[UB];
 #pragma unroll
-            for (int u = 0; u < 4; ++u) {                             // four independent loads in flight
+            for (int u = 0; u < UB; ++u) {                            // eight independent loads in flight
                 const int e = e0 + u * nthr;
                 const int k = e / r4;
                 v[u] = (e < total4 && k < a.K) ? __ldg(reinterpret_cast<const float4 *>(a.U) + e)
                                                : make_float4(0.f, 0.f, 0.f, 0.f);
             }
 #pragma unroll
-            for (int u = 0; u < 4; ++u) {
+            for (int u = 0; u < UB; ++u) {
                 const int e = e0 + u * nthr;
                 if (e >= total4) continue;
                 const int k = e / r4, rb = (e - k * r4) << 2;
@@ -320,7 +327,6 @@ static st_status tc_rows_launch(const float *Bp, int64_t rows, int64_t K, const 
     if (!tc::make_tmap_2d(&tmap, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, Bp, (uint64_t)rows, (uint64_t)K, (uint64_t)K * 4, KC,
                           BM))
         return ST_ERR_CUDA;
-    if (cudaMemsetAsync(ws, 0, kWsHeaderBytes, stream) != cudaSuccess) return ST_ERR_CUDA;
     TtmTcArgs a;
     a.U = U; a.C = C; a.I = (int)I; a.mode = mode; a.out = Ap; a.status = (unsigned *)ws; a.rows = rows; a.K = (int)K; a.R = (int)R;
     a.kchunks = p.kchunks; a.stages = p.stages; a.tmem_cols = p.tmem_cols;
