@@ -271,6 +271,63 @@ class Workload:
             self.host_out[k].copy_(self.out[k], non_blocking=True)
 
 
+def dense_controls(w, torch, reps=5):
+    """Every compute kernel against the same kernel forced onto the dense, unstructured iteration
+    space (ST_FLAG_DENSE_CONTROL): isolated timings with an L2 flush between repetitions.  The
+    gain from structure should approach dense work / unique work."""
+    st, d, o, c = w.st, w.dev, w.out, w.cfg
+    c1, c2, c3, c4, c5 = (c[k] for k in ("moment2", "moment3", "mttkrp", "ttm", "moment2_large"))
+    DC = st.ST_FLAG_DENSE_CONTROL
+    dev = w.ws.device
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+    x5dt = st.ST_BF16 if c["m2_large_dtype"] == "bf16" else st.ST_F32
+    wsb = max(st.st_workspace_bytes(st.ST_OP_SYM_MOMENT2, c1["N"], c1["d"], st.ST_F32, 0, DC),
+              st.st_workspace_bytes(st.ST_OP_SYM_MOMENT3, c2["N"], c2["d"], 0, 0, DC),
+              st.st_workspace_bytes(st.ST_OP_SYM_MOMENT2, c5["N"], c5["d"], x5dt, 0, DC), 256)
+    wsc = torch.empty(wsb, dtype=torch.uint8, device=dev)
+    d4 = c4["nb"] * c4["bs"]
+    lay4k = st.Layout(st.ST_BLOCKDIAG, d4, inner=c4["K"], nblocks=c4["nb"], bs=c4["bs"])
+    B4_dense = st.st_unpack(d["Bp4"].view(-1), lay4k)                # 16 GiB: zeros off the diagonal blocks
+    A4_dense = torch.empty((d4 * d4, c4["R"]), dtype=torch.float32, device=dev)
+    pairs = {
+        "sym_moment2": (lambda: st.st_sym_moment2(d["X1"], out=o["m2"], ws=w.ws),
+                        lambda: st.st_sym_moment2(d["X1"], out=o["m2"], ws=wsc, flags=DC), c1["d"] ** 2 / tri(c1["d"])),
+        "sym_moment3": (lambda: st.st_sym_moment3(d["X2"], out=o["m3"], ws=w.ws),
+                        lambda: st.st_sym_moment3(d["X2"], out=o["m3"], ws=wsc, flags=DC), c2["d"] ** 3 / tet(c2["d"])),
+        "mttkrp_tri": (lambda: st.st_mttkrp_tri(o["Bp3"], d["C3"], d["D3"], out=o["A3"], ws=w.ws, flags=w.mttkrp_flags),
+                       lambda: st.st_mttkrp_tri(d["B3"], d["C3"], d["D3"], out=o["A3"], ws=w.ws,
+                                                flags=w.mttkrp_flags | DC), c3["I"] ** 2 / tri(c3["I"])),
+        "ttm_blockdiag": (lambda: st.st_ttm_blockdiag(d["Bp4"], d["U4"], c4["nb"], c4["bs"], out=o["Ap4"], ws=w.ws,
+                                                      flags=w.ttm_flags),
+                          lambda: st.st_ttm_blockdiag(B4_dense, d["U4"], c4["nb"], c4["bs"], out=A4_dense, ws=w.ws,
+                                                      flags=w.ttm_flags | DC), float(c4["nb"])),
+        "sym_moment2_large": (lambda: st.st_sym_moment2(d["X5"], out=o["m2l"], ws=w.ws),
+                              lambda: st.st_sym_moment2(d["X5"], out=o["m2l"], ws=wsc, flags=DC),
+                              c5["d"] ** 2 / tri(c5["d"])),
+    }
+
+    def timed(fn):
+        for _ in range(2):
+            fn()
+        torch.cuda.synchronize()
+        ts = []
+        for _ in range(reps):
+            flush.zero_()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(); fn(); e1.record()
+            torch.cuda.synchronize()
+            ts.append(e0.elapsed_time(e1) * 1e3)
+        return float(np.median(ts))
+
+    out = {}
+    for name, (structured, control, ideal) in pairs.items():
+        a, b = timed(structured), timed(control)
+        out[name] = {"structured_us": round(a, 2), "control_us": round(b, 2), "ratio": round(b / a, 3),
+                     "dense_over_unique": round(ideal, 3)}
+    del B4_dense, A4_dense
+    return out
+
+
 def run_ours(args):
     import torch
     import torch.distributed as dist
@@ -407,6 +464,8 @@ def run_ours(args):
                   "bf16_tflops_sustained": peaks.get("bf16_tflops_sustained"), "fp32_tflops": FP32_PEAK_TFLOPS,
                   "source": peaks["source"]},
     }
+    if world == 1 and not args.no_controls:
+        line["dense_control"] = dense_controls(w, torch)
     if rank == 0:
         if world == 1 and not args.no_cpu_baseline:
             line["cpu_baseline"] = cpu_baseline(budget_s=args.cpu_budget)
@@ -511,6 +570,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-controls", action="store_true", help="skip the dense-iteration controls")
     ap.add_argument("--cpu-budget", type=float, default=15.0)
     ap.add_argument("--m2-large", default="bf16", choices=["bf16", "f32"])
     ap.add_argument("--ttm", default="tf32", choices=["tf32", "f32"])
