@@ -328,6 +328,21 @@ def dense_controls(w, torch, reps=5):
     return out
 
 
+def max_over_ranks(values, dist, device):
+    """Element-wise maximum of a list of floats over all ranks (the slowest rank sets the time)."""
+    import torch
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return [float(v) for v in values]
+    t = torch.tensor(list(values), device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(v) for v in t]
+
+
+def whole_job_value(step_flops, world, ms_per_step):
+    """Replicas only: every rank runs the same step on its own data, so the job does world x flops."""
+    return world * step_flops / (ms_per_step * 1e-3) / 1e9
+
+
 def run_ours(args):
     import torch
     import torch.distributed as dist
@@ -409,15 +424,12 @@ def run_ours(args):
     e2e_ms = e0.elapsed_time(e1)
     clocks = sampler.stop() if rank == 0 else None   # sampled over both timed regions
 
-    if world > 1:
-        tt = torch.tensor([total_ms, e2e_ms], device=device, dtype=torch.float64)
-        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-        total_ms, e2e_ms = float(tt[0]), float(tt[1])
+    total_ms, e2e_ms = max_over_ranks([total_ms, e2e_ms], dist, device)
 
     step_flops = sum(table[n]["flops"] for n in names)
     ms_per_step = total_ms / args.steps
-    value = world * step_flops / (ms_per_step * 1e-3) / 1e9
-    e2e_value = world * step_flops / (e2e_ms / args.steps * 1e-3) / 1e9
+    value = whole_job_value(step_flops, world, ms_per_step)
+    e2e_value = whole_job_value(step_flops, world, e2e_ms / args.steps)
 
     kernels = {}
     for n in names:
