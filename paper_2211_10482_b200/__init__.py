@@ -152,10 +152,11 @@ def st_workspace_bytes(op: int, a: int, b: int, c: int = 0, e: int = 0, flags: i
     return int(lib().st_workspace_bytes(op, a, b, c, e, flags))
 
 
-def _workspace(nbytes: int, device, ws: torch.Tensor | None) -> torch.Tensor:
+def _workspace(query, device, ws: torch.Tensor | None) -> torch.Tensor:
+    """The caller's workspace, or a fresh one of the size that `query()` reports."""
     if ws is not None:
         return ws
-    return torch.empty(max(int(nbytes), 256), dtype=torch.uint8, device=device)
+    return torch.empty(max(int(query()), 256), dtype=torch.uint8, device=device)
 
 
 def st_pack(dense: torch.Tensor, layout: Layout, out: torch.Tensor | None = None) -> torch.Tensor:
@@ -192,7 +193,7 @@ def st_sym_moment2(X: torch.Tensor, out: torch.Tensor | None = None, ws: torch.T
     xdt = _dtype(X)
     if out is None:
         out = torch.empty(d * (d + 1) // 2, dtype=torch.float32, device=X.device)
-    ws = _workspace(st_workspace_bytes(ST_OP_SYM_MOMENT2, N, d, xdt, 0, flags), X.device, ws)
+    ws = _workspace(lambda: st_workspace_bytes(ST_OP_SYM_MOMENT2, N, d, xdt, 0, flags), X.device, ws)
     _check(lib().st_sym_moment2(_dev(X, "X"), xdt, N, d, X.stride(0), _dev(out, "out"), ws.data_ptr(),
                                 ws.numel() * ws.element_size(), flags, _stream()), "st_sym_moment2")
     return out
@@ -206,7 +207,7 @@ def st_sym_moment3(X: torch.Tensor, out: torch.Tensor | None = None, ws: torch.T
         raise TypeError("X must be float32")
     if out is None:
         out = torch.empty(d * (d + 1) * (d + 2) // 6, dtype=torch.float32, device=X.device)
-    ws = _workspace(st_workspace_bytes(ST_OP_SYM_MOMENT3, N, d, 0, 0, flags), X.device, ws)
+    ws = _workspace(lambda: st_workspace_bytes(ST_OP_SYM_MOMENT3, N, d, 0, 0, flags), X.device, ws)
     _check(lib().st_sym_moment3(_dev(X, "X"), N, d, X.stride(0), _dev(out, "out"), ws.data_ptr(),
                                 ws.numel() * ws.element_size(), flags, _stream()), "st_sym_moment3")
     return out
@@ -240,7 +241,7 @@ def st_mttkrp_tri(Bp: torch.Tensor, C: torch.Tensor, D: torch.Tensor, out: torch
         raise ValueError("shape mismatch")
     if out is None:
         out = torch.empty((I, R), dtype=torch.float32, device=Bp.device)
-    ws = _workspace(st_workspace_bytes(ST_OP_MTTKRP_TRI, I, K, R, 0, flags), Bp.device, ws)
+    ws = _workspace(lambda: st_workspace_bytes(ST_OP_MTTKRP_TRI, I, K, R, 0, flags), Bp.device, ws)
     _check(lib().st_mttkrp_tri(_dev(Bp, "Bp"), I, K, _dev(C, "C"), _dev(D, "D"), R, _dev(out, "out"),
                                ws.data_ptr(), ws.numel() * ws.element_size(), flags, _stream()),
            "st_mttkrp_tri")
@@ -260,7 +261,7 @@ def st_ttm_blockdiag(Bp: torch.Tensor, U: torch.Tensor, nblocks: int, bs: int,
         raise ValueError("shape mismatch")
     if out is None:
         out = torch.empty((rows, R), dtype=torch.float32, device=Bp.device)
-    ws = _workspace(st_workspace_bytes(ST_OP_TTM_BLOCKDIAG, nblocks, bs, K, R, flags), Bp.device, ws)
+    ws = _workspace(lambda: st_workspace_bytes(ST_OP_TTM_BLOCKDIAG, nblocks, bs, K, R, flags), Bp.device, ws)
     _check(lib().st_ttm_blockdiag(_dev(Bp, "Bp"), nblocks, bs, K, _dev(U, "U"), R, _dev(out, "out"),
                                   ws.data_ptr(), ws.numel() * ws.element_size(), flags, _stream()),
            "st_ttm_blockdiag")

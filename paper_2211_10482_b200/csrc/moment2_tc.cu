@@ -245,19 +245,26 @@ moment2_tc_reduce_kernel(const float *__restrict__ partials, float *__restrict__
 // the B operand); on diagonal tiles the two coincide and are loaded once.  The leader block
 // issues one MMA of M = 256, N = 256 for the pair; each block keeps the accumulator of its 128
 // rows in its own tensor memory.  Per MMA cycle a block now fetches a third less from L2 than in
-// the one-block kernel and has six stages in flight, which is what that kernel was short of
-// (its tensor pipe idled ~30% of the time waiting for operands).
+// the one-block kernel (whose tensor pipe idled ~30% of the time waiting for operands).  Four
+// stages of 64 samples are the measured optimum: with 6 or 7 stages the blocks of a sample range
+// drift apart, share less of X in L2 and the kernel gets 5-12% slower; with 3 it starves.
 namespace m2tc2 {
 constexpr int BM = 256, BN = 256;               // tile of the pair
 constexpr int HALF = 128;                       // rows / B columns staged per block
-constexpr int KROWS = m2tc::KROWS, BOXC = m2tc::BOXC, BOX_BYTES = m2tc::BOX_BYTES;
+#ifndef ST_M2PAIR_KROWS
+#define ST_M2PAIR_KROWS 64
+#endif
+constexpr int KROWS = ST_M2PAIR_KROWS, BOXC = m2tc::BOXC, BOX_BYTES = BOXC * KROWS * 2;
 constexpr int NBOX = HALF / BOXC;               // 2 boxes per operand per block
 constexpr int STAGE_BYTES = 2 * NBOX * BOX_BYTES;   // 32 KiB
-constexpr int STAGES = 6;
+#ifndef ST_M2PAIR_STAGES
+#define ST_M2PAIR_STAGES 4
+#endif
+constexpr int STAGES = ST_M2PAIR_STAGES;
 constexpr int THREADS = 192;
 constexpr int MAX_TILES = 160;
 constexpr uint32_t TMEM_COLS = 512;
-constexpr int FLUSH_CHUNKS = 64;
+constexpr int FLUSH_CHUNKS = 4096 / KROWS;        // 4096 samples (256 MMAs) per accumulator phase
 constexpr size_t SMEM_BYTES = (size_t)STAGES * STAGE_BYTES + 1024 + 256;
 
 struct TileTable {
@@ -566,7 +573,7 @@ st_status moment2_bf16_tc(const void *X, int64_t N, int64_t d, int64_t ldx, floa
         if (!aligned256(ws)) return ST_ERR_ALIGN;
         CUtensorMap tm2;
         if (!tc::make_tmap_2d(&tm2, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, X, (uint64_t)N, (uint64_t)d, (uint64_t)ldx * 2,
-                              BOXC, KROWS))
+                              m2tc2::BOXC, m2tc2::KROWS))
             return ST_ERR_CUDA;
         float *part2 = (float *)((unsigned char *)ws + kWsHeaderBytes);
         if (cudaFuncSetAttribute(moment2_tc_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,

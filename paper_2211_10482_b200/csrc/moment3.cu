@@ -201,12 +201,12 @@ sum_slices_kernel(const float *__restrict__ partials, float *__restrict__ out, i
     const int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (e >= elems) return;
     float s = 0.f;
-    for (int k0 = 0; k0 < slices; k0 += 8) {
-        float v[8];                       // eight loads in flight before the first add
+    for (int k0 = 0; k0 < slices; k0 += 40) {
+        float v[40];                      // forty loads in flight before the first add
 #pragma unroll
-        for (int u = 0; u < 8; ++u) v[u] = (k0 + u < slices) ? __ldcg(&partials[(size_t)(k0 + u) * elems + e]) : 0.f;
+        for (int u = 0; u < 40; ++u) v[u] = (k0 + u < slices) ? __ldcg(&partials[(size_t)(k0 + u) * elems + e]) : 0.f;
 #pragma unroll
-        for (int u = 0; u < 8; ++u) s += v[u];
+        for (int u = 0; u < 40; ++u) s += v[u];
     }
     out[e] = s;
 }
@@ -346,8 +346,21 @@ template <int WARPS>
 static st_status moment3_launch(const float *X, int64_t N, int64_t d, int64_t ldx, float *out, void *ws,
                                 size_t ws_bytes, unsigned flags, cudaStream_t stream)
 {
-    M3Table<WARPS> local;   // rebuilt on every call: a few microseconds of host work
-    if (!build_table<WARPS>((int)d, (flags & ST_FLAG_DENSE_CONTROL) != 0, local)) return ST_ERR_UNSUPPORTED;
+    // the tile table depends on d only; building it costs tens of microseconds of host time during
+    // which the GPU would sit idle, so it is built once per d and kept
+    static M3Table<WARPS> cache[M3_MAX_D / 8 + 1];
+    static bool cached[M3_MAX_D / 8 + 1] = {false};
+    static std::mutex cache_lock;
+    M3Table<WARPS> local;
+    {
+        std::lock_guard<std::mutex> guard(cache_lock);
+        const int slot = (int)d / 8;
+        if (!cached[slot]) {
+            if (!build_table<WARPS>((int)d, (flags & ST_FLAG_DENSE_CONTROL) != 0, cache[slot])) return ST_ERR_UNSUPPORTED;
+            cached[slot] = true;
+        }
+        local = cache[slot];
+    }
     const M3Plan p = moment3_plan(N, d, local.groups);
     const size_t need = kWsHeaderBytes + (size_t)p.slices * p.out_elems * sizeof(float);
     if (!ws || ws_bytes < need) return ST_ERR_WORKSPACE;
@@ -370,12 +383,22 @@ static st_status moment3_launch(const float *X, int64_t N, int64_t d, int64_t ld
 
 static int moment3_groups(int64_t d, unsigned flags)
 {
-    if (flags & ST_FLAG_DENSE_CONTROL) {
-        M3Table<128> t;
-        return build_table<128>((int)d, true, t) ? t.groups : 0;
+    // groups per d, remembered: the size query must stay cheap
+    static int cache[2][M3_MAX_D / 8 + 1] = {{0}};
+    static std::mutex lock;
+    const int dense = (flags & ST_FLAG_DENSE_CONTROL) ? 1 : 0;
+    std::lock_guard<std::mutex> guard(lock);
+    int &g = cache[dense][d / 8];
+    if (g == 0) {
+        if (dense) {
+            M3Table<128> t;
+            g = build_table<128>((int)d, true, t) ? t.groups : -1;
+        } else {
+            M3Table<32> t;
+            g = build_table<32>((int)d, false, t) ? t.groups : -1;
+        }
     }
-    M3Table<32> t;
-    return build_table<32>((int)d, false, t) ? t.groups : 0;
+    return g > 0 ? g : 0;
 }
 
 size_t moment3_workspace(int64_t N, int64_t d, unsigned flags)
