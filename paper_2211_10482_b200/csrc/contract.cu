@@ -263,8 +263,7 @@ static st_status rowgemm_launch(const RgArgs &a0, cudaStream_t stream)
     const int64_t items = (int64_t)a.tiles * a.ksplit;
     const int grid = (int)(items < di.sm_count ? items : di.sm_count);
     auto run = [&](auto kernel) -> st_status {
-        if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
-            return ST_ERR_CUDA;
+        if (!ensure_dynamic_smem(kernel, smem)) return ST_ERR_CUDA;
         kernel<<<grid, RG_THREADS, smem, stream>>>(a);
         return launch_status();
     };

@@ -15,6 +15,10 @@ namespace st {
 st_status moment2_bf16_tc(const void *X, int64_t N, int64_t d, int64_t ldx, float *out, void *ws,
                           size_t ws_bytes, unsigned flags, cudaStream_t stream);
 size_t moment2_bf16_tc_workspace(int64_t N, int64_t d, unsigned flags);
+bool moment2_small_applies(int64_t N, int64_t d);
+size_t moment2_small_workspace(int64_t N, int64_t d, unsigned flags);
+st_status moment2_small(const float *X, int64_t N, int64_t d, int64_t ldx, float *out, void *ws, size_t ws_bytes,
+                        unsigned flags, cudaStream_t stream);
 
 constexpr int M2_T = 64;    // output tile edge
 constexpr int M2_KC = 64;   // sample rows staged per step
@@ -176,6 +180,8 @@ static st_status moment2_f32(const float *X, int64_t N, int64_t d, int64_t ldx, 
                              size_t ws_bytes, unsigned flags, cudaStream_t stream)
 {
     if (d > 32768) return ST_ERR_UNSUPPORTED;
+    // few features, many samples: the register-tile kernel of moment2_small.cu
+    if (moment2_small_applies(N, d) && ldx % 4 == 0) return moment2_small(X, N, d, ldx, out, ws, ws_bytes, flags, stream);
     const M2Plan p = moment2_plan(N, d, flags);
     const size_t need = kWsHeaderBytes + p.ticket_bytes + p.partial_bytes;
     if (!ws || ws_bytes < need) return ST_ERR_WORKSPACE;
@@ -201,7 +207,12 @@ size_t moment2_workspace(int64_t N, int64_t d, int xdt, unsigned flags)
     if (xdt == ST_BF16) return moment2_bf16_tc_workspace(N, d, flags);
     if (xdt != ST_F32 || d > 32768) return 0;
     const M2Plan p = moment2_plan(N, d, flags);
-    return kWsHeaderBytes + p.ticket_bytes + p.partial_bytes;
+    size_t need = kWsHeaderBytes + p.ticket_bytes + p.partial_bytes;
+    if (moment2_small_applies(N, d)) {     // which kernel runs depends on ldx: size for either
+        const size_t small = moment2_small_workspace(N, d, flags);
+        if (small > need) need = small;
+    }
+    return need;
 }
 
 }  // namespace st

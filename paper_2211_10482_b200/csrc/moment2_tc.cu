@@ -576,9 +576,7 @@ st_status moment2_bf16_tc(const void *X, int64_t N, int64_t d, int64_t ldx, floa
                               m2tc2::BOXC, m2tc2::KROWS))
             return ST_ERR_CUDA;
         float *part2 = (float *)((unsigned char *)ws + kWsHeaderBytes);
-        if (cudaFuncSetAttribute(moment2_tc_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 (int)m2tc2::SMEM_BYTES) != cudaSuccess)
-            return ST_ERR_CUDA;
+        if (!ensure_dynamic_smem(moment2_tc_pair_kernel, m2tc2::SMEM_BYTES)) return ST_ERR_CUDA;
         cudaLaunchConfig_t cfg = {};
         cfg.gridDim = dim3(2 * q.tab.ntiles * q.tab.nsplit);
         cfg.blockDim = dim3(m2tc2::THREADS);
@@ -609,9 +607,7 @@ st_status moment2_bf16_tc(const void *X, int64_t N, int64_t d, int64_t ldx, floa
                           BOXC, KROWS))
         return ST_ERR_CUDA;
     float *partials = (float *)((unsigned char *)ws + kWsHeaderBytes);
-    if (cudaFuncSetAttribute(moment2_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES) !=
-        cudaSuccess)
-        return ST_ERR_CUDA;
+    if (!ensure_dynamic_smem(moment2_tc_kernel, SMEM_BYTES)) return ST_ERR_CUDA;
     moment2_tc_kernel<<<p.tab.nblocks, THREADS, SMEM_BYTES, stream>>>(tmap, partials, (unsigned *)ws, p.chunks_total,
                                                                       p.tab);
     if (cudaGetLastError() != cudaSuccess) return ST_ERR_CUDA;

@@ -367,11 +367,7 @@ static st_status moment3_launch(const float *X, int64_t N, int64_t d, int64_t ld
     if (!aligned256(ws)) return ST_ERR_ALIGN;
     float *partials = (float *)((unsigned char *)ws + kWsHeaderBytes);
     const size_t smem = (size_t)M3_BUFFERS * M3_STAGE_ROWS * d * sizeof(float);
-    if (smem > 48 * 1024) {
-        if (cudaFuncSetAttribute(moment3_kernel<WARPS>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
-            cudaSuccess)
-            return ST_ERR_CUDA;
-    }
+    if (!ensure_dynamic_smem(moment3_kernel<WARPS>, smem)) return ST_ERR_CUDA;
     dim3 grid(p.groups, p.slices);
     moment3_kernel<WARPS><<<grid, M3_THREADS, smem, stream>>>(X, N, (int)d, ldx, partials, p.rows_per_slice,
                                                               (int)p.out_elems, local);

@@ -3,6 +3,9 @@
 #include <cuda_runtime.h>
 #include <cstdint>
 #include <cstddef>
+#include <map>
+#include <mutex>
+#include <utility>
 #include "structtensor.h"
 
 namespace st {
@@ -49,6 +52,27 @@ inline int sm_count_or_default()
 {
     DeviceInfo di = device_info();
     return di.ok ? di.sm_count : 148;
+}
+
+// Raises a kernel's dynamic shared-memory limit once per (kernel, device): the runtime call costs
+// tens of microseconds, during which the GPU would idle if it were repeated on every launch.
+template <typename Kernel>
+inline bool ensure_dynamic_smem(Kernel kernel, size_t bytes)
+{
+    if (bytes <= 48 * 1024) return true;
+    static std::mutex lock;
+    static std::map<std::pair<const void *, int>, size_t> done;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return false;
+    std::lock_guard<std::mutex> guard(lock);
+    size_t &have = done[std::make_pair((const void *)kernel, dev)];
+    if (have >= bytes) return true;
+    if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return false;
+    }
+    have = bytes;
+    return true;
 }
 
 inline st_status launch_status()

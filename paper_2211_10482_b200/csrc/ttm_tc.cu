@@ -331,8 +331,7 @@ static st_status tc_rows_launch(const float *Bp, int64_t rows, int64_t K, const 
     a.U = U; a.C = C; a.I = (int)I; a.mode = mode; a.out = Ap; a.status = (unsigned *)ws; a.rows = rows; a.K = (int)K; a.R = (int)R;
     a.kchunks = p.kchunks; a.stages = p.stages; a.tmem_cols = p.tmem_cols;
     a.ntiles = (int)((rows + BM - 1) / BM);
-    if (cudaFuncSetAttribute(ttm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)p.smem) != cudaSuccess)
-        return ST_ERR_CUDA;
+    if (!ensure_dynamic_smem(ttm_tc_kernel, p.smem)) return ST_ERR_CUDA;
     const int grid = a.ntiles < di.sm_count ? a.ntiles : di.sm_count;
     ttm_tc_kernel<<<grid, THREADS, p.smem, stream>>>(tmap, a);
     return launch_status();
