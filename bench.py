@@ -38,10 +38,10 @@ FP32_PEAK_TFLOPS = 2 * 148 * 128 * 1.965e9 / 1e12
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 # DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) per launch from the ncu captures summarised
-# under profiles/.  moment2_tc_pair_kernel was captured at [131072, 1024] (329.9 MB) and scaled by the
+# under profiles/.  moment2_tc_pair_kernel was captured at [131072, 1024] (314.7 MB) and scaled by the
 # sample count to [1048576, 1024]; the TF32 kernels were captured at the benchmark configuration.
 # An entry is dropped (null) when its kernel changes after the capture.
-NCU_TRAFFIC_BYTES = {"sym_moment2_large": 8 * 329.9e6, "ttm_blockdiag": 312.4e6, "mttkrp_tri": 273.9e6}
+NCU_TRAFFIC_BYTES = {"sym_moment2_large": 8 * 314.7e6, "ttm_blockdiag": 313.5e6, "mttkrp_tri": 273.3e6}
 
 
 def load_peaks():
