@@ -3,24 +3,25 @@
 //
 // out[p(i,j)] = sum_n X[n,i] X[n,j], 0 <= i <= j < d  (Section 3, M1; Section 5.5, y_U = i <= j).
 //
-// The upper triangle is cut into 8x8 register tiles (ib <= jb): 36 of the 64 tiles for d = 64; tiles
-// below the diagonal do not exist here.  The rows of a shared-memory stage are dealt to RG "row
-// groups"; one thread owns (tile, row group) and keeps the 64 sums of its tile over its rows in
-// registers, so a block of tiles*RG threads needs 4 shared-memory loads per 64 FMAs.  Blocks own
-// slices of the samples (one block per SM), stream them through a 3-buffer cp.async pipeline in
-// the same bank-conflict-free "split halves" row layout as the third-moment kernel, add their row
-// groups in shared memory and write one partial per block; a second kernel adds the partials in
-// fixed order.  Diagonal tiles compute all 64 products (the 28 below the diagonal are dropped):
-// 36*64 = 2304 FMAs issued per sample for 2080 useful.
+// The d columns are dealt to d/8 "column blocks"; block b owns columns 4b..4b+3 of the first half
+// of a row and the same four of the second half (two 16-byte chunks, so that the threads of a warp
+// read one contiguous 128-byte segment per load and a row can stay in its natural layout).  Every
+// unordered pair of columns lies in exactly one unordered pair of blocks, so the 8x8 register tiles
+// (ib <= jb) cover the unique set once: 36 tiles for d = 64, not 64.  The rows of a shared-memory
+// stage are dealt to RG "row groups"; one thread owns (tile, row group) and keeps the 64 sums of
+// its tile over its rows in registers: 4 shared-memory loads per 64 FMAs.  Blocks own slices of the
+// samples (one block per SM), stream them through a 3-buffer cp.async pipeline, add their row
+// groups in shared memory in a fixed order and write one partial per block; a second kernel adds
+// the partials in slice order.  Diagonal tiles compute all 64 products (the 28 below the diagonal
+// are dropped): 36*64 = 2304 FMAs issued per sample for 2080 useful.
 #include "st_common.cuh"
 #include "st_index.cuh"
 
 namespace st {
 
 constexpr int M2S_MAX_THREADS = 512;
-constexpr int M2S_ROWS_PER_GROUP = 8;      // rows of a stage handled by one row group
 constexpr int M2S_BUFFERS = 3;
-constexpr int M2S_RED_STRIDE = 65;         // floats per tile in the block-level sum array
+constexpr int M2S_STAGE_BYTES = 57344;     // upper bound of one stage (3 stages + slack fit in 227 KB)
 
 __device__ __forceinline__ void m2s_cp_async16(void *smem, const void *gmem, bool valid)
 {
@@ -31,30 +32,37 @@ __device__ __forceinline__ void m2s_cp_async16(void *smem, const void *gmem, boo
 
 struct M2SmallArgs {
     const float *X;
-    float *partials;      // [slices][ntiles*64]
+    float *partials;      // [slices][64][ntiles]
     int64_t N, ldx, rows_per_slice;
-    int d, nbk, ntiles, rg, dense;
+    int d, nbk, ntiles, rg, rpg, dense;
 };
+
+// column of element e (0..7) of column block b
+__device__ __forceinline__ int m2s_column(int b, int e, int half) { return (e < 4) ? 4 * b + e : half + 4 * b + (e - 4); }
+
+__device__ __forceinline__ void m2s_tile(int tile, int nbk, int dense, int &ib, int &jb)
+{
+    if (dense) {
+        ib = tile / nbk;
+        jb = tile - ib * nbk;
+    } else {
+        int64_t x, y;
+        tri_decode(nbk, tile, x, y);
+        ib = (int)x;
+        jb = (int)y;
+    }
+}
 
 __global__ void __launch_bounds__(M2S_MAX_THREADS, 1) moment2_small_kernel(const M2SmallArgs a)
 {
     extern __shared__ __align__(16) float smem[];
-    const int stage_rows = a.rg * M2S_ROWS_PER_GROUP;
+    const int stage_rows = a.rg * a.rpg;
     const int stage_floats = stage_rows * a.d;
-    float *red = smem + M2S_BUFFERS * stage_floats;          // [ntiles][M2S_RED_STRIDE] block-level sums
     const int tid = threadIdx.x, nthreads = blockDim.x;
     const int item_rg = tid / a.ntiles, tile = tid - item_rg * a.ntiles;
     const bool active = item_rg < a.rg;
     int ib, jb;
-    if (a.dense) {
-        ib = tile / a.nbk;
-        jb = tile - ib * a.nbk;
-    } else {
-        int64_t x, y;
-        tri_decode(a.nbk, tile, x, y);
-        ib = (int)x;
-        jb = (int)y;
-    }
+    m2s_tile(tile, a.nbk, a.dense, ib, jb);
     const int half = 4 * a.nbk;
     const int oi = 4 * ib, oj = 4 * jb;
 
@@ -67,17 +75,26 @@ __global__ void __launch_bounds__(M2S_MAX_THREADS, 1) moment2_small_kernel(const
     const int64_t n_begin = (int64_t)blockIdx.x * a.rows_per_slice;
     int64_t n_end = n_begin + a.rows_per_slice;
     if (n_end > a.N) n_end = a.N;
-    const int chunks_per_row = a.d / 4;
-    const int stage_chunks = stage_rows * chunks_per_row;
+
+    // 16-byte chunk c = tid + k*nthreads of a stage is chunk g of row r; (r, g) advance by a fixed
+    // step per k, so the copy loop needs no division
+    const int cpr = a.d / 4;
+    const int r0 = tid / cpr, g0 = tid - r0 * cpr;
+    const int dr = nthreads / cpr, dg = nthreads - dr * cpr;
 
     auto load_stage = [&](int buf, int64_t n0) {
         float *dst = smem + buf * stage_floats;
-        for (int c = tid; c < stage_chunks; c += nthreads) {
-            const int r = c / chunks_per_row, g = c - r * chunks_per_row;
+        int r = r0, g = g0;
+        while (r < stage_rows) {
             const int64_t n = n0 + r;
-            const int sc = (g & 1) ? a.nbk + (g >> 1) : (g >> 1);    // split-half position of chunk g
             const bool ok = n < n_end;
-            m2s_cp_async16(dst + r * a.d + 4 * sc, a.X + (ok ? n : n_begin) * a.ldx + 4 * g, ok);
+            m2s_cp_async16(dst + r * a.d + 4 * g, a.X + (ok ? n : n_begin) * a.ldx + 4 * g, ok);
+            g += dg;
+            r += dr;
+            if (g >= cpr) {
+                g -= cpr;
+                ++r;
+            }
         }
         asm volatile("cp.async.commit_group;\n" ::);
     };
@@ -87,6 +104,7 @@ __global__ void __launch_bounds__(M2S_MAX_THREADS, 1) moment2_small_kernel(const
         if (s < nstages) load_stage(s, n_begin + (int64_t)s * stage_rows);
         else asm volatile("cp.async.commit_group;\n" ::);
     }
+    const int step = a.rg * a.d;
     for (int64_t s = 0; s < nstages; ++s) {
         asm volatile("cp.async.wait_group %0;\n" ::"n"(M2S_BUFFERS - 2));
         __syncthreads();
@@ -95,11 +113,9 @@ __global__ void __launch_bounds__(M2S_MAX_THREADS, 1) moment2_small_kernel(const
         else
             asm volatile("cp.async.commit_group;\n" ::);
         if (active) {
-            const float *xs = smem + (int)(s % M2S_BUFFERS) * stage_floats + item_rg * a.d;
-            const int step = a.rg * a.d;
+            const float *row = smem + (int)(s % M2S_BUFFERS) * stage_floats + item_rg * a.d;
 #pragma unroll 2
-            for (int q = 0; q < M2S_ROWS_PER_GROUP; ++q) {
-                const float *row = xs + q * step;
+            for (int q = 0; q < a.rpg; ++q, row += step) {
                 const float4 i0 = *reinterpret_cast<const float4 *>(row + oi);
                 const float4 i1 = *reinterpret_cast<const float4 *>(row + oi + half);
                 const float4 j0 = *reinterpret_cast<const float4 *>(row + oj);
@@ -114,56 +130,83 @@ __global__ void __launch_bounds__(M2S_MAX_THREADS, 1) moment2_small_kernel(const
         }
     }
     asm volatile("cp.async.wait_group 0;\n" ::);
+    __syncthreads();                                   // every thread is done with the stage buffers
 
-    // add the row groups of the block one after the other (fixed order: the result is reproducible)
-    for (int g = 0; g < a.rg; ++g) {
-        if (active && item_rg == g) {
-            float *t = red + tile * M2S_RED_STRIDE;      // odd stride: lanes (tiles) hit different banks
+    // block-level sum over the row groups, in group order (reproducible): the sums go to shared
+    // memory as red[k][group][tile] (consecutive threads, consecutive words), output (k, tile) is
+    // then summed over the groups by `parts` threads, each over a fixed range, and by one thread
+    // over the parts.
+    float *red = smem;
+    const int items = a.rg * a.ntiles;
+    if (active) {
 #pragma unroll
-            for (int i = 0; i < 8; ++i)
+        for (int i = 0; i < 8; ++i)
 #pragma unroll
-                for (int j = 0; j < 8; ++j) t[i * 8 + j] = (g == 0 ? 0.f : t[i * 8 + j]) + acc[i][j];
+            for (int j = 0; j < 8; ++j) red[(i * 8 + j) * items + tid] = acc[i][j];
+    }
+    __syncthreads();
+    const int nout = 64 * a.ntiles;
+    int parts = nthreads / nout;
+    if (parts < 1) parts = 1;
+    if (parts > a.rg) parts = a.rg;
+    float *mine = a.partials + (size_t)blockIdx.x * nout;
+    if (parts == 1) {
+        for (int o = tid; o < nout; o += nthreads) {
+            const int k = o / a.ntiles, t = o - k * a.ntiles;
+            const float *p = red + k * items + t;
+            float sum = 0.f;
+            for (int g = 0; g < a.rg; ++g) sum += p[g * a.ntiles];
+            mine[o] = sum;
+        }
+    } else {
+        float *scratch = red + 64 * items;             // [parts][nout]
+        const int per = (a.rg + parts - 1) / parts;
+        if (tid < parts * nout) {
+            const int part = tid / nout, o = tid - part * nout;
+            const int k = o / a.ntiles, t = o - k * a.ntiles;
+            const float *p = red + k * items + t;
+            int g_end = (part + 1) * per;
+            if (g_end > a.rg) g_end = a.rg;
+            float sum = 0.f;
+            for (int g = part * per; g < g_end; ++g) sum += p[g * a.ntiles];
+            scratch[part * nout + o] = sum;
         }
         __syncthreads();
+        if (tid < nout) {
+            float sum = 0.f;
+            for (int part = 0; part < parts; ++part) sum += scratch[part * nout + tid];
+            mine[tid] = sum;
+        }
     }
-    float *mine = a.partials + (size_t)blockIdx.x * a.ntiles * 64;
-    for (int e = tid; e < a.ntiles * 64; e += nthreads) mine[e] = red[(e >> 6) * M2S_RED_STRIDE + (e & 63)];
 }
 
-// out[p(i,j)] = sum over the slices, in slice order, i <= j only.
+// out[p(ci,cj)] = sum over the slices, in slice order, of element (k, tile) of the partials.
 __global__ void __launch_bounds__(256)
 moment2_small_reduce_kernel(const float *__restrict__ partials, float *__restrict__ out, int d, int nbk, int ntiles,
                             int slices, int dense)
 {
-    const int e = blockIdx.x * 256 + threadIdx.x;
-    if (e >= ntiles * 64) return;
-    const int tile = e >> 6, i8 = (e >> 3) & 7, j8 = e & 7;
+    const int o = blockIdx.x * 256 + threadIdx.x;
+    if (o >= ntiles * 64) return;
+    const int k = o / ntiles, tile = o - k * ntiles;
+    const int i8 = k >> 3, j8 = k & 7;
     int ib, jb;
-    if (dense) {
-        ib = tile / nbk;
-        jb = tile - ib * nbk;
-    } else {
-        int64_t x, y;
-        tri_decode(nbk, tile, x, y);
-        ib = (int)x;
-        jb = (int)y;
-    }
-    const int gi = 8 * ib + i8, gj = 8 * jb + j8;
-    if (gi > gj) return;
+    m2s_tile(tile, nbk, dense, ib, jb);
+    if (ib > jb || (ib == jb && i8 > j8)) return;      // dense control: the other half is discarded
+    const int ci = m2s_column(ib, i8, 4 * nbk), cj = m2s_column(jb, j8, 4 * nbk);
     float s = 0.f;
     const size_t stride = (size_t)ntiles * 64;
     for (int k0 = 0; k0 < slices; k0 += 32) {
         float v[32];
 #pragma unroll
-        for (int u = 0; u < 32; ++u) v[u] = (k0 + u < slices) ? __ldcg(partials + (size_t)(k0 + u) * stride + e) : 0.f;
+        for (int u = 0; u < 32; ++u) v[u] = (k0 + u < slices) ? __ldcg(partials + (size_t)(k0 + u) * stride + o) : 0.f;
 #pragma unroll
         for (int u = 0; u < 32; ++u) s += v[u];
     }
-    out[tri_encode(d, gi, gj)] = s;
+    out[tri_encode(d, ci < cj ? ci : cj, ci < cj ? cj : ci)] = s;
 }
 
 struct M2SmallPlan {
-    int nbk, ntiles, rg, threads, slices;
+    int nbk, ntiles, rg, rpg, threads, slices;
     int64_t rows_per_slice;
     size_t smem, partial_bytes;
 };
@@ -178,17 +221,23 @@ static M2SmallPlan moment2_small_plan(int64_t N, int64_t d, unsigned flags)
     M2SmallPlan p;
     p.nbk = (int)d / 8;
     p.ntiles = (flags & ST_FLAG_DENSE_CONTROL) ? p.nbk * p.nbk : p.nbk * (p.nbk + 1) / 2;
+    const int max_stage_rows = M2S_STAGE_BYTES / (4 * (int)d);
     p.rg = M2S_MAX_THREADS / p.ntiles;
-    if (p.rg > 16) p.rg = 16;
+    if (p.rg > max_stage_rows / 8) p.rg = max_stage_rows / 8;
     if (p.rg < 1) p.rg = 1;
     p.threads = (p.ntiles * p.rg + 31) / 32 * 32;
-    const int stage_rows = p.rg * M2S_ROWS_PER_GROUP;
+    p.rpg = 8;
     int64_t slices = sm_count_or_default();
-    const int64_t max_slices = (N + stage_rows - 1) / stage_rows;
+    const int64_t max_slices = (N + p.rg * 8 - 1) / (p.rg * 8);
     if (slices > max_slices) slices = max_slices;
     p.rows_per_slice = (N + slices - 1) / slices;
     p.slices = (int)((N + p.rows_per_slice - 1) / p.rows_per_slice);
-    p.smem = ((size_t)M2S_BUFFERS * stage_rows * d + (size_t)p.ntiles * M2S_RED_STRIDE) * sizeof(float);
+    // long slices: 16 rows per thread and stage halve the number of block-wide barriers
+    if (p.rg * 16 <= max_stage_rows && p.rows_per_slice >= 4 * p.rg * 16) p.rpg = 16;
+    const size_t items = (size_t)p.rg * p.ntiles;
+    const size_t main_bytes = (size_t)M2S_BUFFERS * p.rg * p.rpg * d * sizeof(float);
+    const size_t sum_bytes = (64 * items + (size_t)M2S_MAX_THREADS) * sizeof(float);
+    p.smem = main_bytes > sum_bytes ? main_bytes : sum_bytes;
     p.partial_bytes = (size_t)p.slices * p.ntiles * 64 * sizeof(float);
     return p;
 }
@@ -208,7 +257,7 @@ st_status moment2_small(const float *X, int64_t N, int64_t d, int64_t ldx, float
     a.X = X;
     a.partials = (float *)((unsigned char *)ws + kWsHeaderBytes);
     a.N = N; a.ldx = ldx; a.rows_per_slice = p.rows_per_slice;
-    a.d = (int)d; a.nbk = p.nbk; a.ntiles = p.ntiles; a.rg = p.rg;
+    a.d = (int)d; a.nbk = p.nbk; a.ntiles = p.ntiles; a.rg = p.rg; a.rpg = p.rpg;
     a.dense = (flags & ST_FLAG_DENSE_CONTROL) ? 1 : 0;
     if (!ensure_dynamic_smem(moment2_small_kernel, p.smem)) return ST_ERR_CUDA;
     moment2_small_kernel<<<p.slices, p.threads, p.smem, stream>>>(a);
