@@ -16,6 +16,7 @@
 // are dropped): 36*64 = 2304 FMAs issued per sample for 2080 useful.
 #include "st_common.cuh"
 #include "st_index.cuh"
+#include "tc_common.cuh"
 
 namespace st {
 
@@ -23,18 +24,22 @@ constexpr int M2S_MAX_THREADS = 512;
 constexpr int M2S_BUFFERS = 3;
 constexpr int M2S_STAGE_BYTES = 57344;     // upper bound of one stage (3 stages + slack fit in 227 KB)
 
-__device__ __forceinline__ void m2s_cp_async16(void *smem, const void *gmem, bool valid)
+// bulk copy global -> shared of `bytes` (a multiple of 16, both addresses 16-byte aligned),
+// completion counted in bytes on `bar`
+__device__ __forceinline__ void m2s_bulk_load(void *dst, const void *src, uint32_t bytes, uint64_t *bar)
 {
-    const unsigned s = (unsigned)__cvta_generic_to_shared(smem);
-    const int sz = valid ? 16 : 0;
-    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;\n" ::"r"(s), "l"(gmem), "r"(sz));
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
+                     tc::smem_u32(dst)),
+                 "l"(src), "r"(bytes), "r"(tc::smem_u32(bar))
+                 : "memory");
 }
 
 struct M2SmallArgs {
     const float *X;
     float *partials;      // [slices][64][ntiles]
+    unsigned *status;     // workspace header (status and detail words)
     int64_t N, ldx, rows_per_slice;
-    int d, nbk, ntiles, rg, rpg, dense;
+    int d, nbk, ntiles, rg, rpg, dense, bar_floats;
 };
 
 // column of element e (0..7) of column block b
@@ -76,46 +81,59 @@ __global__ void __launch_bounds__(M2S_MAX_THREADS, 1) moment2_small_kernel(const
     int64_t n_end = n_begin + a.rows_per_slice;
     if (n_end > a.N) n_end = a.N;
 
-    // 16-byte chunk c = tid + k*nthreads of a stage is chunk g of row r; (r, g) advance by a fixed
-    // step per k, so the copy loop needs no division
-    const int cpr = a.d / 4;
-    const int r0 = tid / cpr, g0 = tid - r0 * cpr;
-    const int dr = nthreads / cpr, dg = nthreads - dr * cpr;
-
-    auto load_stage = [&](int buf, int64_t n0) {
-        float *dst = smem + buf * stage_floats;
-        int r = r0, g = g0;
-        while (r < stage_rows) {
-            const int64_t n = n0 + r;
-            const bool ok = n < n_end;
-            m2s_cp_async16(dst + r * a.d + 4 * g, a.X + (ok ? n : n_begin) * a.ldx + 4 * g, ok);
-            g += dg;
-            r += dr;
-            if (g >= cpr) {
-                g -= cpr;
-                ++r;
-            }
+    uint64_t *full = reinterpret_cast<uint64_t *>(smem + a.bar_floats);      // one barrier per buffer
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(full + M2S_BUFFERS);
+    if (tid == 0) {
+        for (int b = 0; b < M2S_BUFFERS; ++b) tc::mbar_init(&full[b], 1);
+        *abort_flag = 0;
+        if (blockIdx.x == 0) {      // a time-out report can only be written 2^24 failed polls later
+            a.status[kWsStatusWord] = 0;
+            a.status[kWsDetailWord] = 0;
         }
-        asm volatile("cp.async.commit_group;\n" ::);
+        tc::fence_barrier_init();
+    }
+    __syncthreads();
+
+    const int nstages = (n_end > n_begin) ? (int)((n_end - n_begin + stage_rows - 1) / stage_rows) : 0;
+    const bool contiguous = (a.ldx == a.d);
+    // the rows of a stage arrive by bulk copies issued from warp 0: one copy when the rows are
+    // contiguous in memory, one per row otherwise; rows past the end of the slice are not copied
+    // and not read
+    auto issue_stage = [&](int buf, int s) {
+        if (tid >= 32) return;
+        const int64_t n0 = n_begin + (int64_t)s * stage_rows;
+        const int rows = (n_end - n0 < stage_rows) ? (int)(n_end - n0) : stage_rows;
+        float *dst = smem + buf * stage_floats;
+        const uint32_t row_bytes = (uint32_t)a.d * 4u;
+        if (tid == 0) tc::mbar_expect_tx(&full[buf], (uint32_t)rows * row_bytes);
+        __syncwarp();
+        if (contiguous) {
+            if (tid == 0) m2s_bulk_load(dst, a.X + n0 * a.ldx, (uint32_t)rows * row_bytes, &full[buf]);
+        } else {
+            for (int r = tid; r < rows; r += 32) m2s_bulk_load(dst + r * a.d, a.X + (n0 + r) * a.ldx, row_bytes, &full[buf]);
+        }
     };
 
-    const int64_t nstages = (n_end > n_begin) ? (n_end - n_begin + stage_rows - 1) / stage_rows : 0;
-    for (int s = 0; s < M2S_BUFFERS - 1; ++s) {
-        if (s < nstages) load_stage(s, n_begin + (int64_t)s * stage_rows);
-        else asm volatile("cp.async.commit_group;\n" ::);
-    }
+    for (int s = 0; s < M2S_BUFFERS - 1 && s < nstages; ++s) issue_stage(s, s);
     const int step = a.rg * a.d;
-    for (int64_t s = 0; s < nstages; ++s) {
-        asm volatile("cp.async.wait_group %0;\n" ::"n"(M2S_BUFFERS - 2));
-        __syncthreads();
-        if (s + M2S_BUFFERS - 1 < nstages)
-            load_stage((int)((s + M2S_BUFFERS - 1) % M2S_BUFFERS), n_begin + (s + M2S_BUFFERS - 1) * stage_rows);
-        else
-            asm volatile("cp.async.commit_group;\n" ::);
+    int buf = 0;
+    uint32_t parity = 0;
+    for (int s = 0; s < nstages; ++s) {
+        // a wait that gives up raises the abort flag; every thread still walks all stages so that
+        // the block-wide barriers stay matched, and the host reads the status word afterwards
+        (void)tc::mbar_wait(&full[buf], parity, abort_flag, a.status, 1);
+        __syncthreads();                                // stage s-1 is consumed: its buffer may be refilled
+        if (s + M2S_BUFFERS - 1 < nstages) issue_stage(buf == 0 ? M2S_BUFFERS - 1 : buf - 1, s + M2S_BUFFERS - 1);
+        int qn = a.rpg;
+        if (s == nstages - 1) {                         // last stage of the slice: only the rows that exist
+            const int rows = (int)(n_end - n_begin - (int64_t)s * stage_rows);
+            qn = (rows - item_rg + a.rg - 1) / a.rg;
+            if (qn > a.rpg) qn = a.rpg;
+        }
         if (active) {
-            const float *row = smem + (int)(s % M2S_BUFFERS) * stage_floats + item_rg * a.d;
+            const float *row = smem + buf * stage_floats + item_rg * a.d;
 #pragma unroll 2
-            for (int q = 0; q < a.rpg; ++q, row += step) {
+            for (int q = 0; q < qn; ++q, row += step) {
                 const float4 i0 = *reinterpret_cast<const float4 *>(row + oi);
                 const float4 i1 = *reinterpret_cast<const float4 *>(row + oi + half);
                 const float4 j0 = *reinterpret_cast<const float4 *>(row + oj);
@@ -128,8 +146,18 @@ __global__ void __launch_bounds__(M2S_MAX_THREADS, 1) moment2_small_kernel(const
                     for (int j = 0; j < 8; ++j) acc[i][j] = fmaf(xi[i], xj[j], acc[i][j]);
             }
         }
+        if (++buf == M2S_BUFFERS) {
+            buf = 0;
+            parity ^= 1u;
+        }
     }
-    asm volatile("cp.async.wait_group 0;\n" ::);
+    if (*abort_flag && tid == 0) {
+        // after a time-out: give the copies still in flight a bounded time to land before the
+        // shared memory is reused or released
+        for (int s = (nstages > M2S_BUFFERS ? nstages - M2S_BUFFERS : 0); s < nstages; ++s)
+            for (uint32_t it = 0; it < tc::kSpinLimit; ++it)
+                if (tc::mbar_try_wait(&full[s % M2S_BUFFERS], (uint32_t)((s / M2S_BUFFERS) & 1))) break;
+    }
     __syncthreads();                                   // every thread is done with the stage buffers
 
     // block-level sum over the row groups, in group order (reproducible): the sums go to shared
@@ -208,7 +236,7 @@ moment2_small_reduce_kernel(const float *__restrict__ partials, float *__restric
 struct M2SmallPlan {
     int nbk, ntiles, rg, rpg, threads, slices;
     int64_t rows_per_slice;
-    size_t smem, partial_bytes;
+    size_t smem, data_bytes, partial_bytes;
 };
 
 bool moment2_small_applies(int64_t N, int64_t d)
@@ -237,7 +265,8 @@ static M2SmallPlan moment2_small_plan(int64_t N, int64_t d, unsigned flags)
     const size_t items = (size_t)p.rg * p.ntiles;
     const size_t main_bytes = (size_t)M2S_BUFFERS * p.rg * p.rpg * d * sizeof(float);
     const size_t sum_bytes = (64 * items + (size_t)M2S_MAX_THREADS) * sizeof(float);
-    p.smem = main_bytes > sum_bytes ? main_bytes : sum_bytes;
+    p.data_bytes = round_up(main_bytes > sum_bytes ? main_bytes : sum_bytes, 16);
+    p.smem = p.data_bytes + 64;                        // barriers and the abort flag behind the data
     p.partial_bytes = (size_t)p.slices * p.ntiles * 64 * sizeof(float);
     return p;
 }
@@ -258,6 +287,8 @@ st_status moment2_small(const float *X, int64_t N, int64_t d, int64_t ldx, float
     a.partials = (float *)((unsigned char *)ws + kWsHeaderBytes);
     a.N = N; a.ldx = ldx; a.rows_per_slice = p.rows_per_slice;
     a.d = (int)d; a.nbk = p.nbk; a.ntiles = p.ntiles; a.rg = p.rg; a.rpg = p.rpg;
+    a.status = (unsigned *)ws;
+    a.bar_floats = (int)(p.data_bytes / sizeof(float));
     a.dense = (flags & ST_FLAG_DENSE_CONTROL) ? 1 : 0;
     if (!ensure_dynamic_smem(moment2_small_kernel, p.smem)) return ST_ERR_CUDA;
     moment2_small_kernel<<<p.slices, p.threads, p.smem, stream>>>(a);
