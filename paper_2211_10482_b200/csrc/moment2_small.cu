@@ -6,21 +6,27 @@
 // The d columns are dealt to d/8 "column blocks"; block b owns columns 4b..4b+3 of the first half
 // of a row and the same four of the second half (two 16-byte chunks, so that the threads of a warp
 // read one contiguous 128-byte segment per load and a row can stay in its natural layout).  Every
-// unordered pair of columns lies in exactly one unordered pair of blocks, so the 8x8 register tiles
-// (ib <= jb) cover the unique set once: 36 tiles for d = 64, not 64.  The rows of a shared-memory
-// stage are dealt to RG "row groups"; one thread owns (tile, row group) and keeps the 64 sums of
-// its tile over its rows in registers: 4 shared-memory loads per 64 FMAs.  Blocks own slices of the
-// samples (one block per SM), stream them through a 3-buffer cp.async pipeline, add their row
-// groups in shared memory in a fixed order and write one partial per block; a second kernel adds
-// the partials in slice order.  Diagonal tiles compute all 64 products (the 28 below the diagonal
-// are dropped): 36*64 = 2304 FMAs issued per sample for 2080 useful.
+// unordered pair of columns lies in exactly one unordered pair of blocks, so the 8x8 tiles {x,y}
+// (x <= y) cover the unique set once: 36 tiles for d = 64, not 64.
+//
+// Shared memory returns 32 words per cycle to the registers of an SM, against 128 FMA lanes: an
+// 8x8 register tile (16 operand words per 64 FMAs) saturates both at once.  A work item is
+// therefore two tiles with one block in common, {s,p} and {s,q}: 24 operand words per 128 FMAs.
+// The host pairs the tiles up (an odd one out computes its tile twice and drops one copy).  The
+// rows of a shared-memory stage are dealt to RG "row groups"; one thread owns (item, row group)
+// and keeps the 128 sums of its item over its rows in registers.  Blocks own slices of the samples
+// (one block per SM), receive them in a 3-buffer pipeline of bulk copies, add their row groups in
+// shared memory in a fixed order and write one partial per block; a second kernel adds the
+// partials in slice order.  Diagonal tiles compute all 64 products (the 28 below the diagonal are
+// dropped): 36*64 = 2304 FMAs issued per sample for 2080 useful.
 #include "st_common.cuh"
 #include "st_index.cuh"
 #include "tc_common.cuh"
 
 namespace st {
 
-constexpr int M2S_MAX_THREADS = 512;
+constexpr int M2S_MAX_THREADS = 256;
+constexpr int M2S_MAX_ITEMS = 32;
 constexpr int M2S_BUFFERS = 3;
 constexpr int M2S_STAGE_BYTES = 57344;     // upper bound of one stage (3 stages + slack fit in 227 KB)
 
@@ -34,29 +40,23 @@ __device__ __forceinline__ void m2s_bulk_load(void *dst, const void *src, uint32
                  : "memory");
 }
 
+// work items: tiles {s,p} and {s,q} of column blocks; q == 255 marks an item with one tile only
+struct M2SmallItems {
+    int n;
+    unsigned char s[M2S_MAX_ITEMS], p[M2S_MAX_ITEMS], q[M2S_MAX_ITEMS];
+};
+
 struct M2SmallArgs {
     const float *X;
-    float *partials;      // [slices][64][ntiles]
+    float *partials;      // [slices][128][nitems]
     unsigned *status;     // workspace header (status and detail words)
     int64_t N, ldx, rows_per_slice;
-    int d, nbk, ntiles, rg, rpg, dense, bar_floats;
+    int d, nbk, rg, rpg, dense, bar_floats;
+    M2SmallItems items;
 };
 
 // column of element e (0..7) of column block b
 __device__ __forceinline__ int m2s_column(int b, int e, int half) { return (e < 4) ? 4 * b + e : half + 4 * b + (e - 4); }
-
-__device__ __forceinline__ void m2s_tile(int tile, int nbk, int dense, int &ib, int &jb)
-{
-    if (dense) {
-        ib = tile / nbk;
-        jb = tile - ib * nbk;
-    } else {
-        int64_t x, y;
-        tri_decode(nbk, tile, x, y);
-        ib = (int)x;
-        jb = (int)y;
-    }
-}
 
 __global__ void __launch_bounds__(M2S_MAX_THREADS, 1) moment2_small_kernel(const M2SmallArgs a)
 {
@@ -64,18 +64,19 @@ __global__ void __launch_bounds__(M2S_MAX_THREADS, 1) moment2_small_kernel(const
     const int stage_rows = a.rg * a.rpg;
     const int stage_floats = stage_rows * a.d;
     const int tid = threadIdx.x, nthreads = blockDim.x;
-    const int item_rg = tid / a.ntiles, tile = tid - item_rg * a.ntiles;
+    const int nitems = a.items.n;
+    const int item_rg = tid / nitems, item = tid - item_rg * nitems;
     const bool active = item_rg < a.rg;
-    int ib, jb;
-    m2s_tile(tile, a.nbk, a.dense, ib, jb);
     const int half = 4 * a.nbk;
-    const int oi = 4 * ib, oj = 4 * jb;
+    const int bs = a.items.s[item], bp = a.items.p[item];
+    const int bq = a.items.q[item] == 255 ? bp : a.items.q[item];
+    const int os = 4 * bs, op = 4 * bp, oq = 4 * bq;
 
-    float acc[8][8];
+    float accp[8][8], accq[8][8];                      // tiles {s,p} and {s,q}
 #pragma unroll
     for (int i = 0; i < 8; ++i)
 #pragma unroll
-        for (int j = 0; j < 8; ++j) acc[i][j] = 0.f;
+        for (int j = 0; j < 8; ++j) accp[i][j] = accq[i][j] = 0.f;
 
     const int64_t n_begin = (int64_t)blockIdx.x * a.rows_per_slice;
     int64_t n_end = n_begin + a.rows_per_slice;
@@ -134,16 +135,22 @@ __global__ void __launch_bounds__(M2S_MAX_THREADS, 1) moment2_small_kernel(const
             const float *row = smem + buf * stage_floats + item_rg * a.d;
 #pragma unroll 2
             for (int q = 0; q < qn; ++q, row += step) {
-                const float4 i0 = *reinterpret_cast<const float4 *>(row + oi);
-                const float4 i1 = *reinterpret_cast<const float4 *>(row + oi + half);
-                const float4 j0 = *reinterpret_cast<const float4 *>(row + oj);
-                const float4 j1 = *reinterpret_cast<const float4 *>(row + oj + half);
-                const float xi[8] = {i0.x, i0.y, i0.z, i0.w, i1.x, i1.y, i1.z, i1.w};
-                const float xj[8] = {j0.x, j0.y, j0.z, j0.w, j1.x, j1.y, j1.z, j1.w};
+                const float4 s0 = *reinterpret_cast<const float4 *>(row + os);
+                const float4 s1 = *reinterpret_cast<const float4 *>(row + os + half);
+                const float4 p0 = *reinterpret_cast<const float4 *>(row + op);
+                const float4 p1 = *reinterpret_cast<const float4 *>(row + op + half);
+                const float4 q0 = *reinterpret_cast<const float4 *>(row + oq);
+                const float4 q1 = *reinterpret_cast<const float4 *>(row + oq + half);
+                const float xs[8] = {s0.x, s0.y, s0.z, s0.w, s1.x, s1.y, s1.z, s1.w};
+                const float xp[8] = {p0.x, p0.y, p0.z, p0.w, p1.x, p1.y, p1.z, p1.w};
+                const float xq[8] = {q0.x, q0.y, q0.z, q0.w, q1.x, q1.y, q1.z, q1.w};
 #pragma unroll
                 for (int i = 0; i < 8; ++i)
 #pragma unroll
-                    for (int j = 0; j < 8; ++j) acc[i][j] = fmaf(xi[i], xj[j], acc[i][j]);
+                    for (int j = 0; j < 8; ++j) {
+                        accp[i][j] = fmaf(xs[i], xp[j], accp[i][j]);
+                        accq[i][j] = fmaf(xs[i], xq[j], accq[i][j]);
+                    }
             }
         }
         if (++buf == M2S_BUFFERS) {
@@ -161,42 +168,45 @@ __global__ void __launch_bounds__(M2S_MAX_THREADS, 1) moment2_small_kernel(const
     __syncthreads();                                   // every thread is done with the stage buffers
 
     // block-level sum over the row groups, in group order (reproducible): the sums go to shared
-    // memory as red[k][group][tile] (consecutive threads, consecutive words), output (k, tile) is
-    // then summed over the groups by `parts` threads, each over a fixed range, and by one thread
-    // over the parts.
+    // memory as red[k][group][item] (consecutive threads, consecutive words; k < 64 is tile {s,p},
+    // k >= 64 tile {s,q}), output (k, item) is then summed over the groups by `parts` threads, each
+    // over a fixed range, and by one thread over the parts.
     float *red = smem;
-    const int items = a.rg * a.ntiles;
+    const int cells = a.rg * nitems;
     if (active) {
 #pragma unroll
         for (int i = 0; i < 8; ++i)
 #pragma unroll
-            for (int j = 0; j < 8; ++j) red[(i * 8 + j) * items + tid] = acc[i][j];
+            for (int j = 0; j < 8; ++j) {
+                red[(i * 8 + j) * cells + tid] = accp[i][j];
+                red[(64 + i * 8 + j) * cells + tid] = accq[i][j];
+            }
     }
     __syncthreads();
-    const int nout = 64 * a.ntiles;
+    const int nout = 128 * nitems;
     int parts = nthreads / nout;
     if (parts < 1) parts = 1;
     if (parts > a.rg) parts = a.rg;
     float *mine = a.partials + (size_t)blockIdx.x * nout;
     if (parts == 1) {
         for (int o = tid; o < nout; o += nthreads) {
-            const int k = o / a.ntiles, t = o - k * a.ntiles;
-            const float *p = red + k * items + t;
+            const int k = o / nitems, t = o - k * nitems;
+            const float *p = red + k * cells + t;
             float sum = 0.f;
-            for (int g = 0; g < a.rg; ++g) sum += p[g * a.ntiles];
+            for (int g = 0; g < a.rg; ++g) sum += p[g * nitems];
             mine[o] = sum;
         }
     } else {
-        float *scratch = red + 64 * items;             // [parts][nout]
+        float *scratch = red + 128 * cells;            // [parts][nout]
         const int per = (a.rg + parts - 1) / parts;
         if (tid < parts * nout) {
             const int part = tid / nout, o = tid - part * nout;
-            const int k = o / a.ntiles, t = o - k * a.ntiles;
-            const float *p = red + k * items + t;
+            const int k = o / nitems, t = o - k * nitems;
+            const float *p = red + k * cells + t;
             int g_end = (part + 1) * per;
             if (g_end > a.rg) g_end = a.rg;
             float sum = 0.f;
-            for (int g = part * per; g < g_end; ++g) sum += p[g * a.ntiles];
+            for (int g = part * per; g < g_end; ++g) sum += p[g * nitems];
             scratch[part * nout + o] = sum;
         }
         __syncthreads();
@@ -208,21 +218,25 @@ __global__ void __launch_bounds__(M2S_MAX_THREADS, 1) moment2_small_kernel(const
     }
 }
 
-// out[p(ci,cj)] = sum over the slices, in slice order, of element (k, tile) of the partials.
+// out[p(ci,cj)] = sum over the slices, in slice order, of element (k, item) of the partials.
 __global__ void __launch_bounds__(256)
-moment2_small_reduce_kernel(const float *__restrict__ partials, float *__restrict__ out, int d, int nbk, int ntiles,
-                            int slices, int dense)
+moment2_small_reduce_kernel(const float *__restrict__ partials, float *__restrict__ out, int d, int nbk, int slices,
+                            int dense, const M2SmallItems items)
 {
     const int o = blockIdx.x * 256 + threadIdx.x;
-    if (o >= ntiles * 64) return;
-    const int k = o / ntiles, tile = o - k * ntiles;
-    const int i8 = k >> 3, j8 = k & 7;
-    int ib, jb;
-    m2s_tile(tile, nbk, dense, ib, jb);
-    if (ib > jb || (ib == jb && i8 > j8)) return;      // dense control: the other half is discarded
-    const int ci = m2s_column(ib, i8, 4 * nbk), cj = m2s_column(jb, j8, 4 * nbk);
+    const int nitems = items.n;
+    if (o >= nitems * 128) return;
+    const int k = o / nitems, item = o - k * nitems;
+    const int i8 = (k >> 3) & 7, j8 = k & 7;
+    const int x = items.s[item];
+    const int y = (k < 64) ? items.p[item] : items.q[item];
+    if (y == 255) return;                              // odd item out: no second tile
+    // a diagonal tile keeps its upper half; the dense control also computes the tiles below the
+    // diagonal and discards them here
+    if ((x == y && i8 > j8) || (dense && x > y)) return;
+    const int ci = m2s_column(x, i8, 4 * nbk), cj = m2s_column(y, j8, 4 * nbk);
     float s = 0.f;
-    const size_t stride = (size_t)ntiles * 64;
+    const size_t stride = (size_t)nitems * 128;
     for (int k0 = 0; k0 < slices; k0 += 32) {
         float v[32];
 #pragma unroll
@@ -234,9 +248,10 @@ moment2_small_reduce_kernel(const float *__restrict__ partials, float *__restric
 }
 
 struct M2SmallPlan {
-    int nbk, ntiles, rg, rpg, threads, slices;
+    int nbk, rg, rpg, threads, slices;
     int64_t rows_per_slice;
     size_t smem, data_bytes, partial_bytes;
+    M2SmallItems items;
 };
 
 bool moment2_small_applies(int64_t N, int64_t d)
@@ -244,16 +259,50 @@ bool moment2_small_applies(int64_t N, int64_t d)
     return d % 8 == 0 && d >= 8 && d <= 64 && N >= 1;
 }
 
+// Pairs the tiles up into items with a common block.  Structured: for every block y the tiles
+// {x,y}, x <= y, are paired along x with y as the common block; when their number is odd, tile
+// {0,y} is held back, and the held-back tiles are paired with block 0 in common.  Dense control:
+// all ordered tiles (x,y), paired along y with x in common.
+static M2SmallItems moment2_small_items(int nbk, bool dense)
+{
+    M2SmallItems t;
+    t.n = 0;
+    auto add = [&](int s, int p, int q) {
+        t.s[t.n] = (unsigned char)s;
+        t.p[t.n] = (unsigned char)p;
+        t.q[t.n] = (unsigned char)q;
+        ++t.n;
+    };
+    if (dense) {
+        for (int x = 0; x < nbk; ++x)
+            for (int y = 0; y < nbk; y += 2) add(x, y, y + 1 < nbk ? y + 1 : 255);
+    } else {
+        int held[8], nheld = 0;
+        for (int y = 0; y < nbk; ++y) {
+            int x = 0;
+            if ((y + 1) % 2 == 1) {
+                held[nheld++] = y;
+                x = 1;
+            }
+            for (; x + 1 <= y; x += 2) add(y, x, x + 1);
+        }
+        for (int h = 0; h < nheld; h += 2) add(0, held[h], h + 1 < nheld ? held[h + 1] : 255);
+    }
+    for (int i = t.n; i < M2S_MAX_ITEMS; ++i) t.s[i] = t.p[i] = t.q[i] = 0;
+    return t;
+}
+
 static M2SmallPlan moment2_small_plan(int64_t N, int64_t d, unsigned flags)
 {
     M2SmallPlan p;
     p.nbk = (int)d / 8;
-    p.ntiles = (flags & ST_FLAG_DENSE_CONTROL) ? p.nbk * p.nbk : p.nbk * (p.nbk + 1) / 2;
+    p.items = moment2_small_items(p.nbk, (flags & ST_FLAG_DENSE_CONTROL) != 0);
+    const int nitems = p.items.n;
     const int max_stage_rows = M2S_STAGE_BYTES / (4 * (int)d);
-    p.rg = M2S_MAX_THREADS / p.ntiles;
+    p.rg = M2S_MAX_THREADS / nitems;
     if (p.rg > max_stage_rows / 8) p.rg = max_stage_rows / 8;
     if (p.rg < 1) p.rg = 1;
-    p.threads = (p.ntiles * p.rg + 31) / 32 * 32;
+    p.threads = (nitems * p.rg + 31) / 32 * 32;
     p.rpg = 8;
     int64_t slices = sm_count_or_default();
     const int64_t max_slices = (N + p.rg * 8 - 1) / (p.rg * 8);
@@ -262,12 +311,12 @@ static M2SmallPlan moment2_small_plan(int64_t N, int64_t d, unsigned flags)
     p.slices = (int)((N + p.rows_per_slice - 1) / p.rows_per_slice);
     // long slices: 16 rows per thread and stage halve the number of block-wide barriers
     if (p.rg * 16 <= max_stage_rows && p.rows_per_slice >= 4 * p.rg * 16) p.rpg = 16;
-    const size_t items = (size_t)p.rg * p.ntiles;
+    const size_t cells = (size_t)p.rg * nitems;
     const size_t main_bytes = (size_t)M2S_BUFFERS * p.rg * p.rpg * d * sizeof(float);
-    const size_t sum_bytes = (64 * items + (size_t)M2S_MAX_THREADS) * sizeof(float);
+    const size_t sum_bytes = (128 * cells + (size_t)M2S_MAX_THREADS) * sizeof(float);
     p.data_bytes = round_up(main_bytes > sum_bytes ? main_bytes : sum_bytes, 16);
     p.smem = p.data_bytes + 64;                        // barriers and the abort flag behind the data
-    p.partial_bytes = (size_t)p.slices * p.ntiles * 64 * sizeof(float);
+    p.partial_bytes = (size_t)p.slices * nitems * 128 * sizeof(float);
     return p;
 }
 
@@ -286,16 +335,17 @@ st_status moment2_small(const float *X, int64_t N, int64_t d, int64_t ldx, float
     a.X = X;
     a.partials = (float *)((unsigned char *)ws + kWsHeaderBytes);
     a.N = N; a.ldx = ldx; a.rows_per_slice = p.rows_per_slice;
-    a.d = (int)d; a.nbk = p.nbk; a.ntiles = p.ntiles; a.rg = p.rg; a.rpg = p.rpg;
+    a.d = (int)d; a.nbk = p.nbk; a.rg = p.rg; a.rpg = p.rpg;
+    a.items = p.items;
     a.status = (unsigned *)ws;
     a.bar_floats = (int)(p.data_bytes / sizeof(float));
     a.dense = (flags & ST_FLAG_DENSE_CONTROL) ? 1 : 0;
     if (!ensure_dynamic_smem(moment2_small_kernel, p.smem)) return ST_ERR_CUDA;
     moment2_small_kernel<<<p.slices, p.threads, p.smem, stream>>>(a);
     if (cudaGetLastError() != cudaSuccess) return ST_ERR_CUDA;
-    const int n = p.ntiles * 64;
-    moment2_small_reduce_kernel<<<(n + 255) / 256, 256, 0, stream>>>(a.partials, out, (int)d, p.nbk, p.ntiles, p.slices,
-                                                                     a.dense);
+    const int n = p.items.n * 128;
+    moment2_small_reduce_kernel<<<(n + 255) / 256, 256, 0, stream>>>(a.partials, out, (int)d, p.nbk, p.slices, a.dense,
+                                                                     p.items);
     return launch_status();
 }
 
