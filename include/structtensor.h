@@ -70,7 +70,8 @@ typedef enum { ST_OP_SYM_MOMENT2 = 0, ST_OP_SYM_MOMENT3 = 1, ST_OP_MTTKRP_TRI = 
 /* flags (bit mask) */
 #define ST_FLAG_DENSE_CONTROL 1u /* run the same kernel over the dense, unstructured iteration
                                     space (a control for measurements; see each call) */
-#define ST_FLAG_TC_TF32       2u /* st_ttm_blockdiag, st_mttkrp_tri: tensor cores, operands read as TF32 */
+#define ST_FLAG_TC_TF32       2u /* st_ttm_blockdiag, st_mttkrp_tri, st_sym_moment3: tensor cores, operands read as TF32 */
+#define ST_FLAG_TC_BF16       4u /* st_sym_moment3: tensor cores, operands rounded to bf16 */
 
 typedef struct {
     int32_t kind;      /* st_kind */
@@ -108,7 +109,7 @@ st_status st_unpack(const st_layout *layout, st_dtype dtype, const void *packed,
 
 /* Scratch bytes needed by one compute call.  Arguments by op:
  *   ST_OP_SYM_MOMENT2   a=N, b=d, c=st_dtype of X, e unused
- *   ST_OP_SYM_MOMENT3   a=N, b=d
+ *   ST_OP_SYM_MOMENT3   a=N, b=d (flags select the kernel: they change the size)
  *   ST_OP_MTTKRP_TRI    a=I, b=K, c=R
  *   ST_OP_TTM_BLOCKDIAG a=nblocks, b=bs, c=K, e=R
  * Returns 0 for an invalid request (the call itself reports the error).  The current
@@ -133,7 +134,14 @@ st_status st_sym_moment2(const void *X, st_dtype xdt, int64_t N, int64_t d, int6
  * X: fp32 [N, ldx], ldx >= d, ldx % 4 == 0.  out_packed: d(d+1)(d+2)/6 floats in ST_TET
  * order.  Supported: d % 8 == 0, 8 <= d <= 64.
  * ST_FLAG_DENSE_CONTROL: all d*d*d products are computed and the results outside the
- * unique set discarded; the output is the same. */
+ * unique set discarded; the output is the same.
+ * ST_FLAG_TC_TF32 / ST_FLAG_TC_BF16 (one of them, not with the dense control) select the
+ * tensor-core path: with the pair product hoisted out of the k loop (Section 5.5, code
+ * motion) the sum is the contraction sum_n P[n,(i,j)] X[n,k] with P = X[n,i] X[n,j]; the
+ * kernel makes P on the fly as the left operand of a GEMM over the samples and never issues
+ * the tiles with k < j.  Any 1 <= d <= 64 and any ldx >= d.  TF32: x and the products
+ * rounded to TF32; bf16: x_k and the fp32 products rounded to bf16; fp32 accumulation.
+ * Tolerance 5e-3 of sum |terms| (bf16: for N >= 1000; 2^-7 for any N). */
 st_status st_sym_moment3(const float *X, int64_t N, int64_t d, int64_t ldx,
                          float *out_packed, void *ws, size_t ws_bytes, unsigned flags,
                          void *stream);

@@ -195,20 +195,44 @@ moment3_kernel(const float *__restrict__ X, int64_t N, int d, int64_t ldx, float
     }
 }
 
-__global__ void __launch_bounds__(256)
+// out[e] = sum over slices of partials[slice][e], in a fixed order.  A block covers 32 consecutive
+// elements; warp w adds the slices w, w+8, w+16, ... (all loads of a batch in flight before the first
+// add), then the eight partial sums are added through shared memory.
+constexpr int SUM_GROUPS = 8;
+__global__ void __launch_bounds__(32 * SUM_GROUPS)
 sum_slices_kernel(const float *__restrict__ partials, float *__restrict__ out, int64_t elems, int slices)
 {
-    const int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-    if (e >= elems) return;
+    __shared__ float part[SUM_GROUPS][32];
+    const int lane = threadIdx.x & 31, g = threadIdx.x >> 5;
+    const int64_t e = (int64_t)blockIdx.x * 32 + lane;
     float s = 0.f;
-    for (int k0 = 0; k0 < slices; k0 += 40) {
-        float v[40];                      // forty loads in flight before the first add
+    if (e < elems) {
+        constexpr int BATCH = 12;
+        for (int k0 = g; k0 < slices; k0 += BATCH * SUM_GROUPS) {
+            float v[BATCH];
 #pragma unroll
-        for (int u = 0; u < 40; ++u) v[u] = (k0 + u < slices) ? __ldcg(&partials[(size_t)(k0 + u) * elems + e]) : 0.f;
+            for (int u = 0; u < BATCH; ++u) {
+                const int k = k0 + u * SUM_GROUPS;
+                v[u] = k < slices ? __ldcg(&partials[(size_t)k * elems + e]) : 0.f;
+            }
 #pragma unroll
-        for (int u = 0; u < 40; ++u) s += v[u];
+            for (int u = 0; u < BATCH; ++u) s += v[u];
+        }
     }
-    out[e] = s;
+    part[g][lane] = s;
+    __syncthreads();
+    if (g == 0 && e < elems) {
+        float t = part[0][lane];
+#pragma unroll
+        for (int w = 1; w < SUM_GROUPS; ++w) t += part[w][lane];
+        out[e] = t;
+    }
+}
+
+st_status sum_slices_launch(const float *partials, float *out, int64_t elems, int slices, cudaStream_t stream)
+{
+    sum_slices_kernel<<<(unsigned)((elems + 31) / 32), 32 * SUM_GROUPS, 0, stream>>>(partials, out, elems, slices);
+    return launch_status();
 }
 
 // ---- host side: tile table ------------------------------------------------------------
@@ -372,9 +396,7 @@ static st_status moment3_launch(const float *X, int64_t N, int64_t d, int64_t ld
     moment3_kernel<WARPS><<<grid, M3_THREADS, smem, stream>>>(X, N, (int)d, ldx, partials, p.rows_per_slice,
                                                               (int)p.out_elems, local);
     if (cudaGetLastError() != cudaSuccess) return ST_ERR_CUDA;
-    const int64_t e = p.out_elems;
-    sum_slices_kernel<<<(unsigned)((e + 255) / 256), 256, 0, stream>>>(partials, out, e, p.slices);
-    return launch_status();
+    return sum_slices_launch(partials, out, p.out_elems, p.slices, stream);
 }
 
 static int moment3_groups(int64_t d, unsigned flags)
@@ -397,8 +419,14 @@ static int moment3_groups(int64_t d, unsigned flags)
     return g > 0 ? g : 0;
 }
 
+size_t moment3_tc_workspace(int64_t N, int64_t d, bool bf16);
+st_status moment3_tc(const float *X, int64_t N, int64_t d, int64_t ldx, float *out, void *ws, size_t ws_bytes,
+                     bool bf16, cudaStream_t stream);
+
 size_t moment3_workspace(int64_t N, int64_t d, unsigned flags)
 {
+    if (flags & (ST_FLAG_TC_TF32 | ST_FLAG_TC_BF16))
+        return (flags & ST_FLAG_DENSE_CONTROL) ? 0 : moment3_tc_workspace(N, d, (flags & ST_FLAG_TC_BF16) != 0);
     if (N <= 0 || d < 8 || d > M3_MAX_D || d % 8) return 0;
     const int groups = moment3_groups(d, flags);
     if (groups == 0) return 0;
@@ -413,7 +441,14 @@ extern "C" st_status st_sym_moment3(const float *X, int64_t N, int64_t d, int64_
 {
     if (!X || !out_packed) return ST_ERR_NULL;
     if (N <= 0 || d <= 0 || ldx < d) return ST_ERR_SHAPE;
-    if (flags & ~(ST_FLAG_DENSE_CONTROL)) return ST_ERR_UNSUPPORTED;
+    if (flags & ~(ST_FLAG_DENSE_CONTROL | ST_FLAG_TC_TF32 | ST_FLAG_TC_BF16)) return ST_ERR_UNSUPPORTED;
+    if (flags & (ST_FLAG_TC_TF32 | ST_FLAG_TC_BF16)) {
+        if ((flags & ST_FLAG_DENSE_CONTROL) || d > st::M3_MAX_D) return ST_ERR_UNSUPPORTED;
+        if ((flags & ST_FLAG_TC_TF32) && (flags & ST_FLAG_TC_BF16)) return ST_ERR_UNSUPPORTED;
+        if (!st::aligned16(X) || !st::aligned16(out_packed)) return ST_ERR_ALIGN;
+        return st::moment3_tc(X, N, d, ldx, out_packed, ws, ws_bytes, (flags & ST_FLAG_TC_BF16) != 0,
+                              (cudaStream_t)stream);
+    }
     if (d < 8 || d > st::M3_MAX_D || d % 8) return ST_ERR_UNSUPPORTED;
     if (!st::aligned16(X) || !st::aligned16(out_packed) || ldx % 4) return ST_ERR_ALIGN;
     if (flags & ST_FLAG_DENSE_CONTROL)

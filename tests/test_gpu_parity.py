@@ -228,6 +228,98 @@ def test_moment3_config(st):
     assert abs(lhs - rhs) <= TOL_F32 * scale
 
 
+# tensor-core third moment: pair products made on the fly as the left operand of a tcgen05 GEMM over
+# the samples.  TF32: x and x_i*x_j rounded to 10 mantissa bits (three roundings of <= 2^-11 per term).
+# bf16: x_k and the fp32 product x_i*x_j rounded to bf16 (two roundings of <= 2^-8 per term, so the
+# stated 5e-3 is asserted where rounding errors average out, N >= 1000; 2^-7 holds for any N).
+TOL_TC = 5e-3
+
+
+def _tc_flag(st, kind):
+    return st.ST_FLAG_TC_TF32 if kind == "tf32" else st.ST_FLAG_TC_BF16
+
+
+@pytest.mark.parametrize("d", [1, 2, 5, 8, 16, 17, 33, 40, 63, 64])
+@pytest.mark.parametrize("N", [1, 31, 32, 33, 65, 1000])
+def test_moment3_tf32_tensor_core_small(st, N, d):
+    X = workloads.draw((N, d), "normal", 300 + N + d)
+    T, S = oracle.moment3(X)
+    got = st.st_sym_moment3(dev(X), flags=st.ST_FLAG_TC_TF32)
+    assert got.numel() == workloads.tet(d)
+    assert oracle.rel_err(expand3(st, got, d), T, S) <= TOL_TC, (N, d)
+
+
+@pytest.mark.parametrize("N,d", [(1, 5), (63, 64), (64, 16), (129, 40), (1000, 64), (4000, 33), (20000, 64)])
+def test_moment3_bf16_tensor_core_small(st, N, d):
+    X = workloads.draw((N, d), "normal", 400 + N + d)
+    T, S = oracle.moment3(X)
+    got = st.st_sym_moment3(dev(X), flags=st.ST_FLAG_TC_BF16)
+    assert oracle.rel_err(expand3(st, got, d), T, S) <= (TOL_TC if N >= 1000 else 2.0 ** -7), (N, d)
+
+
+@pytest.mark.parametrize("kind", ["tf32", "bf16"])
+def test_moment3_tensor_core_many_slices_of_few_tiles(st, kind):
+    # small d (one or two tiles per block) with many sample slices per block: every ring of the kernel
+    # wraps many times while few producer warps are at work
+    for N, d in ((300000, 8), (200000, 16), (150000, 24)):
+        X = workloads.draw((N, d), "uniform", 500 + d)
+        got = st.st_sym_moment3(dev(X), flags=_tc_flag(st, kind)).cpu().numpy()
+        idx = [(i, j, k) for i in range(d) for j in range(i, d) for k in range(j, d)]
+        ii, jj, kk = (np.array(v) for v in zip(*idx))
+        T, S = oracle.moment3_at(X, ii, jj, kk)
+        assert oracle.rel_err(got, T, S) <= TOL_TC, (N, d)
+
+
+@pytest.mark.parametrize("kind", ["tf32", "bf16"])
+def test_moment3_tensor_core_all_ones_strided_rows_and_repeat(st, kind):
+    flag = _tc_flag(st, kind)
+    ones = torch.ones((1234, 64), dtype=torch.float32, device="cuda")
+    assert torch.all(st.st_sym_moment3(ones, flags=flag) == 1234.0)      # 1.0 and small integers are exact
+    # rows with a pitch: X is a view of a wider matrix
+    wide = dev(workloads.draw((700, 48), "normal", 77))
+    Xv = wide[:, :40]
+    got = torch.empty(workloads.tet(40), dtype=torch.float32, device="cuda")
+    ws = torch.empty(st.st_workspace_bytes(st.ST_OP_SYM_MOMENT3, 700, 40, 0, 0, flag), dtype=torch.uint8, device="cuda")
+    rc = st.lib().st_sym_moment3(Xv.data_ptr(), 700, 40, 48, got.data_ptr(), ws.data_ptr(), ws.numel(), flag,
+                                 torch.cuda.current_stream().cuda_stream)
+    assert rc == st.ST_OK and st.st_check_status(ws) == st.ST_OK
+    T, S = oracle.moment3(np.ascontiguousarray(wide.cpu().numpy()[:, :40]))
+    assert oracle.rel_err(expand3(st, got, 40), T, S) <= TOL_TC
+    # fixed-order reduction: two calls give the same bits
+    X = dev(workloads.draw((5000, 64), "normal", 78))
+    assert torch.equal(st.st_sym_moment3(X, flags=flag), st.st_sym_moment3(X, flags=flag))
+    # the two tensor-core flags exclude each other; the dense control exists for the fp32 kernel only
+    both = st.ST_FLAG_TC_TF32 | st.ST_FLAG_TC_BF16
+    assert st.lib().st_sym_moment3(X.data_ptr(), 5000, 64, 64, got.data_ptr(), ws.data_ptr(), ws.numel(), both,
+                                   torch.cuda.current_stream().cuda_stream) == st.ST_ERR_UNSUPPORTED
+    assert st.st_workspace_bytes(st.ST_OP_SYM_MOMENT3, 5000, 64, 0, 0, flag | st.ST_FLAG_DENSE_CONTROL) == 0
+
+
+@pytest.mark.parametrize("kind", ["tf32", "bf16"])
+def test_moment3_tensor_core_config(st, kind):
+    X = workloads.moment_input("moment3")
+    N, d = X.shape
+    ws = torch.empty(st.st_workspace_bytes(st.ST_OP_SYM_MOMENT3, N, d, 0, 0, _tc_flag(st, kind)), dtype=torch.uint8,
+                     device="cuda")
+    got = st.st_sym_moment3(dev(X), ws=ws, flags=_tc_flag(st, kind))
+    assert st.st_check_status(ws) == st.ST_OK
+    got = got.cpu().numpy()
+    rng = np.random.default_rng(43)
+    tri = [(i, i, i) for i in range(d)]
+    tri += [(a, b, c) for a in (0, 7, 8, 15, 16, 63) for b in (0, 15, 16, 31, 32, 48, 63) for c in (0, 16, 47, 48, 63)
+            if a <= b <= c]
+    tri += [tuple(sorted(int(v) for v in rng.integers(0, d, 3))) for _ in range(3000)]
+    ii, jj, kk = (np.array(v) for v in zip(*tri))
+    T, S = oracle.moment3_at(X, ii, jj, kk)
+    pos = np.array([oracle.locate(oracle.KIND_TET, d, *t) for t in tri])
+    assert oracle.rel_err(got[pos], T, S) <= TOL_TC
+    mult = np.array([{1: 1, 2: 3, 3: 6}[len({i, j, k})]
+                     for i in range(d) for j in range(i, d) for k in range(j, d)], np.float64)
+    Xd = X.astype(np.float64)
+    lhs, rhs = float(np.dot(mult, got.astype(np.float64))), float(np.sum(Xd.sum(axis=1) ** 3))
+    assert abs(lhs - rhs) <= TOL_TC * float(np.sum(np.abs(Xd).sum(axis=1) ** 3))
+
+
 # ------------------------------------------------------------------------------ MTTKRP / TTM
 
 @pytest.mark.parametrize("I,K,R", [(1, 4, 8), (2, 8, 16), (5, 36, 32), (16, 64, 64), (40, 100, 32), (70, 32, 8),
