@@ -32,6 +32,7 @@ struct TtmTcArgs {
     unsigned *status;
     int64_t rows;
     int K, R, kchunks, ntiles, stages;
+    int reverse;         // walk the tiles from the last one down (see tc_rows_launch)
     uint32_t tmem_cols;
 };
 
@@ -126,7 +127,8 @@ ttm_tc_kernel(const __grid_constant__ CUtensorMap tmap, const TtmTcArgs a)
             int64_t step = 0;
             bool ok = true;
             for (int t = 0; t < my_tiles && ok; ++t) {
-                const int64_t tile = blockIdx.x + (int64_t)t * gridDim.x;
+                int64_t tile = blockIdx.x + (int64_t)t * gridDim.x;
+                if (a.reverse) tile = a.ntiles - 1 - tile;
                 for (int kc = 0; kc < a.kchunks; ++kc, ++step) {
                     const int s = (int)(step % a.stages);
                     const int64_t use = step / a.stages;
@@ -174,7 +176,8 @@ ttm_tc_kernel(const __grid_constant__ CUtensorMap tmap, const TtmTcArgs a)
         const int q = warp & 3;
         for (int t = 0; t < my_tiles; ++t) {
             const int buf = t & 1;
-            const int64_t tile = blockIdx.x + (int64_t)t * gridDim.x;
+            int64_t tile = blockIdx.x + (int64_t)t * gridDim.x;
+            if (a.reverse) tile = a.ntiles - 1 - tile;
             if (!mbar_wait(&acc_full[buf], (uint32_t)((t >> 1) & 1), abort_flag, a.status, 4)) break;
             tc_fence_after();
             const int64_t row = tile * BM + q * 32 + lane;
@@ -331,6 +334,10 @@ static st_status tc_rows_launch(const float *Bp, int64_t rows, int64_t K, const 
     a.U = U; a.C = C; a.I = (int)I; a.mode = mode; a.out = Ap; a.status = (unsigned *)ws; a.rows = rows; a.K = (int)K; a.R = (int)R;
     a.kchunks = p.kchunks; a.stages = p.stages; a.tmem_cols = p.tmem_cols;
     a.ntiles = (int)((rows + BM - 1) / BM);
+    // MTTKRP usually runs right after the call that produced its packed operand (st_pack, or a kernel
+    // that writes packed output).  The end of that operand is then still in L2, so the tiles are walked
+    // from the last one down: what was written last is read first, before later fills evict it.
+    a.reverse = mode != TC_TTM ? 1 : 0;
     if (!ensure_dynamic_smem(ttm_tc_kernel, p.smem)) return ST_ERR_CUDA;
     const int grid = a.ntiles < di.sm_count ? a.ntiles : di.sm_count;
     ttm_tc_kernel<<<grid, THREADS, p.smem, stream>>>(tmap, a);
