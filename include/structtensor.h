@@ -65,13 +65,13 @@ typedef enum { ST_F32 = 0, ST_BF16 = 1, ST_F64 = 2 } st_dtype;
 typedef enum { ST_TRI_UPPER = 0, ST_TET = 1, ST_BAND = 2, ST_BLOCKDIAG = 3 } st_kind;
 typedef enum { ST_FILL_ZERO = 0, ST_FILL_SYMMETRIC = 1 } st_fill;
 typedef enum { ST_OP_SYM_MOMENT2 = 0, ST_OP_SYM_MOMENT3 = 1, ST_OP_MTTKRP_TRI = 2,
-               ST_OP_TTM_BLOCKDIAG = 3 } st_op;
+               ST_OP_TTM_BLOCKDIAG = 3, ST_OP_SYM_MOMENT4 = 4 } st_op;
 
 /* flags (bit mask) */
 #define ST_FLAG_DENSE_CONTROL 1u /* run the same kernel over the dense, unstructured iteration
                                     space (a control for measurements; see each call) */
 #define ST_FLAG_TC_TF32       2u /* st_ttm_blockdiag, st_mttkrp_tri, st_sym_moment3: tensor cores, operands read as TF32 */
-#define ST_FLAG_TC_BF16       4u /* st_sym_moment3: tensor cores, operands rounded to bf16 */
+#define ST_FLAG_TC_BF16       4u /* st_sym_moment3, st_sym_moment4: tensor cores, operands rounded to bf16 */
 
 typedef struct {
     int32_t kind;      /* st_kind */
@@ -110,6 +110,7 @@ st_status st_unpack(const st_layout *layout, st_dtype dtype, const void *packed,
 /* Scratch bytes needed by one compute call.  Arguments by op:
  *   ST_OP_SYM_MOMENT2   a=N, b=d, c=st_dtype of X, e unused
  *   ST_OP_SYM_MOMENT3   a=N, b=d (flags select the kernel: they change the size)
+ *   ST_OP_SYM_MOMENT4   a=N, b=d (flags as for the call)
  *   ST_OP_MTTKRP_TRI    a=I, b=K, c=R
  *   ST_OP_TTM_BLOCKDIAG a=nblocks, b=bs, c=K, e=R
  * Returns 0 for an invalid request (the call itself reports the error).  The current
@@ -143,6 +144,21 @@ st_status st_sym_moment2(const void *X, st_dtype xdt, int64_t N, int64_t d, int6
  * rounded to TF32; bf16: x_k and the fp32 products rounded to bf16; fp32 accumulation.
  * Tolerance 5e-3 of sum |terms| (bf16: for N >= 1000; 2^-7 for any N). */
 st_status st_sym_moment3(const float *X, int64_t N, int64_t d, int64_t ldx,
+                         float *out_packed, void *ws, size_t ws_bytes, unsigned flags,
+                         void *stream);
+
+/* Fourth moment over the unique set (Section 3, M3 = vec(f (x) f) (x) vec(f (x) f) summed over
+ * samples: the last block of the degree-2 polynomial-regression covariance; its unique elements
+ * are the 4-tuples with repetition i<=j<=k<=l, "about 23x" fewer than d^4):
+ *     out[s(i,j,k,l)] = sum_n X[n,i] X[n,j] X[n,k] X[n,l]   for 0 <= i <= j <= k <= l < d
+ * X: fp32 [N, ldx], ldx >= d, 1 <= d <= 64.  out_packed: d(d+1)(d+2)(d+3)/24 floats in the
+ * lexicographic order of the unique set (slab i holds the tetrahedron (j,k,l) of side d-i).
+ * Computed as the second moment of the pair features P[n,(i,j)] = X[n,i] X[n,j], i<=j, which
+ * the call materialises in the workspace (N * roundup(d(d+1)/2, 64) elements; query the size
+ * with ST_OP_SYM_MOMENT4), followed by a gather of the entries with j <= k.  fp32 arithmetic by
+ * default (1e-4 tolerance); ST_FLAG_TC_BF16 stores P in bf16 and runs the tensor-core triangular
+ * tile GEMM (5e-3 tolerance for N >= 1000). */
+st_status st_sym_moment4(const float *X, int64_t N, int64_t d, int64_t ldx,
                          float *out_packed, void *ws, size_t ws_bytes, unsigned flags,
                          void *stream);
 

@@ -52,6 +52,7 @@ def _load():
         lib.oracle_moment3.argtypes = [vp, i64, i64, i64, vp, vp]
         lib.oracle_moment3_at.argtypes = [vp, i64, i64, i64, vp, vp, vp, i64, vp, vp]
         lib.oracle_moment4.argtypes = [vp, i64, i64, i64, vp, vp]
+        lib.oracle_moment4_at.argtypes = [vp, i64, i64, i64, vp, vp, vp, vp, i64, vp, vp]
         lib.oracle_mttkrp.argtypes = [vp, i64, i64, i64, vp, vp, i64, i64, i64, vp, vp]
         lib.oracle_ttm.argtypes = [vp, i64, i64, vp, i64, vp, vp]
         lib.oracle_pack.argtypes = [ci, i64, i64, i64, i64, i64, i64, i64, vp, vp]
@@ -144,6 +145,20 @@ def moment4(X):
     T = np.zeros((d, d, d, d), np.float64)
     S = np.zeros((d, d, d, d), np.float64)
     _load().oracle_moment4(_ptr(X), N, d, ldx, _ptr(T), _ptr(S))
+    return T, S
+
+
+def moment4_at(X, ii, jj, kk, ll):
+    """The same sums for sampled entries (ii[e], jj[e], kk[e], ll[e]) only."""
+    X, N, d, ldx = _x2d(X)
+    idx = [np.ascontiguousarray(a, dtype=np.int64) for a in (ii, jj, kk, ll)]
+    assert idx[0].ndim == 1 and all(a.shape == idx[0].shape for a in idx)
+    for a in idx:
+        if a.size and (a.min() < 0 or a.max() >= d):
+            raise IndexError("sample index out of range")
+    T = np.zeros(idx[0].size, np.float64)
+    S = np.zeros(idx[0].size, np.float64)
+    _load().oracle_moment4_at(_ptr(X), N, d, ldx, *[_ptr(a) for a in idx], idx[0].size, _ptr(T), _ptr(S))
     return T, S
 
 

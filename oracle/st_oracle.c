@@ -159,6 +159,27 @@ void oracle_moment4(const float *X, int64_t N, int64_t d, int64_t ldx,
     }
 }
 
+/* Same definition, for a list of sampled (i,j,k,l) entries only. */
+void oracle_moment4_at(const float *X, int64_t N, int64_t d, int64_t ldx,
+                       const int64_t *ii, const int64_t *jj, const int64_t *kk, const int64_t *ll,
+                       int64_t m, double *T, double *S)
+{
+    (void)d;
+    #pragma omp parallel for schedule(static)
+    for (int64_t e = 0; e < m; ++e) {
+        double t = 0.0, s = 0.0;
+        const int64_t i = ii[e], j = jj[e], k = kk[e], l = ll[e];
+        for (int64_t n = 0; n < N; ++n) {
+            const float *x = X + n * ldx;
+            double term = (double)x[i] * (double)x[j] * (double)x[k] * (double)x[l];
+            t += term;
+            s += fabs(term);
+        }
+        T[e] = t;
+        S[e] = s;
+    }
+}
+
 /* ---------------------------------------------------------------------------
  * MTTKRP (Table 1): A(i,r) = sum_j sum_k B(i,j,k) C(j,r) D(k,r) over the FULL
  * J x K range of a dense B (zeros wherever the structure says so).  Rows

@@ -28,7 +28,7 @@ ST_TRI_UPPER, ST_TET, ST_BAND, ST_BLOCKDIAG = 0, 1, 2, 3
 # st_fill
 ST_FILL_ZERO, ST_FILL_SYMMETRIC = 0, 1
 # st_op
-ST_OP_SYM_MOMENT2, ST_OP_SYM_MOMENT3, ST_OP_MTTKRP_TRI, ST_OP_TTM_BLOCKDIAG = 0, 1, 2, 3
+ST_OP_SYM_MOMENT2, ST_OP_SYM_MOMENT3, ST_OP_MTTKRP_TRI, ST_OP_TTM_BLOCKDIAG, ST_OP_SYM_MOMENT4 = 0, 1, 2, 3, 4
 # flags
 ST_FLAG_DENSE_CONTROL = 1
 ST_FLAG_TC_TF32 = 2
@@ -36,7 +36,7 @@ ST_FLAG_TC_BF16 = 4
 
 EXPORTS = [
     "st_packed_elems", "st_dense_elems", "st_pack", "st_unpack", "st_workspace_bytes", "st_sym_moment2",
-    "st_sym_moment3", "st_sym_moment3_static", "st_mttkrp_tri", "st_ttm_blockdiag", "st_check_status", "st_status_string",
+    "st_sym_moment3", "st_sym_moment3_static", "st_sym_moment4", "st_mttkrp_tri", "st_ttm_blockdiag", "st_check_status", "st_status_string",
     "st_abi_version",
 ]
 
@@ -92,13 +92,14 @@ def lib() -> ctypes.CDLL:
         L.st_sym_moment2.argtypes = [vp, ci, i64, i64, i64, vp, vp, sz, cu, vp]
         L.st_sym_moment3.argtypes = [vp, i64, i64, i64, vp, vp, sz, cu, vp]
         L.st_sym_moment3_static.argtypes = [vp, i64, i64, i64, vp, cu, vp]
+        L.st_sym_moment4.argtypes = [vp, i64, i64, i64, vp, vp, sz, cu, vp]
         L.st_mttkrp_tri.argtypes = [vp, i64, i64, vp, vp, i64, vp, vp, sz, cu, vp]
         L.st_ttm_blockdiag.argtypes = [vp, i64, i64, i64, vp, i64, vp, vp, sz, cu, vp]
         L.st_check_status.argtypes = [vp, vp]
         L.st_status_string.argtypes = [ci]
         L.st_status_string.restype = ctypes.c_char_p
         L.st_abi_version.restype = ci
-        for name in ("st_pack", "st_unpack", "st_sym_moment2", "st_sym_moment3", "st_sym_moment3_static", "st_mttkrp_tri",
+        for name in ("st_pack", "st_unpack", "st_sym_moment2", "st_sym_moment3", "st_sym_moment3_static", "st_sym_moment4", "st_mttkrp_tri",
                      "st_ttm_blockdiag", "st_check_status"):
             getattr(L, name).restype = ci
         _lib = L
@@ -211,6 +212,20 @@ def st_sym_moment3(X: torch.Tensor, out: torch.Tensor | None = None, ws: torch.T
     ws = _workspace(lambda: st_workspace_bytes(ST_OP_SYM_MOMENT3, N, d, 0, 0, flags), X.device, ws)
     _check(lib().st_sym_moment3(_dev(X, "X"), N, d, X.stride(0), _dev(out, "out"), ws.data_ptr(),
                                 ws.numel() * ws.element_size(), flags, _stream()), "st_sym_moment3")
+    return out
+
+
+def st_sym_moment4(X: torch.Tensor, out: torch.Tensor | None = None, ws: torch.Tensor | None = None,
+                   flags: int = 0) -> torch.Tensor:
+    """Packed 4-simplex sum_n X[n,i] X[n,j] X[n,k] X[n,l], i<=j<=k<=l; X is [N, d] float32."""
+    N, d = X.shape
+    if X.dtype != torch.float32:
+        raise TypeError("X must be float32")
+    if out is None:
+        out = torch.empty(d * (d + 1) * (d + 2) * (d + 3) // 24, dtype=torch.float32, device=X.device)
+    ws = _workspace(lambda: st_workspace_bytes(ST_OP_SYM_MOMENT4, N, d, 0, 0, flags), X.device, ws)
+    _check(lib().st_sym_moment4(_dev(X, "X"), N, d, X.stride(0), _dev(out, "out"), ws.data_ptr(),
+                                ws.numel() * ws.element_size(), flags, _stream()), "st_sym_moment4")
     return out
 
 

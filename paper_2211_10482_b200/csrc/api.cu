@@ -4,6 +4,7 @@
 namespace st {
 size_t moment2_workspace(int64_t N, int64_t d, int xdt, unsigned flags);
 size_t moment3_workspace(int64_t N, int64_t d, unsigned flags);
+size_t moment4_workspace(int64_t N, int64_t d, unsigned flags);
 size_t ttm_tf32_tc_workspace(int64_t rows, int64_t K, int64_t R);
 }  // namespace st
 
@@ -14,6 +15,7 @@ size_t st_workspace_bytes(st_op op, int64_t a, int64_t b, int64_t c, int64_t e, 
     switch (op) {
     case ST_OP_SYM_MOMENT2: return st::moment2_workspace(a, b, (int)c, flags);
     case ST_OP_SYM_MOMENT3: return st::moment3_workspace(a, b, flags);
+    case ST_OP_SYM_MOMENT4: return st::moment4_workspace(a, b, flags);
     case ST_OP_MTTKRP_TRI: return (a > 0 && b > 0 && c > 0) ? st::kWsHeaderBytes : 0;
     case ST_OP_TTM_BLOCKDIAG:
         if (a <= 0 || b <= 0 || c <= 0 || e <= 0) return 0;

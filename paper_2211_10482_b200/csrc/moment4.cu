@@ -1,0 +1,156 @@
+// st_sym_moment4: out[s(i,j,k,l)] = sum_n X[n,i] X[n,j] X[n,k] X[n,l] over the unique set
+// 0<=i<=j<=k<=l<d (Section 3, M3 = vec(f (x) f) (x) vec(f (x) f) summed over samples; its unique
+// elements are the 4-tuples with repetition, about 23x fewer than d^4).
+//
+// M3 is the second moment of the pair features: with P[n,(i,j)] = X[n,i] X[n,j] over the unique
+// pairs i<=j (the rows of vec(f (x) f) that are not redundant),
+//     out[s(i,j,k,l)] = sum_n P[n,(i,j)] P[n,(k,l)],
+// and (i,j,k,l) is a unique 4-tuple exactly when j <= k.  Three steps, all on the GPU:
+//   1. pair_expand_kernel    P [N, dP], dP = d(d+1)/2 rounded up to 64 (zero columns), fp32 or bf16
+//   2. st_sym_moment2 on P   the packed upper triangle of P^T P (fp32 kernels, or the bf16
+//                            tensor-core triangular tile GEMM with ST_FLAG_TC_BF16)
+//   3. simplex_gather_kernel rows (i,j,k,*) of the 4-simplex are runs of row (i,j), columns
+//                            (k,k)..(k,d-1) of that triangle: contiguous on both sides
+// Step 2 works on the symmetric pair-by-pair matrix, whose unique set (pairs p <= q) is about
+// three times larger than the set of unique 4-tuples: the entries with j > k are computed and
+// not gathered.
+#include "st_common.cuh"
+#include "st_index.cuh"
+#include <cuda_bf16.h>
+
+namespace st {
+
+size_t moment2_workspace(int64_t N, int64_t d, int xdt, unsigned flags);
+
+namespace m4 {
+
+constexpr int MAX_D = 64;
+constexpr int EXP_ROWS = 8;         // sample rows per pass of a block
+constexpr int EXP_THREADS = 256;
+
+struct Plan {
+    int64_t dP, p_bytes, m2_elems, m2_ws;
+    size_t off_p, off_m2, off_ws, total;
+    bool bf16, ok;
+};
+
+static Plan plan(int64_t N, int64_t d, unsigned flags)
+{
+    Plan p{};
+    p.ok = false;
+    if (N <= 0 || d < 1 || d > MAX_D) return p;
+    p.bf16 = (flags & ST_FLAG_TC_BF16) != 0;
+    p.dP = (tri_rows(d) + 63) / 64 * 64;
+    p.p_bytes = N * p.dP * (p.bf16 ? 2 : 4);
+    p.m2_elems = tri_rows(p.dP);
+    p.m2_ws = (int64_t)moment2_workspace(N, p.dP, p.bf16 ? ST_BF16 : ST_F32, 0);
+    if (p.m2_ws == 0) return p;
+    p.off_p = kWsHeaderBytes;
+    p.off_m2 = round_up(p.off_p + (size_t)p.p_bytes, 256);
+    p.off_ws = round_up(p.off_m2 + (size_t)p.m2_elems * 4, 256);
+    p.total = p.off_ws + (size_t)p.m2_ws;
+    p.ok = true;
+    return p;
+}
+
+__device__ __forceinline__ void store_pair(float *P, int64_t at, float a, float b)
+{
+    *reinterpret_cast<float2 *>(P + at) = make_float2(a, b);
+}
+__device__ __forceinline__ void store_pair(__nv_bfloat16 *P, int64_t at, float a, float b)
+{
+    *reinterpret_cast<__nv_bfloat162 *>(P + at) = __floats2bfloat162_rn(a, b);
+}
+
+// P[n, p(i,j)] = X[n,i] X[n,j] for the unique pairs in packed order, zeros in the padding
+// columns.  A block stages EXP_ROWS rows of X and writes their rows of P two columns per thread.
+template <typename OutT>
+__global__ void __launch_bounds__(EXP_THREADS)
+pair_expand_kernel(const float *__restrict__ X, int64_t N, int d, int64_t ldx, OutT *__restrict__ P, int dP, int npairs)
+{
+    extern __shared__ __align__(16) unsigned char sm[];
+    unsigned short *tab = reinterpret_cast<unsigned short *>(sm);              // [dP]: i | j << 8, 0xffff = padding
+    float *xs = reinterpret_cast<float *>(sm + ((size_t)dP * 2 + 15) / 16 * 16);  // [EXP_ROWS][d]
+    for (int p = threadIdx.x; p < dP; p += EXP_THREADS) {
+        int64_t i = 0, j = 0;
+        if (p < npairs) tri_decode(d, p, i, j);
+        tab[p] = p < npairs ? (unsigned short)(i | (j << 8)) : (unsigned short)0xffff;
+    }
+    const int half = dP / 2;
+    for (int64_t row0 = (int64_t)blockIdx.x * EXP_ROWS; row0 < N; row0 += (int64_t)gridDim.x * EXP_ROWS) {
+        __syncthreads();
+        for (int e = threadIdx.x; e < EXP_ROWS * d; e += EXP_THREADS) {
+            const int r = e / d, c = e - r * d;
+            xs[e] = row0 + r < N ? X[(row0 + r) * ldx + c] : 0.f;
+        }
+        __syncthreads();
+        for (int e = threadIdx.x; e < EXP_ROWS * half; e += EXP_THREADS) {
+            const int r = e / half, p = 2 * (e - r * half);
+            if (row0 + r >= N) break;
+            const unsigned t0 = tab[p], t1 = tab[p + 1];
+            const float *x = xs + r * d;
+            const float a = t0 == 0xffffu ? 0.f : x[t0 & 255u] * x[t0 >> 8];
+            const float b = t1 == 0xffffu ? 0.f : x[t1 & 255u] * x[t1 >> 8];
+            store_pair(P, (row0 + r) * dP + p, a, b);
+        }
+    }
+}
+
+// One block per row (i,j,k) of the 4-simplex: out[s(i,j,k,l)], l = k..d-1, is the run of row (i,j),
+// columns (k,k)..(k,d-1) of the packed pair-by-pair triangle.
+__global__ void __launch_bounds__(64)
+simplex_gather_kernel(const float *__restrict__ M2, float *__restrict__ out, int d, int64_t dP)
+{
+    int64_t i, j, k;
+    tet_decode(d, blockIdx.x, i, j, k);
+    const int64_t p = tri_encode(d, i, j), q = tri_encode(d, k, k);       // p <= q because j <= k
+    const float *src = M2 + tri_encode(dP, p, q);
+    float *dst = out + simp4_encode(d, i, j, k, k);
+    for (int o = threadIdx.x; o < d - k; o += 64) dst[o] = src[o];
+}
+
+}  // namespace m4
+
+size_t moment4_workspace(int64_t N, int64_t d, unsigned flags)
+{
+    const m4::Plan p = m4::plan(N, d, flags);
+    return p.ok ? p.total : 0;
+}
+
+}  // namespace st
+
+extern "C" st_status st_sym_moment4(const float *X, int64_t N, int64_t d, int64_t ldx, float *out_packed, void *ws,
+                                    size_t ws_bytes, unsigned flags, void *stream_)
+{
+    using namespace st;
+    using namespace st::m4;
+    if (!X || !out_packed) return ST_ERR_NULL;
+    if (N <= 0 || d <= 0 || ldx < d) return ST_ERR_SHAPE;
+    if (flags & ~(ST_FLAG_TC_BF16)) return ST_ERR_UNSUPPORTED;
+    if (d > MAX_D) return ST_ERR_UNSUPPORTED;
+    if (!aligned16(X) || !aligned16(out_packed)) return ST_ERR_ALIGN;
+    const Plan p = plan(N, d, flags);
+    if (!p.ok) return ST_ERR_UNSUPPORTED;
+    if (!ws || ws_bytes < p.total) return ST_ERR_WORKSPACE;
+    if (!aligned256(ws)) return ST_ERR_ALIGN;
+    cudaStream_t stream = (cudaStream_t)stream_;
+    unsigned char *w = (unsigned char *)ws;
+    float *M2 = (float *)(w + p.off_m2);
+    const int npairs = (int)tri_rows(d);
+    const size_t smem = ((size_t)p.dP * 2 + 15) / 16 * 16 + (size_t)EXP_ROWS * d * sizeof(float);
+    const int64_t passes = (N + EXP_ROWS - 1) / EXP_ROWS;
+    const int64_t cap = (int64_t)sm_count_or_default() * 8;
+    const unsigned grid = (unsigned)(passes < cap ? passes : cap);
+    if (p.bf16)
+        pair_expand_kernel<__nv_bfloat16><<<grid, EXP_THREADS, smem, stream>>>(X, N, (int)d, ldx, (__nv_bfloat16 *)(w + p.off_p),
+                                                                                (int)p.dP, npairs);
+    else
+        pair_expand_kernel<float><<<grid, EXP_THREADS, smem, stream>>>(X, N, (int)d, ldx, (float *)(w + p.off_p), (int)p.dP,
+                                                                        npairs);
+    if (cudaGetLastError() != cudaSuccess) return ST_ERR_CUDA;
+    const st_status rc = st_sym_moment2(w + p.off_p, p.bf16 ? ST_BF16 : ST_F32, N, p.dP, p.dP, M2, w + p.off_ws,
+                                        (size_t)p.m2_ws, 0, stream_);
+    if (rc != ST_OK) return rc;
+    simplex_gather_kernel<<<(unsigned)tet_rows(d), 64, 0, stream>>>(M2, out_packed, (int)d, p.dP);
+    return launch_status();
+}

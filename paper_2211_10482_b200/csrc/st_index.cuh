@@ -63,4 +63,12 @@ ST_HD void tet_decode(int64_t d, int64_t q, int64_t &i, int64_t &j, int64_t &k)
     k = i + kk;
 }
 
+// Packed 4-simplex 0<=i<=j<=k<=l<d in lexicographic order: slabs i, each a tetrahedron of side d-i.
+ST_HD int64_t simp4_rows(int64_t d) { return tet_rows(d) * (d + 3) / 4; }   // C(d+3, 4), exact
+ST_HD int64_t simp4_slab_start(int64_t d, int64_t i) { return simp4_rows(d) - simp4_rows(d - i); }
+ST_HD int64_t simp4_encode(int64_t d, int64_t i, int64_t j, int64_t k, int64_t l)
+{
+    return simp4_slab_start(d, i) + tet_encode(d - i, j - i, k - i, l - i);
+}
+
 }  // namespace st

@@ -43,4 +43,15 @@ long long shim_check_all_tet(long long d)
             }
     return bad + (q != st::tet_rows(d));
 }
+long long shim_simp4_rows(long long d) { return st::simp4_rows(d); }
+// every position of the 4-simplex against a running counter; returns the number of mismatches
+long long shim_check_all_simp4(long long d)
+{
+    long long bad = 0, s = 0;
+    for (long long i = 0; i < d; ++i)
+        for (long long j = i; j < d; ++j)
+            for (long long k = j; k < d; ++k)
+                for (long long l = k; l < d; ++l, ++s) bad += st::simp4_encode(d, i, j, k, l) != s;
+    return bad + (s != st::simp4_rows(d));
+}
 }

@@ -2,6 +2,7 @@
 seeded inputs.  Integer / byte work must be bit-exact; fp32 paths must satisfy
 max |gpu - oracle| / sum|terms| <= 1e-4."""
 import itertools
+import math
 
 import numpy as np
 import pytest
@@ -318,6 +319,68 @@ def test_moment3_tensor_core_config(st, kind):
     Xd = X.astype(np.float64)
     lhs, rhs = float(np.dot(mult, got.astype(np.float64))), float(np.sum(Xd.sum(axis=1) ** 3))
     assert abs(lhs - rhs) <= TOL_TC * float(np.sum(np.abs(Xd).sum(axis=1) ** 3))
+
+
+# fourth moment: packed 4-simplex i<=j<=k<=l in lexicographic order
+
+def simplex4_tuples(d):
+    """The unique set in packed order, by a running walk (no closed form)."""
+    return [(i, j, k, l) for i in range(d) for j in range(i, d) for k in range(j, d) for l in range(k, d)]
+
+
+@pytest.mark.parametrize("N,d", [(1, 1), (5, 2), (33, 3), (100, 5), (257, 8), (1000, 11), (64, 12), (500, 16)])
+def test_moment4_f32_small(st, N, d):
+    X = workloads.draw((N, d), "normal", 600 + N + d)
+    T, S = oracle.moment4(X)
+    got = st.st_sym_moment4(dev(X)).cpu().numpy()
+    tup = simplex4_tuples(d)
+    assert got.size == len(tup) == math.comb(d + 3, 4)
+    ii, jj, kk, ll = (np.array(v) for v in zip(*tup))
+    assert oracle.rel_err(got, T[ii, jj, kk, ll], S[ii, jj, kk, ll]) <= TOL_F32, (N, d)
+
+
+@pytest.mark.parametrize("flag_name,N,d,tol", [("f32", 3000, 24, TOL_F32), ("f32", 700, 40, TOL_F32),
+                                               ("bf16", 1000, 8, 5e-3), ("bf16", 5000, 24, 5e-3),
+                                               ("bf16", 2000, 64, 5e-3), ("bf16", 65536, 32, 5e-3)])
+def test_moment4_sampled_entries_and_multiplicity_identity(st, flag_name, N, d, tol):
+    flags = st.ST_FLAG_TC_BF16 if flag_name == "bf16" else 0
+    X = workloads.draw((N, d), "normal", 700 + N + d)
+    got = st.st_sym_moment4(dev(X), flags=flags).cpu().numpy()
+    tup = simplex4_tuples(d)
+    assert got.size == len(tup)
+    rng = np.random.default_rng(7)
+    pick = np.unique(np.concatenate([rng.integers(0, len(tup), 4000), [0, len(tup) - 1]]))
+    pick = np.concatenate([pick, [n for n, t in enumerate(tup) if len(set(t)) == 1]])      # all (i,i,i,i)
+    ii, jj, kk, ll = (np.array([tup[n][c] for n in pick]) for c in range(4))
+    T, S = oracle.moment4_at(X, ii, jj, kk, ll)
+    assert oracle.rel_err(got[pick], T, S) <= tol, (N, d)
+    # sum over the unique set weighted by the number of index tuples each entry stands for equals
+    # sum_n (sum_i x_i)^4 (holds at any size)
+    mult = np.array([24 // math.prod(math.factorial(t.count(v)) for v in set(t)) for t in tup], np.float64)
+    Xd = X.astype(np.float64)
+    lhs, rhs = float(np.dot(mult, got.astype(np.float64))), float(np.sum(Xd.sum(axis=1) ** 4))
+    assert abs(lhs - rhs) <= tol * float(np.sum(np.abs(Xd).sum(axis=1) ** 4))
+
+
+def test_moment4_all_ones_pitch_and_errors(st):
+    ones = torch.ones((321, 20), dtype=torch.float32, device="cuda")
+    assert torch.all(st.st_sym_moment4(ones) == 321.0)
+    assert torch.all(st.st_sym_moment4(ones, flags=st.ST_FLAG_TC_BF16) == 321.0)
+    wide = dev(workloads.draw((300, 20), "uniform", 5))
+    d, N = 9, 300
+    out = torch.empty(math.comb(d + 3, 4), dtype=torch.float32, device="cuda")
+    ws = torch.empty(st.st_workspace_bytes(st.ST_OP_SYM_MOMENT4, N, d), dtype=torch.uint8, device="cuda")
+    s = torch.cuda.current_stream().cuda_stream
+    L = st.lib()
+    assert L.st_sym_moment4(wide.data_ptr(), N, d, 20, out.data_ptr(), ws.data_ptr(), ws.numel(), 0, s) == st.ST_OK
+    T, S = oracle.moment4(np.ascontiguousarray(wide.cpu().numpy()[:, :d]))
+    ii, jj, kk, ll = (np.array(v) for v in zip(*simplex4_tuples(d)))
+    assert oracle.rel_err(out.cpu().numpy(), T[ii, jj, kk, ll], S[ii, jj, kk, ll]) <= TOL_F32
+    assert L.st_sym_moment4(None, N, d, 20, out.data_ptr(), ws.data_ptr(), ws.numel(), 0, s) == st.ST_ERR_NULL
+    assert L.st_sym_moment4(wide.data_ptr(), N, 65, 65, out.data_ptr(), ws.data_ptr(), ws.numel(), 0, s) == st.ST_ERR_UNSUPPORTED
+    assert L.st_sym_moment4(wide.data_ptr(), N, d, 20, out.data_ptr(), ws.data_ptr(), 1024, 0, s) == st.ST_ERR_WORKSPACE
+    assert L.st_sym_moment4(wide.data_ptr(), N, d, 8, out.data_ptr(), ws.data_ptr(), ws.numel(), 0, s) == st.ST_ERR_SHAPE
+    assert L.st_sym_moment4(wide.data_ptr(), N, d, 20, out.data_ptr(), ws.data_ptr(), ws.numel(), 1, s) == st.ST_ERR_UNSUPPORTED
 
 
 # ------------------------------------------------------------------------------ MTTKRP / TTM

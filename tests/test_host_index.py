@@ -22,7 +22,8 @@ def shim():
                            os.path.join(ROOT, "tests", "index_host_shim.cpp"), "-o", out])
     L = ctypes.CDLL(out)
     ll = ctypes.c_longlong
-    for name in ("shim_tri_rows", "shim_tet_rows", "shim_check_all_tri", "shim_check_all_tet"):
+    for name in ("shim_tri_rows", "shim_tet_rows", "shim_check_all_tri", "shim_check_all_tet", "shim_simp4_rows",
+                 "shim_check_all_simp4"):
         getattr(L, name).argtypes = [ll]
         getattr(L, name).restype = ll
     L.shim_tri_encode.argtypes = [ll, ll, ll]
@@ -54,6 +55,15 @@ def test_decode_is_exact_for_every_position(shim):
         assert shim.shim_check_all_tet(d) == 0
     for d in (1000, 1024, 4097):
         assert shim.shim_check_all_tri(d) == 0
+
+
+def test_four_simplex_positions_and_the_count_the_paper_gives(shim):
+    # Section 2, "Intricate Structures": the degree-2 polynomial-regression covariance on 4 features has
+    # 65 distinct elements = 10 (pairs) + 20 (triples) + 35 (4-tuples with repetition)
+    assert shim.shim_tri_rows(4) + shim.shim_tet_rows(4) + shim.shim_simp4_rows(4) == 65
+    assert shim.shim_simp4_rows(4) == 35
+    for d in list(range(1, 20)) + [33, 64]:
+        assert shim.shim_check_all_simp4(d) == 0
 
 
 def test_decode_at_boundaries_of_large_extents(shim):

@@ -127,6 +127,19 @@ def test_moment3_d1_is_sum_of_cubes():
     assert abs(S[0, 0, 0] - np.sum(np.abs(X.astype(np.float64)) ** 3)) < 1e-12
 
 
+def test_moment4_at_is_the_dense_sum_at_sampled_entries():
+    X = workloads.draw((37, 6), "normal", 21)
+    T, S = oracle.moment4(X)
+    idx = [(i, j, k, l) for i in range(6) for j in range(6) for k in range(6) for l in range(6)][::7]
+    ii, jj, kk, ll = (np.array(v) for v in zip(*idx))
+    t, sabs = oracle.moment4_at(X, ii, jj, kk, ll)
+    assert np.array_equal(t, T[ii, jj, kk, ll]) and np.array_equal(sabs, S[ii, jj, kk, ll])
+    # d = 1 reduces to a plain sum of fourth powers
+    x = workloads.draw((50, 1), "uniform", 22)
+    t1, _ = oracle.moment4_at(x, [0], [0], [0], [0])
+    assert abs(t1[0] - float(np.sum(x.astype(np.float64) ** 4))) <= 1e-12
+
+
 def test_moment4_einsum():
     X = rnd((33, 5), 13)
     Xd = X.astype(np.float64)
