@@ -213,6 +213,28 @@ st_status st_ttm_blockdiag(const float *Bp, int64_t nblocks, int64_t bs, int64_t
                            const float *U, int64_t R, float *Ap, void *ws, size_t ws_bytes,
                            unsigned flags, void *stream);
 
+/* TTM (Table 1) on a tensor with any supported structure in its first two modes:
+ *     Ap[p, r] = sum_k Bp[p, k] * U[k, r]      for every packed position p of the layout
+ * `layout` describes B with inner = K: ST_TRI_UPPER is Table 1's "upper half cube" (i <= j),
+ * ST_BLOCKDIAG with bs = 1 (or ST_BAND with kl = ku = 0) its "diagonal plane" (i = j), ST_TET a
+ * 4-mode tensor with i <= j <= k.  The output has the structure of the input with inner = R
+ * (the unique set of the product, projected over k, keeps B's (i,j) part: Section 5.1).
+ * Same kernels, flags (ST_FLAG_TC_TF32 only) and shape limits as st_ttm_blockdiag; the
+ * workspace is that of ST_OP_TTM_BLOCKDIAG. */
+st_status st_ttm_packed(const st_layout *layout, const float *Bp, const float *U, int64_t R,
+                        float *Ap, void *ws, size_t ws_bytes, unsigned flags, void *stream);
+
+/* THP (Table 1), the element-wise product A(i,j,k) = B(i,j,k) * C(i,j,k) of a structured B
+ * and a dense C.  The unique set of a product is the intersection of the operands' unique sets
+ * (Section 5.1), so A has the structure of B:
+ *     Ap[p, k] = Bp[p, k] * C[position of p in the dense tensor, k]
+ * `layout` describes B (inner = K); Bp and Ap are packed fp32 arrays of st_packed_elems(layout)
+ * elements, C is the dense fp32 tensor [d,d,inner] ([d,d,d,inner] for ST_TET), read only at
+ * the positions of the unique set.  Ap may not overlap Bp or C.  ST_BAND slots outside the
+ * matrix are written as +0.0. */
+st_status st_thp(const st_layout *layout, const float *Bp, const float *C_dense, float *Ap,
+                 void *stream);
+
 /* Synchronises `stream`, then reads the status word a kernel may have written into the
  * workspace (a bounded wait that ran out, a failed consistency check).  ws may be NULL. */
 st_status st_check_status(const void *ws, void *stream);

@@ -191,6 +191,14 @@ def ttm(B, U):
     return A.reshape(shp), S.reshape(shp)
 
 
+def thp(B, C):
+    """A = B * C element by element (Table 1, THP) over the full dense iteration space."""
+    B, C = _f32(B), _f32(C)
+    assert B.shape == C.shape
+    A = B.astype(np.float64) * C.astype(np.float64)
+    return A, np.abs(A)
+
+
 def _dense_rows(kind, d):
     return d * d * d if kind == KIND_TET else d * d
 

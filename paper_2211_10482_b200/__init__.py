@@ -36,7 +36,8 @@ ST_FLAG_TC_BF16 = 4
 
 EXPORTS = [
     "st_packed_elems", "st_dense_elems", "st_pack", "st_unpack", "st_workspace_bytes", "st_sym_moment2",
-    "st_sym_moment3", "st_sym_moment3_static", "st_sym_moment4", "st_mttkrp_tri", "st_ttm_blockdiag", "st_check_status", "st_status_string",
+    "st_sym_moment3", "st_sym_moment3_static", "st_sym_moment4", "st_mttkrp_tri", "st_ttm_blockdiag", "st_ttm_packed",
+    "st_thp", "st_check_status", "st_status_string",
     "st_abi_version",
 ]
 
@@ -95,12 +96,14 @@ def lib() -> ctypes.CDLL:
         L.st_sym_moment4.argtypes = [vp, i64, i64, i64, vp, vp, sz, cu, vp]
         L.st_mttkrp_tri.argtypes = [vp, i64, i64, vp, vp, i64, vp, vp, sz, cu, vp]
         L.st_ttm_blockdiag.argtypes = [vp, i64, i64, i64, vp, i64, vp, vp, sz, cu, vp]
+        L.st_ttm_packed.argtypes = [LP, vp, vp, i64, vp, vp, sz, cu, vp]
+        L.st_thp.argtypes = [LP, vp, vp, vp, vp]
         L.st_check_status.argtypes = [vp, vp]
         L.st_status_string.argtypes = [ci]
         L.st_status_string.restype = ctypes.c_char_p
         L.st_abi_version.restype = ci
         for name in ("st_pack", "st_unpack", "st_sym_moment2", "st_sym_moment3", "st_sym_moment3_static", "st_sym_moment4", "st_mttkrp_tri",
-                     "st_ttm_blockdiag", "st_check_status"):
+                     "st_ttm_blockdiag", "st_ttm_packed", "st_thp", "st_check_status"):
             getattr(L, name).restype = ci
         _lib = L
     return _lib
@@ -281,6 +284,35 @@ def st_ttm_blockdiag(Bp: torch.Tensor, U: torch.Tensor, nblocks: int, bs: int,
     _check(lib().st_ttm_blockdiag(_dev(Bp, "Bp"), nblocks, bs, K, _dev(U, "U"), R, _dev(out, "out"),
                                   ws.data_ptr(), ws.numel() * ws.element_size(), flags, _stream()),
            "st_ttm_blockdiag")
+    return out
+
+
+def st_ttm_packed(Bp: torch.Tensor, U: torch.Tensor, layout: Layout, out: torch.Tensor | None = None,
+                  ws: torch.Tensor | None = None, flags: int = 0) -> torch.Tensor:
+    """Ap[p,r] = sum_k Bp[p,k] U[k,r] for every packed position p of `layout` (inner = K)."""
+    K, R = U.shape
+    if Bp.dtype != torch.float32 or U.dtype != torch.float32:
+        raise TypeError("inputs must be float32")
+    if layout.inner != K or Bp.numel() != st_packed_elems(layout):
+        raise ValueError("shape mismatch")
+    rows = Bp.numel() // K
+    if out is None:
+        out = torch.empty((rows, R), dtype=torch.float32, device=Bp.device)
+    ws = _workspace(lambda: st_workspace_bytes(ST_OP_TTM_BLOCKDIAG, rows, 1, K, R, flags), Bp.device, ws)
+    _check(lib().st_ttm_packed(ctypes.byref(layout.c()), _dev(Bp, "Bp"), _dev(U, "U"), R, _dev(out, "out"),
+                               ws.data_ptr(), ws.numel() * ws.element_size(), flags, _stream()), "st_ttm_packed")
+    return out
+
+
+def st_thp(Bp: torch.Tensor, C: torch.Tensor, layout: Layout, out: torch.Tensor | None = None) -> torch.Tensor:
+    """Ap = Bp * (C at the unique positions of `layout`): packed B, dense C, packed result."""
+    if Bp.dtype != torch.float32 or C.dtype != torch.float32:
+        raise TypeError("inputs must be float32")
+    if Bp.numel() != st_packed_elems(layout) or C.numel() != st_dense_elems(layout):
+        raise ValueError("shape mismatch")
+    if out is None:
+        out = torch.empty_like(Bp)
+    _check(lib().st_thp(ctypes.byref(layout.c()), _dev(Bp, "Bp"), _dev(C, "C"), _dev(out, "out"), _stream()), "st_thp")
     return out
 
 

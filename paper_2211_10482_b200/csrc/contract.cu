@@ -300,6 +300,27 @@ st_status st_ttm_blockdiag(const float *Bp, int64_t nblocks, int64_t bs, int64_t
     return rowgemm_launch<RG_TTM>(a, (cudaStream_t)stream);
 }
 
+st_status st_ttm_packed(const st_layout *layout, const float *Bp, const float *U, int64_t R, float *Ap, void *ws,
+                        size_t ws_bytes, unsigned flags, void *stream)
+{
+    using namespace st;
+    if (!layout || !Bp || !U || !Ap) return ST_ERR_NULL;
+    if (R <= 0) return ST_ERR_SHAPE;
+    if (flags & ~(ST_FLAG_TC_TF32)) return ST_ERR_UNSUPPORTED;
+    if (!aligned16(Bp) || !aligned16(U) || !aligned16(Ap)) return ST_ERR_ALIGN;
+    const int64_t K = layout->inner;
+    const int64_t elems = st_packed_elems(layout);      // validates the layout
+    if (elems <= 0 || K <= 0) return ST_ERR_SHAPE;
+    const int64_t rows = elems / K;                      // one fibre along k per packed position
+    if (K > (1 << 20) || rows / 256 + 1 > (int64_t(1) << 28)) return ST_ERR_UNSUPPORTED;
+    if (flags & ST_FLAG_TC_TF32) return ttm_tf32_tc(Bp, rows, K, U, R, Ap, ws, ws_bytes, (cudaStream_t)stream);
+    if (K % 4 != 0) return ST_ERR_UNSUPPORTED;
+    if (R != 8 && R != 16 && R != 32 && R != 64) return ST_ERR_UNSUPPORTED;
+    RgArgs a{};
+    a.B = Bp; a.W = U; a.C = nullptr; a.out = Ap; a.rows = rows; a.K = (int)K; a.R = (int)R; a.I = 0;
+    return rowgemm_launch<RG_TTM>(a, (cudaStream_t)stream);
+}
+
 st_status st_mttkrp_tri(const float *Bp, int64_t I, int64_t K, const float *C, const float *D, int64_t R,
                         float *A, void *ws, size_t ws_bytes, unsigned flags, void *stream)
 {

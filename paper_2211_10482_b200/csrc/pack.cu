@@ -95,6 +95,25 @@ template <> __device__ __forceinline__ uint2 zero_unit<uint2>() { return make_ui
 template <> __device__ __forceinline__ uint32_t zero_unit<uint32_t>() { return 0u; }
 template <> __device__ __forceinline__ uint16_t zero_unit<uint16_t>() { return 0; }
 
+// Element-wise product of two units of fp32 values (the Hadamard variant of st_pack).
+__device__ __forceinline__ uint4 mul_unit(uint4 a, uint4 b)
+{
+    return make_uint4(__float_as_uint(__uint_as_float(a.x) * __uint_as_float(b.x)),
+                      __float_as_uint(__uint_as_float(a.y) * __uint_as_float(b.y)),
+                      __float_as_uint(__uint_as_float(a.z) * __uint_as_float(b.z)),
+                      __float_as_uint(__uint_as_float(a.w) * __uint_as_float(b.w)));
+}
+__device__ __forceinline__ uint2 mul_unit(uint2 a, uint2 b)
+{
+    return make_uint2(__float_as_uint(__uint_as_float(a.x) * __uint_as_float(b.x)),
+                      __float_as_uint(__uint_as_float(a.y) * __uint_as_float(b.y)));
+}
+__device__ __forceinline__ uint32_t mul_unit(uint32_t a, uint32_t b)
+{
+    return __float_as_uint(__uint_as_float(a) * __uint_as_float(b));
+}
+__device__ __forceinline__ uint16_t mul_unit(uint16_t a, uint16_t) { return a; }   // not reached: fp32 rows are whole words
+
 // PACK = true : rows of `dst` are packed rows, source rows are dense rows.
 // PACK = false: rows of `dst` are dense rows, source rows are packed rows.
 template <int KIND, typename U, bool PACK>
@@ -144,8 +163,9 @@ __device__ __forceinline__ void slice_run(const LayoutArgs &a, int64_t s, int64_
 template <int KIND, typename U, bool PACK>
 __global__ void __launch_bounds__(256)
 slice_copy_kernel(const U *__restrict__ src, U *__restrict__ dst, LayoutArgs a, int group_shift, int parts,
-                  int64_t part_units)
+                  int64_t part_units, const U *__restrict__ mul)
 {
+    // mul (pack only, fp32 elements): a second packed operand; the gathered values are multiplied by it
     const int g = 1 << group_shift;
     const int lane = (int)(threadIdx.x & (g - 1));
     const int64_t gid = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> group_shift;
@@ -168,7 +188,12 @@ slice_copy_kernel(const U *__restrict__ src, U *__restrict__ dst, LayoutArgs a, 
         if (PACK) {
             const U *in = src + s * su;
             U *out = dst + prow * a.chunks - c0;                // out[u] for dense unit u of the run
-            for (int64_t u = x0 + lane; u < x1; u += g) out[u] = in[u];
+            if (mul) {
+                const U *m = mul + prow * a.chunks - c0;
+                for (int64_t u = x0 + lane; u < x1; u += g) out[u] = mul_unit(in[u], m[u]);
+            } else {
+                for (int64_t u = x0 + lane; u < x1; u += g) out[u] = in[u];
+            }
             if (KIND == ST_BAND && part == 0) {
                 // slots of the fixed-width packed row that fall outside the matrix
                 U *row = dst + s * a.width * a.chunks;
@@ -230,7 +255,7 @@ static int dtype_bytes(st_dtype t)
 }
 
 template <int KIND, typename U, bool PACK>
-static st_status launch_copy(const void *src, void *dst, const LayoutArgs &a, cudaStream_t s)
+static st_status launch_copy(const void *src, void *dst, const LayoutArgs &a, cudaStream_t s, const void *mul)
 {
     const int64_t cap = (int64_t)sm_count_or_default() * 16;
     if (!PACK && a.fill == ST_FILL_SYMMETRIC) {
@@ -258,24 +283,24 @@ static st_status launch_copy(const void *src, void *dst, const LayoutArgs &a, cu
     const int64_t threads = (nslices * parts) << shift;
     const int64_t want = (threads + 255) / 256;
     const int grid = (int)(want < cap ? (want < 1 ? 1 : want) : cap);
-    slice_copy_kernel<KIND, U, PACK><<<grid, 256, 0, s>>>((const U *)src, (U *)dst, a, shift, parts, pu);
+    slice_copy_kernel<KIND, U, PACK><<<grid, 256, 0, s>>>((const U *)src, (U *)dst, a, shift, parts, pu, (const U *)mul);
     return launch_status();
 }
 
 template <typename U, bool PACK>
-static st_status dispatch_kind(const void *src, void *dst, const LayoutArgs &a, cudaStream_t s)
+static st_status dispatch_kind(const void *src, void *dst, const LayoutArgs &a, cudaStream_t s, const void *mul)
 {
     switch (a.kind) {
-    case ST_TRI_UPPER: return launch_copy<ST_TRI_UPPER, U, PACK>(src, dst, a, s);
-    case ST_TET: return launch_copy<ST_TET, U, PACK>(src, dst, a, s);
-    case ST_BAND: return launch_copy<ST_BAND, U, PACK>(src, dst, a, s);
-    default: return launch_copy<ST_BLOCKDIAG, U, PACK>(src, dst, a, s);
+    case ST_TRI_UPPER: return launch_copy<ST_TRI_UPPER, U, PACK>(src, dst, a, s, mul);
+    case ST_TET: return launch_copy<ST_TET, U, PACK>(src, dst, a, s, mul);
+    case ST_BAND: return launch_copy<ST_BAND, U, PACK>(src, dst, a, s, mul);
+    default: return launch_copy<ST_BLOCKDIAG, U, PACK>(src, dst, a, s, mul);
     }
 }
 
 template <bool PACK>
 static st_status copy_entry(const st_layout *L, st_dtype dtype, const void *src, void *dst, int fill,
-                            void *stream)
+                            void *stream, const void *mul = nullptr)
 {
     if (!L || !src || !dst) return ST_ERR_NULL;
     if (!layout_ok(L)) return ST_ERR_SHAPE;
@@ -293,11 +318,11 @@ static st_status copy_entry(const st_layout *L, st_dtype dtype, const void *src,
     a.dense_rows = dense_rows_of(L);
     const int64_t w = L->inner * es;   // bytes per row
     cudaStream_t s = (cudaStream_t)stream;
-    if (w % 16 == 0) { a.chunks = w / 16; return dispatch_kind<uint4, PACK>(src, dst, a, s); }
-    if (w % 8 == 0)  { a.chunks = w / 8;  return dispatch_kind<uint2, PACK>(src, dst, a, s); }
-    if (w % 4 == 0)  { a.chunks = w / 4;  return dispatch_kind<uint32_t, PACK>(src, dst, a, s); }
+    if (w % 16 == 0) { a.chunks = w / 16; return dispatch_kind<uint4, PACK>(src, dst, a, s, mul); }
+    if (w % 8 == 0)  { a.chunks = w / 8;  return dispatch_kind<uint2, PACK>(src, dst, a, s, mul); }
+    if (w % 4 == 0)  { a.chunks = w / 4;  return dispatch_kind<uint32_t, PACK>(src, dst, a, s, mul); }
     a.chunks = w / 2;
-    return dispatch_kind<uint16_t, PACK>(src, dst, a, s);
+    return dispatch_kind<uint16_t, PACK>(src, dst, a, s, mul);
 }
 
 }  // namespace st
@@ -319,6 +344,14 @@ int64_t st_dense_elems(const st_layout *layout)
 st_status st_pack(const st_layout *layout, st_dtype dtype, const void *dense, void *packed, void *stream)
 {
     return st::copy_entry<true>(layout, dtype, dense, packed, ST_FILL_ZERO, stream);
+}
+
+st_status st_thp(const st_layout *layout, const float *Bp, const float *C_dense, float *Ap, void *stream)
+{
+    if (!Bp) return ST_ERR_NULL;
+    if (!st::aligned16(Bp)) return ST_ERR_ALIGN;
+    // the pack of C with every gathered value multiplied by the packed operand at the same position
+    return st::copy_entry<true>(layout, ST_F32, C_dense, Ap, ST_FILL_ZERO, stream, Bp);
 }
 
 st_status st_unpack(const st_layout *layout, st_dtype dtype, const void *packed, void *dense, st_fill fill,

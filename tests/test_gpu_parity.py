@@ -560,3 +560,61 @@ def test_mttkrp_tf32_config(st):
     for i0 in (0, 1, 255, 256, 300, 480, 510, 511):
         A, S = oracle.mttkrp(Bd, C, D, i0, i0 + 1)
         assert oracle.rel_err(got[i0:i0 + 1], A, S) <= TOL_TC, i0
+
+
+# ------------------------------------------------------------------------------ other structures of Table 1
+
+def _table1_layouts(st, K):
+    return [st.Layout(st.ST_TRI_UPPER, 13, inner=K),                      # upper half cube (i <= j)
+            st.Layout(st.ST_BLOCKDIAG, 37, inner=K, nblocks=37, bs=1),     # diagonal plane (i = j)
+            st.Layout(st.ST_BAND, 21, inner=K, kl=2, ku=1),
+            st.Layout(st.ST_BLOCKDIAG, 24, inner=K, nblocks=3, bs=8),
+            st.Layout(st.ST_TET, 7, inner=K)]
+
+
+def _okind(st, lay):
+    return {st.ST_TRI_UPPER: oracle.KIND_TRI, st.ST_TET: oracle.KIND_TET, st.ST_BAND: oracle.KIND_BAND,
+            st.ST_BLOCKDIAG: oracle.KIND_BLOCKDIAG}[lay.kind]
+
+
+@pytest.mark.parametrize("flag_name,K,R", [("f32", 36, 32), ("f32", 64, 8), ("tf32", 64, 32), ("tf32", 36, 48)])
+def test_ttm_on_every_structure_of_the_first_two_modes(st, flag_name, K, R):
+    flags = st.ST_FLAG_TC_TF32 if flag_name == "tf32" else 0
+    for n, lay in enumerate(_table1_layouts(st, K)):
+        rows = st.st_packed_elems(lay) // K
+        Bp = workloads.draw((rows, K), "normal", 800 + n)
+        U = workloads.draw((K, R), "normal", 850 + n)
+        if lay.kind == st.ST_BAND:      # slots outside the matrix hold zeros in a packed band
+            Bp = oracle.pack(oracle.unpack(Bp.reshape(-1), oracle.KIND_BAND, lay.d, inner=K, **okw(lay)),
+                             oracle.KIND_BAND, lay.d, inner=K, **okw(lay)).reshape(rows, K)
+        # oracle: the dense tensor (zeros outside the structure) times U over the full iteration space,
+        # then the structured part of the result
+        Bd = oracle.unpack(Bp.reshape(-1), _okind(st, lay), lay.d, inner=K, **okw(lay))
+        A, S = oracle.ttm(Bd, U)
+        want = oracle.pack(A, _okind(st, lay), lay.d, inner=R, **okw(lay)).reshape(rows, R)
+        scale = oracle.pack(S, _okind(st, lay), lay.d, inner=R, **okw(lay)).reshape(rows, R)
+        got = st.st_ttm_packed(dev(Bp), dev(U), lay, flags=flags).cpu().numpy()
+        assert oracle.rel_err(got, want, scale) <= (5e-3 if flags else TOL_F32), (flag_name, n)
+        # everything outside the structure of the dense result is exactly zero (output keeps B's structure)
+        mask = oracle.unpack(np.ones(rows * R, np.float32), _okind(st, lay), lay.d, inner=R, **okw(lay))
+        assert np.all(A[mask == 0] == 0)
+
+
+def test_thp_structured_times_dense(st):
+    for n, lay in enumerate(_table1_layouts(st, 12) + [st.Layout(st.ST_TRI_UPPER, 300, inner=5)]):
+        K = lay.inner
+        elems = st.st_packed_elems(lay)
+        Bp = workloads.draw((elems,), "normal", 900 + n)
+        Cd = workloads.draw((st.st_dense_elems(lay),), "uniform", 950 + n)
+        if lay.kind == st.ST_BAND:
+            Bp = oracle.pack(oracle.unpack(Bp, oracle.KIND_BAND, lay.d, inner=K, **okw(lay)), oracle.KIND_BAND, lay.d,
+                             inner=K, **okw(lay))
+        Bd = oracle.unpack(Bp, _okind(st, lay), lay.d, inner=K, **okw(lay))
+        A, _ = oracle.thp(Bd, Cd.reshape(Bd.shape))
+        want = oracle.pack(A.astype(np.float32), _okind(st, lay), lay.d, inner=K, **okw(lay))
+        got = st.st_thp(dev(Bp), dev(Cd), lay).cpu().numpy()
+        # one fp32 multiplication of two fp32 numbers: the correctly rounded product, bit for bit
+        assert np.array_equal(got.view(np.uint32), want.view(np.uint32)), n
+        # the dense result is zero wherever B is (the product keeps B's structure)
+        mask = oracle.unpack(np.ones(elems, np.float32), _okind(st, lay), lay.d, inner=K, **okw(lay))
+        assert np.all(A[mask == 0] == 0)
