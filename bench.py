@@ -83,9 +83,16 @@ def step_table(cfg):
     for kind, scale in (("tf32", 0.5), ("bf16", 1.0)):
         t["sym_moment3_" + kind] = dict(flops=t["sym_moment3"]["flops"], bytes=t["sym_moment3"]["bytes"],
                                         bound="tensor", launches=2, tensor_scale=scale)
+    # fourth moment (last block of the degree-2 polynomial-regression covariance) on the first d features
+    c6 = cfg["moment4"]
+    simp4 = c6["d"] * (c6["d"] + 1) * (c6["d"] + 2) * (c6["d"] + 3) // 24
+    t["sym_moment4_bf16"] = dict(flops=2 * c6["N"] * simp4 + c6["N"] * tri(c6["d"]),
+                                 bytes=4 * (c6["N"] * c6["d"] + simp4), bound="tensor", launches=4)
     t["unpack_tet_sym"] = dict(flops=0, bytes=4 * (tet(c2["d"]) + c2["d"] ** 3), bound="hbm", launches=1)
     nnz3 = tri(c3["I"]) * c3["K"]
     t["pack_tri_x_k"] = dict(flops=0, bytes=2 * 4 * nnz3, bound="hbm", launches=1)
+    # THP of the packed upper-half-cube tensor with a dense one: packed operand, gathered dense operand, packed result
+    t["thp_tri_x_k"] = dict(flops=nnz3, bytes=3 * 4 * nnz3, bound="hbm", launches=1)
     t["mttkrp_tri"] = dict(flops=2 * c3["R"] * nnz3 + 2 * c3["R"] * tri(c3["I"]),
                            bytes=4 * (nnz3 + (2 * c3["I"] + c3["K"]) * c3["R"]),
                            bound=("hbm" if cfg["mttkrp_tc"] else "alu"), launches=1)
@@ -181,6 +188,7 @@ class ClockSampler:
 def bench_config():
     cfg = {k: dict(v) for k, v in workloads.CONFIGS.items()}
     cfg["band"] = dict(d=2048, kl=64, ku=63, inner=16)
+    cfg["moment4"] = dict(N=cfg["moment3"]["N"], d=32)
     cfg["m2_large_dtype"] = "bf16"
     cfg["ttm_tc"] = True
     cfg["mttkrp_tc"] = True
@@ -197,6 +205,7 @@ class Workload:
         host = {}
         host["X1"] = pin(workloads.moment_input("moment2"))
         host["X2"] = pin(workloads.moment_input("moment3"))
+        host["X4"] = pin(host["X2"].numpy()[:, :cfg["moment4"]["d"]])      # the first d features of the same samples
         Bp3, C3, D3 = workloads.mttkrp_inputs()
         host["C3"], host["D3"] = pin(C3), pin(D3)
         Bp4, U4 = workloads.ttm_inputs()
@@ -226,7 +235,9 @@ class Workload:
         self.out = {
             "m2": torch.empty(tri(c1["d"]), **f32), "m2_dense": torch.empty(c1["d"] ** 2, **f32),
             "m3": torch.empty(tet(c2["d"]), **f32), "m3_tc": torch.empty(tet(c2["d"]), **f32), "m3_dense": torch.empty(c2["d"] ** 3, **f32),
-            "Bp3": torch.empty(tri(c3["I"]) * c3["K"], **f32), "A3": torch.empty((c3["I"], c3["R"]), **f32),
+            "Bp3": torch.empty(tri(c3["I"]) * c3["K"], **f32), "thp3": torch.empty(tri(c3["I"]) * c3["K"], **f32),
+            "m4": torch.empty(cfg["moment4"]["d"] * (cfg["moment4"]["d"] + 1) * (cfg["moment4"]["d"] + 2)
+                              * (cfg["moment4"]["d"] + 3) // 24, **f32), "A3": torch.empty((c3["I"], c3["R"]), **f32),
             "Ap4": torch.empty((c4["nb"] * c4["bs"] ** 2, c4["R"]), **f32),
             "A4_dense": torch.empty((c4["nb"] * c4["bs"]) ** 2 * c4["R"], **f32),
             "band_p": torch.empty(st.st_packed_elems(self.lay_band), **f32),
@@ -240,6 +251,7 @@ class Workload:
             st.st_workspace_bytes(st.ST_OP_SYM_MOMENT3, c2["N"], c2["d"]),
             st.st_workspace_bytes(st.ST_OP_SYM_MOMENT3, c2["N"], c2["d"], 0, 0, st.ST_FLAG_TC_TF32),
             st.st_workspace_bytes(st.ST_OP_SYM_MOMENT3, c2["N"], c2["d"], 0, 0, st.ST_FLAG_TC_BF16),
+            st.st_workspace_bytes(st.ST_OP_SYM_MOMENT4, cfg["moment4"]["N"], cfg["moment4"]["d"], 0, 0, st.ST_FLAG_TC_BF16),
             st.st_workspace_bytes(st.ST_OP_MTTKRP_TRI, c3["I"], c3["K"], c3["R"]),
             st.st_workspace_bytes(st.ST_OP_TTM_BLOCKDIAG, c4["nb"], c4["bs"], c4["K"], c4["R"], self.ttm_flags),
             st.st_workspace_bytes(st.ST_OP_SYM_MOMENT2, c5["N"], c5["d"], x5dt), 256)
@@ -264,11 +276,13 @@ class Workload:
             ("pack_tri_x_k", lambda: st.st_pack(d["B3"], self.lay3, out=o["Bp3"])),
             ("mttkrp_tri", lambda: st.st_mttkrp_tri(o["Bp3"], d["C3"], d["D3"], out=o["A3"], ws=self.ws,
                                                        flags=self.mttkrp_flags)),
+            ("thp_tri_x_k", lambda: st.st_thp(o["Bp3"], d["B3"], self.lay3, out=o["thp3"])),
             ("sym_moment3", lambda: st.st_sym_moment3(d["X2"], out=o["m3"], ws=self.ws)),
             ("sym_moment3_tf32", lambda: st.st_sym_moment3(d["X2"], out=o["m3_tc"], ws=self.ws,
                                                              flags=st.ST_FLAG_TC_TF32)),
             ("sym_moment3_bf16", lambda: st.st_sym_moment3(d["X2"], out=o["m3_tc"], ws=self.ws,
                                                              flags=st.ST_FLAG_TC_BF16)),
+            ("sym_moment4_bf16", lambda: st.st_sym_moment4(d["X4"], out=o["m4"], ws=self.ws, flags=st.ST_FLAG_TC_BF16)),
             ("unpack_tet_sym", lambda: st.st_unpack(o["m3"], self.lay2, st.ST_FILL_SYMMETRIC, out=o["m3_dense"])),
             ("pack_band", lambda: st.st_pack(d["band"], self.lay_band, out=o["band_p"])),
             ("sym_moment2", lambda: st.st_sym_moment2(d["X1"], out=o["m2"], ws=self.ws)),
@@ -474,7 +488,8 @@ def run_ours(args):
         "dtype": "f32" + ("+bf16" if cfg["m2_large_dtype"] == "bf16" else "") + ("+tf32" if (cfg["ttm_tc"] or cfg["mttkrp_tc"]) else ""),
         "data": "synthetic",
         "config": {"workload": "all five named configurations in one step: sym_moment2 [4096,64], sym_moment3 "
-                               "[65536,64], mttkrp_tri I=K=512 R=32 (%s), ttm_blockdiag 64x(64x64) K=256 R=64 (%s), "
+                               "[65536,64] (fp32, and its TF32 and bf16 tensor-core variants), sym_moment4 [65536,32] bf16, "
+                               "thp on the packed mttkrp operand, mttkrp_tri I=K=512 R=32 (%s), ttm_blockdiag 64x(64x64) K=256 R=64 (%s), "
                                "sym_moment2 large [1048576,1024] %s; plus pack/unpack of their operands"
                                % ("tf32" if cfg["mttkrp_tc"] else "f32", "tf32" if cfg["ttm_tc"] else "f32",
                                   cfg["m2_large_dtype"]),
