@@ -200,6 +200,20 @@ st_status st_mttkrp_tri(const float *Bp, int64_t I, int64_t K, const float *C, c
                         int64_t R, float *A, void *ws, size_t ws_bytes, unsigned flags,
                         void *stream);
 
+/* MTTKRP (Table 1) on a tensor that is non-zero in one slice only -- Table 1's "fixed i", "fixed j"
+ * and "fixed i,j" structures (the row / column / single-element structures R_r, C_c, H of Figure
+ * "matrix structures" applied to the first two modes):
+ *     A[i,r] = sum_j sum_k B[i,j,k] * C[j,r] * D[k,r],   B[i,j,k] = 0 unless i = fixed_i and / or j = fixed_j
+ * fixed_i, fixed_j: the fixed index, or -1 when that mode is free (at least one is fixed).
+ * Bp: the packed slice, fp32: [J, K] (fixed i; row = j), [I, K] (fixed j; row = i), [K] (both).
+ * C: [J,R]; D: [K,R]; A: dense [I,R], every element written (with fixed i only row fixed_i is
+ * non-zero: A_U(i,r) = (i = fixed_i)).  K % 4 == 0; fp32 path R in {8,16,32,64};
+ * ST_FLAG_TC_TF32 as for st_mttkrp_tri (R % 32 == 0, R <= 256, 5e-3 tolerance).
+ * Workspace: that of ST_OP_MTTKRP_TRI. */
+st_status st_mttkrp_slice(const float *Bp, int64_t I, int64_t J, int64_t K, int64_t fixed_i,
+                          int64_t fixed_j, const float *C, const float *D, int64_t R, float *A,
+                          void *ws, size_t ws_bytes, unsigned flags, void *stream);
+
 /* TTM (Table 1) on a tensor that is block-diagonal in its first two modes (a direct sum
  * of nblocks blocks of bs x bs fibres):
  *     Ap[b,i',j',r] = sum_k Bp[b,i',j',k] * U[k,r]

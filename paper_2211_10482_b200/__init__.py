@@ -36,7 +36,7 @@ ST_FLAG_TC_BF16 = 4
 
 EXPORTS = [
     "st_packed_elems", "st_dense_elems", "st_pack", "st_unpack", "st_workspace_bytes", "st_sym_moment2",
-    "st_sym_moment3", "st_sym_moment3_static", "st_sym_moment4", "st_mttkrp_tri", "st_ttm_blockdiag", "st_ttm_packed",
+    "st_sym_moment3", "st_sym_moment3_static", "st_sym_moment4", "st_mttkrp_tri", "st_mttkrp_slice", "st_ttm_blockdiag", "st_ttm_packed",
     "st_thp", "st_check_status", "st_status_string",
     "st_abi_version",
 ]
@@ -96,6 +96,7 @@ def lib() -> ctypes.CDLL:
         L.st_sym_moment4.argtypes = [vp, i64, i64, i64, vp, vp, sz, cu, vp]
         L.st_mttkrp_tri.argtypes = [vp, i64, i64, vp, vp, i64, vp, vp, sz, cu, vp]
         L.st_ttm_blockdiag.argtypes = [vp, i64, i64, i64, vp, i64, vp, vp, sz, cu, vp]
+        L.st_mttkrp_slice.argtypes = [vp, i64, i64, i64, i64, i64, vp, vp, i64, vp, vp, sz, cu, vp]
         L.st_ttm_packed.argtypes = [LP, vp, vp, i64, vp, vp, sz, cu, vp]
         L.st_thp.argtypes = [LP, vp, vp, vp, vp]
         L.st_check_status.argtypes = [vp, vp]
@@ -103,7 +104,7 @@ def lib() -> ctypes.CDLL:
         L.st_status_string.restype = ctypes.c_char_p
         L.st_abi_version.restype = ci
         for name in ("st_pack", "st_unpack", "st_sym_moment2", "st_sym_moment3", "st_sym_moment3_static", "st_sym_moment4", "st_mttkrp_tri",
-                     "st_ttm_blockdiag", "st_ttm_packed", "st_thp", "st_check_status"):
+                     "st_mttkrp_slice", "st_ttm_blockdiag", "st_ttm_packed", "st_thp", "st_check_status"):
             getattr(L, name).restype = ci
         _lib = L
     return _lib
@@ -264,6 +265,26 @@ def st_mttkrp_tri(Bp: torch.Tensor, C: torch.Tensor, D: torch.Tensor, out: torch
     _check(lib().st_mttkrp_tri(_dev(Bp, "Bp"), I, K, _dev(C, "C"), _dev(D, "D"), R, _dev(out, "out"),
                                ws.data_ptr(), ws.numel() * ws.element_size(), flags, _stream()),
            "st_mttkrp_tri")
+    return out
+
+
+def st_mttkrp_slice(Bp: torch.Tensor, C: torch.Tensor, D: torch.Tensor, I: int, fixed_i: int = -1, fixed_j: int = -1,
+                    out: torch.Tensor | None = None, ws: torch.Tensor | None = None, flags: int = 0) -> torch.Tensor:
+    """MTTKRP on a tensor that is non-zero only where i == fixed_i and / or j == fixed_j; Bp is that slice."""
+    J, R = C.shape
+    K = D.shape[0]
+    for t in (Bp, C, D):
+        if t.dtype != torch.float32:
+            raise TypeError("inputs must be float32")
+    rows = (1 if fixed_j >= 0 else J) if fixed_i >= 0 else I
+    if Bp.numel() != rows * K or D.shape[1] != R:
+        raise ValueError("shape mismatch")
+    if out is None:
+        out = torch.empty((I, R), dtype=torch.float32, device=Bp.device)
+    ws = _workspace(lambda: st_workspace_bytes(ST_OP_MTTKRP_TRI, I, K, R, 0, flags), Bp.device, ws)
+    _check(lib().st_mttkrp_slice(_dev(Bp, "Bp"), I, J, K, fixed_i, fixed_j, _dev(C, "C"), _dev(D, "D"), R,
+                                 _dev(out, "out"), ws.data_ptr(), ws.numel() * ws.element_size(), flags, _stream()),
+           "st_mttkrp_slice")
     return out
 
 

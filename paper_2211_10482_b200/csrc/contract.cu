@@ -21,6 +21,8 @@ namespace st {
 
 st_status ttm_tf32_tc(const float *Bp, int64_t rows, int64_t K, const float *U, int64_t R, float *Ap, void *ws,
                       size_t ws_bytes, cudaStream_t stream);
+st_status mttkrp_slice_tf32_tc(const float *Bp, int64_t rows, int64_t div, int64_t K, const float *C, const float *D,
+                               int64_t R, float *A, void *ws, size_t ws_bytes, cudaStream_t stream);
 st_status mttkrp_tf32_tc(const float *Bp, int64_t I, int64_t K, const float *C, const float *D, int64_t R, float *A,
                          bool dense, void *ws, size_t ws_bytes, cudaStream_t stream);
 
@@ -44,7 +46,8 @@ struct RgArgs {
     const float *C;      // MTTKRP: [I, R]
     float *out;          // TTM: [rows, R];  MTTKRP: A [I, R] (zeroed before the launch)
     int64_t rows;
-    int K, R, I;
+    int K, R, I;         // I: rows of A reachable from `out`
+    int64_t div;         // RG_MTTKRP_DENSE: fibre `row` belongs to (i, j) = (row / div, row % div)
     int tiles, ksplit, kchunks_per_split, kchunks;
 };
 
@@ -149,7 +152,7 @@ __global__ void __launch_bounds__(RG_THREADS, 1) rowgemm_kernel(const RgArgs a)
                 // first row of A touched by this tile
                 int64_t i_first, j_first;
                 if (MODE == RG_MTTKRP_PACKED) tri_decode(a.I, row0, i_first, j_first);
-                else { i_first = row0 / a.I; j_first = 0; }
+                else { i_first = row0 / a.div; j_first = 0; }
                 (void)j_first;
                 for (int e = tid; e < RG_NI * R_; e += RG_THREADS) As[e] = 0.f;
                 __syncthreads();
@@ -165,7 +168,7 @@ __global__ void __launch_bounds__(RG_THREADS, 1) rowgemm_kernel(const RgArgs a)
                     int64_t gi = -1, gj = 0;
                     if (valid) {
                         if (MODE == RG_MTTKRP_PACKED) tri_decode(a.I, row, gi, gj);
-                        else { gi = row / a.I; gj = row - gi * a.I; }
+                        else { gi = row / a.div; gj = row - gi * a.div; }
                     }
                     float v[8];
                     if (valid) {
@@ -338,9 +341,41 @@ st_status st_mttkrp_tri(const float *Bp, int64_t I, int64_t K, const float *C, c
     RgArgs a{};
     a.B = Bp; a.W = D; a.C = C; a.out = A; a.K = (int)K; a.R = (int)R; a.I = (int)I;
     a.rows = dense ? I * I : tri_rows(I);
+    a.div = I;
     if (cudaMemsetAsync(A, 0, (size_t)I * R * sizeof(float), (cudaStream_t)stream) != cudaSuccess) return ST_ERR_CUDA;
     return dense ? rowgemm_launch<RG_MTTKRP_DENSE>(a, (cudaStream_t)stream)
                  : rowgemm_launch<RG_MTTKRP_PACKED>(a, (cudaStream_t)stream);
+}
+
+st_status st_mttkrp_slice(const float *Bp, int64_t I, int64_t J, int64_t K, int64_t fixed_i, int64_t fixed_j,
+                          const float *C, const float *D, int64_t R, float *A, void *ws, size_t ws_bytes,
+                          unsigned flags, void *stream)
+{
+    using namespace st;
+    if (!Bp || !C || !D || !A) return ST_ERR_NULL;
+    if (I <= 0 || J <= 0 || K <= 0 || R <= 0) return ST_ERR_SHAPE;
+    if (fixed_i >= I || fixed_j >= J || (fixed_i < 0 && fixed_j < 0)) return ST_ERR_SHAPE;
+    if (flags & ~(ST_FLAG_TC_TF32)) return ST_ERR_UNSUPPORTED;
+    if (!aligned16(Bp) || !aligned16(C) || !aligned16(D) || !aligned16(A)) return ST_ERR_ALIGN;
+    if (I > (1 << 24) || J > (1 << 24) || K > (1 << 20) || K % 4 != 0 || R % 4 != 0) return ST_ERR_UNSUPPORTED;
+    // The fibres of the slice are the packed rows.  With (i, j) = (row / div, row % div):
+    //   fixed j: row = i, div = 1, C starts at row j0              -> (i, 0)
+    //   fixed i: row = j, div = J, A starts at row i0 (one row)     -> (0, j)
+    //   both   : one fibre, both shifts
+    const int64_t rows = fixed_i >= 0 ? (fixed_j >= 0 ? 1 : J) : I;
+    const int64_t div = fixed_i >= 0 ? (fixed_j >= 0 ? 1 : J) : 1;
+    const float *Cs = fixed_j >= 0 ? C + fixed_j * R : C;
+    float *As = fixed_i >= 0 ? A + fixed_i * R : A;
+    cudaStream_t s = (cudaStream_t)stream;
+    if (cudaMemsetAsync(A, 0, (size_t)I * R * sizeof(float), s) != cudaSuccess) return ST_ERR_CUDA;
+    if (flags & ST_FLAG_TC_TF32) return mttkrp_slice_tf32_tc(Bp, rows, div, K, Cs, D, R, As, ws, ws_bytes, s);
+    if (R != 8 && R != 16 && R != 32 && R != 64) return ST_ERR_UNSUPPORTED;
+    RgArgs a{};
+    a.B = Bp; a.W = D; a.C = Cs; a.out = As; a.K = (int)K; a.R = (int)R;
+    a.I = (int)(fixed_i >= 0 ? 1 : I);
+    a.rows = rows;
+    a.div = div;
+    return rowgemm_launch<RG_MTTKRP_DENSE>(a, s);
 }
 
 }  // extern "C"

@@ -28,6 +28,7 @@ struct TtmTcArgs {
     const float *U;
     const float *C;      // MTTKRP: [I, R]
     int I, mode;
+    int64_t div;         // TC_MTTKRP_DENSE: fibre `row` belongs to (i, j) = (row / div, row % div)
     float *out;
     unsigned *status;
     int64_t rows;
@@ -202,7 +203,7 @@ ttm_tc_kernel(const __grid_constant__ CUtensorMap tmap, const TtmTcArgs a)
                 int64_t gi = -1, gj = 0;
                 if (valid) {
                     if (a.mode == TC_MTTKRP_PACKED) tri_decode(a.I, row, gi, gj);
-                    else { gi = row / a.I; gj = row - gi * a.I; }
+                    else { gi = row / a.div; gj = row - gi * a.div; }
                 }
                 const int gi32 = (int)gi;
                 const bool uniform = __shfl_sync(0xffffffffu, gi32, 0) == __shfl_sync(0xffffffffu, gi32, 31) && gi32 >= 0;
@@ -295,7 +296,8 @@ size_t ttm_tf32_tc_workspace(int64_t rows, int64_t K, int64_t R)
 }
 
 static st_status tc_rows_launch(const float *Bp, int64_t rows, int64_t K, const float *U, int64_t R, float *Ap,
-                                const float *C, int64_t I, int mode, void *ws, size_t ws_bytes, cudaStream_t stream);
+                                const float *C, int64_t I, int mode, void *ws, size_t ws_bytes, cudaStream_t stream,
+                                int64_t div = 0);
 
 st_status ttm_tf32_tc(const float *Bp, int64_t rows, int64_t K, const float *U, int64_t R, float *Ap, void *ws,
                       size_t ws_bytes, cudaStream_t stream)
@@ -314,8 +316,18 @@ st_status mttkrp_tf32_tc(const float *Bp, int64_t I, int64_t K, const float *C, 
     return tc_rows_launch(Bp, rows, K, D, R, A, C, I, dense ? TC_MTTKRP_DENSE : TC_MTTKRP_PACKED, ws, ws_bytes, stream);
 }
 
+// MTTKRP on a slice of B (fixed i and / or fixed j): the fibres of the slice are the rows, A and C arrive
+// already shifted to the fixed row (A is zeroed by the caller).
+st_status mttkrp_slice_tf32_tc(const float *Bp, int64_t rows, int64_t div, int64_t K, const float *C, const float *D,
+                               int64_t R, float *A, void *ws, size_t ws_bytes, cudaStream_t stream)
+{
+    if (R % 32 != 0) return ST_ERR_UNSUPPORTED;
+    return tc_rows_launch(Bp, rows, K, D, R, A, C, 1, TC_MTTKRP_DENSE, ws, ws_bytes, stream, div);
+}
+
 static st_status tc_rows_launch(const float *Bp, int64_t rows, int64_t K, const float *U, int64_t R, float *Ap,
-                                const float *C, int64_t I, int mode, void *ws, size_t ws_bytes, cudaStream_t stream)
+                                const float *C, int64_t I, int mode, void *ws, size_t ws_bytes, cudaStream_t stream,
+                                int64_t div)
 {
     using namespace ttmtc;
     const TtmTcPlan p = ttm_tc_plan(K, R);
@@ -331,7 +343,7 @@ static st_status tc_rows_launch(const float *Bp, int64_t rows, int64_t K, const 
                           BM))
         return ST_ERR_CUDA;
     TtmTcArgs a;
-    a.U = U; a.C = C; a.I = (int)I; a.mode = mode; a.out = Ap; a.status = (unsigned *)ws; a.rows = rows; a.K = (int)K; a.R = (int)R;
+    a.U = U; a.C = C; a.I = (int)I; a.mode = mode; a.div = div > 0 ? div : (I > 0 ? I : 1); a.out = Ap; a.status = (unsigned *)ws; a.rows = rows; a.K = (int)K; a.R = (int)R;
     a.kchunks = p.kchunks; a.stages = p.stages; a.tmem_cols = p.tmem_cols;
     a.ntiles = (int)((rows + BM - 1) / BM);
     // MTTKRP usually runs right after the call that produced its packed operand (st_pack, or a kernel

@@ -618,3 +618,25 @@ def test_thp_structured_times_dense(st):
         # the dense result is zero wherever B is (the product keeps B's structure)
         mask = oracle.unpack(np.ones(elems, np.float32), _okind(st, lay), lay.d, inner=K, **okw(lay))
         assert np.all(A[mask == 0] == 0)
+
+
+@pytest.mark.parametrize("flag_name,I,J,K,R", [("f32", 5, 7, 36, 32), ("f32", 300, 40, 64, 8), ("f32", 33, 700, 32, 64),
+                                               ("tf32", 5, 7, 36, 32), ("tf32", 300, 260, 64, 64), ("tf32", 1, 1, 4, 32)])
+def test_mttkrp_on_slice_structures(st, flag_name, I, J, K, R):
+    flags = st.ST_FLAG_TC_TF32 if flag_name == "tf32" else 0
+    tol = 5e-3 if flags else TOL_F32
+    C = workloads.draw((J, R), "uniform", 1100)
+    D = workloads.draw((K, R), "uniform", 1101)
+    i0, j0 = I // 2, J - 1
+    for fi, fj in ((i0, -1), (-1, j0), (i0, j0)):
+        rows = (1 if fj >= 0 else J) if fi >= 0 else I
+        Bp = workloads.draw((rows, K), "normal", 1102 + rows)
+        # oracle: the dense tensor with the slice in place, full iteration space
+        Bd = np.zeros((I, J, K), np.float32)
+        if fi >= 0 and fj >= 0: Bd[fi, fj, :] = Bp[0]
+        elif fi >= 0: Bd[fi, :, :] = Bp
+        else: Bd[:, fj, :] = Bp
+        A, S = oracle.mttkrp(Bd, C, D)
+        got = torch.full((I, R), float("nan"), dtype=torch.float32, device="cuda")
+        st.st_mttkrp_slice(dev(Bp), dev(C), dev(D), I, fi, fj, out=got, flags=flags)
+        assert oracle.rel_err(got.cpu().numpy(), A, S) <= tol, (flag_name, fi, fj)     # rows outside the slice: exactly 0
