@@ -249,6 +249,19 @@ st_status st_ttm_packed(const st_layout *layout, const float *Bp, const float *U
 st_status st_thp(const st_layout *layout, const float *Bp, const float *C_dense, float *Ap,
                  void *stream);
 
+/* Chained computation in compressed space (Section 5.5: a whole chain of operations runs on T_C
+ * and the reconstruction from T_R happens once, at the end).  Two packed fp32 arrays of the SAME
+ * layout (n = st_packed_elems) are combined position by position; the result has that layout too:
+ *   st_packed_axpby   out = alpha * a + beta * b   (sum of tensors of one structure keeps the
+ *                     structure: inference rule for `+` on equal unique sets / redundancy maps,
+ *                     Figure "inference rules"; e.g. moments of several batches added up)
+ *   st_packed_mul     out = a * b                  (Hadamard product, the UHS example of
+ *                     Section 5.3 with both operands already restricted to the unique set)
+ * out may alias a or b.  Pointers 16-byte aligned. */
+st_status st_packed_axpby(int64_t n, float alpha, const float *a, float beta, const float *b,
+                          float *out, void *stream);
+st_status st_packed_mul(int64_t n, const float *a, const float *b, float *out, void *stream);
+
 /* Synchronises `stream`, then reads the status word a kernel may have written into the
  * workspace (a bounded wait that ran out, a failed consistency check).  ws may be NULL. */
 st_status st_check_status(const void *ws, void *stream);

@@ -37,7 +37,7 @@ ST_FLAG_TC_BF16 = 4
 EXPORTS = [
     "st_packed_elems", "st_dense_elems", "st_pack", "st_unpack", "st_workspace_bytes", "st_sym_moment2",
     "st_sym_moment3", "st_sym_moment3_static", "st_sym_moment4", "st_mttkrp_tri", "st_mttkrp_slice", "st_ttm_blockdiag", "st_ttm_packed",
-    "st_thp", "st_check_status", "st_status_string",
+    "st_thp", "st_packed_axpby", "st_packed_mul", "st_check_status", "st_status_string",
     "st_abi_version",
 ]
 
@@ -99,12 +99,14 @@ def lib() -> ctypes.CDLL:
         L.st_mttkrp_slice.argtypes = [vp, i64, i64, i64, i64, i64, vp, vp, i64, vp, vp, sz, cu, vp]
         L.st_ttm_packed.argtypes = [LP, vp, vp, i64, vp, vp, sz, cu, vp]
         L.st_thp.argtypes = [LP, vp, vp, vp, vp]
+        L.st_packed_axpby.argtypes = [i64, ctypes.c_float, vp, ctypes.c_float, vp, vp, vp]
+        L.st_packed_mul.argtypes = [i64, vp, vp, vp, vp]
         L.st_check_status.argtypes = [vp, vp]
         L.st_status_string.argtypes = [ci]
         L.st_status_string.restype = ctypes.c_char_p
         L.st_abi_version.restype = ci
         for name in ("st_pack", "st_unpack", "st_sym_moment2", "st_sym_moment3", "st_sym_moment3_static", "st_sym_moment4", "st_mttkrp_tri",
-                     "st_mttkrp_slice", "st_ttm_blockdiag", "st_ttm_packed", "st_thp", "st_check_status"):
+                     "st_mttkrp_slice", "st_ttm_blockdiag", "st_ttm_packed", "st_thp", "st_packed_axpby", "st_packed_mul", "st_check_status"):
             getattr(L, name).restype = ci
         _lib = L
     return _lib
@@ -334,6 +336,28 @@ def st_thp(Bp: torch.Tensor, C: torch.Tensor, layout: Layout, out: torch.Tensor 
     if out is None:
         out = torch.empty_like(Bp)
     _check(lib().st_thp(ctypes.byref(layout.c()), _dev(Bp, "Bp"), _dev(C, "C"), _dev(out, "out"), _stream()), "st_thp")
+    return out
+
+
+def st_packed_axpby(alpha: float, a: torch.Tensor, beta: float, b: torch.Tensor,
+                    out: torch.Tensor | None = None) -> torch.Tensor:
+    """out = alpha * a + beta * b for two packed float32 arrays of the same layout (out may be a or b)."""
+    if a.dtype != torch.float32 or b.dtype != torch.float32 or a.numel() != b.numel():
+        raise ValueError("two float32 arrays of the same size are needed")
+    if out is None:
+        out = torch.empty_like(a)
+    _check(lib().st_packed_axpby(a.numel(), alpha, _dev(a, "a"), beta, _dev(b, "b"), _dev(out, "out"), _stream()),
+           "st_packed_axpby")
+    return out
+
+
+def st_packed_mul(a: torch.Tensor, b: torch.Tensor, out: torch.Tensor | None = None) -> torch.Tensor:
+    """out = a * b for two packed float32 arrays of the same layout (out may be a or b)."""
+    if a.dtype != torch.float32 or b.dtype != torch.float32 or a.numel() != b.numel():
+        raise ValueError("two float32 arrays of the same size are needed")
+    if out is None:
+        out = torch.empty_like(a)
+    _check(lib().st_packed_mul(a.numel(), _dev(a, "a"), _dev(b, "b"), _dev(out, "out"), _stream()), "st_packed_mul")
     return out
 
 

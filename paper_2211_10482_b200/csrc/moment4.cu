@@ -25,7 +25,7 @@ size_t moment2_workspace(int64_t N, int64_t d, int xdt, unsigned flags);
 namespace m4 {
 
 constexpr int MAX_D = 64;
-constexpr int EXP_ROWS = 8;         // sample rows per pass of a block
+constexpr int EXP_ROWS = 32;        // sample rows per pass of a block
 constexpr int EXP_THREADS = 256;
 
 struct Plan {
@@ -63,34 +63,36 @@ __device__ __forceinline__ void store_pair(__nv_bfloat16 *P, int64_t at, float a
 }
 
 // P[n, p(i,j)] = X[n,i] X[n,j] for the unique pairs in packed order, zeros in the padding
-// columns.  A block stages EXP_ROWS rows of X and writes their rows of P two columns per thread.
+// columns.  A block stages EXP_ROWS rows of X per pass; a thread owns two adjacent columns of P
+// (their index pairs are decoded once) and writes them for every staged row, so a warp writes
+// 256 (fp32) or 128 (bf16) contiguous bytes per row.  HBM bound: the write of P.
 template <typename OutT>
 __global__ void __launch_bounds__(EXP_THREADS)
 pair_expand_kernel(const float *__restrict__ X, int64_t N, int d, int64_t ldx, OutT *__restrict__ P, int dP, int npairs)
 {
-    extern __shared__ __align__(16) unsigned char sm[];
-    unsigned short *tab = reinterpret_cast<unsigned short *>(sm);              // [dP]: i | j << 8, 0xffff = padding
-    float *xs = reinterpret_cast<float *>(sm + ((size_t)dP * 2 + 15) / 16 * 16);  // [EXP_ROWS][d]
-    for (int p = threadIdx.x; p < dP; p += EXP_THREADS) {
-        int64_t i = 0, j = 0;
-        if (p < npairs) tri_decode(d, p, i, j);
-        tab[p] = p < npairs ? (unsigned short)(i | (j << 8)) : (unsigned short)0xffff;
-    }
+    extern __shared__ __align__(16) float xs[];                       // [EXP_ROWS][d]
     const int half = dP / 2;
-    for (int64_t row0 = (int64_t)blockIdx.x * EXP_ROWS; row0 < N; row0 += (int64_t)gridDim.x * EXP_ROWS) {
+    const int cols_per_block = 2 * EXP_THREADS;
+    // gridDim.x = column groups, gridDim.y = row groups
+    const int p = blockIdx.x * cols_per_block + 2 * threadIdx.x;      // this thread's columns p, p+1
+    int i0 = 0, j0 = 0, i1 = 0, j1 = 0;
+    const bool have0 = p < npairs, have1 = p + 1 < npairs, inside = p < 2 * half;
+    if (have0) { int64_t a, b; tri_decode(d, p, a, b); i0 = (int)a; j0 = (int)b; }
+    if (have1) { int64_t a, b; tri_decode(d, p + 1, a, b); i1 = (int)a; j1 = (int)b; }
+    for (int64_t row0 = (int64_t)blockIdx.y * EXP_ROWS; row0 < N; row0 += (int64_t)gridDim.y * EXP_ROWS) {
         __syncthreads();
         for (int e = threadIdx.x; e < EXP_ROWS * d; e += EXP_THREADS) {
             const int r = e / d, c = e - r * d;
             xs[e] = row0 + r < N ? X[(row0 + r) * ldx + c] : 0.f;
         }
         __syncthreads();
-        for (int e = threadIdx.x; e < EXP_ROWS * half; e += EXP_THREADS) {
-            const int r = e / half, p = 2 * (e - r * half);
+        if (!inside) continue;
+#pragma unroll 8
+        for (int r = 0; r < EXP_ROWS; ++r) {
             if (row0 + r >= N) break;
-            const unsigned t0 = tab[p], t1 = tab[p + 1];
             const float *x = xs + r * d;
-            const float a = t0 == 0xffffu ? 0.f : x[t0 & 255u] * x[t0 >> 8];
-            const float b = t1 == 0xffffu ? 0.f : x[t1 & 255u] * x[t1 >> 8];
+            const float a = have0 ? x[i0] * x[j0] : 0.f;
+            const float b = have1 ? x[i1] * x[j1] : 0.f;
             store_pair(P, (row0 + r) * dP + p, a, b);
         }
     }
@@ -137,10 +139,11 @@ extern "C" st_status st_sym_moment4(const float *X, int64_t N, int64_t d, int64_
     unsigned char *w = (unsigned char *)ws;
     float *M2 = (float *)(w + p.off_m2);
     const int npairs = (int)tri_rows(d);
-    const size_t smem = ((size_t)p.dP * 2 + 15) / 16 * 16 + (size_t)EXP_ROWS * d * sizeof(float);
+    const size_t smem = (size_t)EXP_ROWS * d * sizeof(float);
+    const unsigned col_groups = (unsigned)((p.dP + 2 * EXP_THREADS - 1) / (2 * EXP_THREADS));
     const int64_t passes = (N + EXP_ROWS - 1) / EXP_ROWS;
-    const int64_t cap = (int64_t)sm_count_or_default() * 8;
-    const unsigned grid = (unsigned)(passes < cap ? passes : cap);
+    const int64_t cap = ((int64_t)sm_count_or_default() * 8 + col_groups - 1) / col_groups;
+    const dim3 grid(col_groups, (unsigned)(passes < cap ? passes : cap));
     if (p.bf16)
         pair_expand_kernel<__nv_bfloat16><<<grid, EXP_THREADS, smem, stream>>>(X, N, (int)d, ldx, (__nv_bfloat16 *)(w + p.off_p),
                                                                                 (int)p.dP, npairs);

@@ -214,6 +214,26 @@ slice_copy_kernel(const U *__restrict__ src, U *__restrict__ dst, LayoutArgs a, 
     }
 }
 
+// out = alpha * a + beta * b (OP 0) or out = a * b (OP 1) over packed arrays of the same layout
+template <int OP>
+__global__ void __launch_bounds__(256)
+packed_binary_kernel(const float *__restrict__ a, const float *__restrict__ b, float *__restrict__ out, int64_t n,
+                     float alpha, float beta)
+{
+    const int64_t n4 = n >> 2;
+    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    for (int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; e < n4; e += stride) {
+        const float4 x = reinterpret_cast<const float4 *>(a)[e];
+        const float4 y = reinterpret_cast<const float4 *>(b)[e];
+        float4 r;
+        if (OP == 0) r = make_float4(alpha * x.x + beta * y.x, alpha * x.y + beta * y.y, alpha * x.z + beta * y.z, alpha * x.w + beta * y.w);
+        else r = make_float4(x.x * y.x, x.y * y.y, x.z * y.z, x.w * y.w);
+        reinterpret_cast<float4 *>(out)[e] = r;
+    }
+    for (int64_t e = 4 * n4 + (int64_t)blockIdx.x * blockDim.x + threadIdx.x; e < n; e += stride)
+        out[e] = OP == 0 ? alpha * a[e] + beta * b[e] : a[e] * b[e];
+}
+
 static bool layout_ok(const st_layout *L)
 {
     if (!L) return false;
@@ -344,6 +364,29 @@ int64_t st_dense_elems(const st_layout *layout)
 st_status st_pack(const st_layout *layout, st_dtype dtype, const void *dense, void *packed, void *stream)
 {
     return st::copy_entry<true>(layout, dtype, dense, packed, ST_FILL_ZERO, stream);
+}
+
+static st_status packed_binary(int op, int64_t n, const float *a, const float *b, float *out, float alpha, float beta,
+                               void *stream)
+{
+    if (!a || !b || !out) return ST_ERR_NULL;
+    if (n <= 0) return ST_ERR_SHAPE;
+    if (!st::aligned16(a) || !st::aligned16(b) || !st::aligned16(out)) return ST_ERR_ALIGN;
+    const int64_t want = (n / 4 + 255) / 256, cap = (int64_t)st::sm_count_or_default() * 16;
+    const unsigned grid = (unsigned)(want < 1 ? 1 : (want < cap ? want : cap));
+    if (op == 0) st::packed_binary_kernel<0><<<grid, 256, 0, (cudaStream_t)stream>>>(a, b, out, n, alpha, beta);
+    else st::packed_binary_kernel<1><<<grid, 256, 0, (cudaStream_t)stream>>>(a, b, out, n, alpha, beta);
+    return st::launch_status();
+}
+
+st_status st_packed_axpby(int64_t n, float alpha, const float *a, float beta, const float *b, float *out, void *stream)
+{
+    return packed_binary(0, n, a, b, out, alpha, beta, stream);
+}
+
+st_status st_packed_mul(int64_t n, const float *a, const float *b, float *out, void *stream)
+{
+    return packed_binary(1, n, a, b, out, 0.f, 0.f, stream);
 }
 
 st_status st_thp(const st_layout *layout, const float *Bp, const float *C_dense, float *Ap, void *stream)

@@ -640,3 +640,35 @@ def test_mttkrp_on_slice_structures(st, flag_name, I, J, K, R):
         got = torch.full((I, R), float("nan"), dtype=torch.float32, device="cuda")
         st.st_mttkrp_slice(dev(Bp), dev(C), dev(D), I, fi, fj, out=got, flags=flags)
         assert oracle.rel_err(got.cpu().numpy(), A, S) <= tol, (flag_name, fi, fj)     # rows outside the slice: exactly 0
+
+
+# ------------------------------------------------------------------------------ chains in compressed space
+
+def test_chain_in_packed_space_with_one_reconstruction_at_the_end(st):
+    # covariance blocks of three batches are added up in packed space, scaled, multiplied position by
+    # position by a packed upper-triangular mask, and only then reconstructed (Section 5.5)
+    d = 24
+    batches = [workloads.draw((n, d), "normal", 1200 + n) for n in (700, 1300, 64)]
+    acc = None
+    for Xb in batches:
+        m = st.st_sym_moment2(dev(Xb))
+        acc = m if acc is None else st.st_packed_axpby(1.0, acc, 1.0, m, out=acc)
+    total = sum(b.shape[0] for b in batches)
+    acc = st.st_packed_axpby(1.0 / total, acc, 0.0, acc, out=acc)
+    W = workloads.draw((workloads.tri(d),), "uniform", 1299)
+    prod = st.st_packed_mul(acc, dev(W))
+    full = st.st_unpack(prod, st.Layout(st.ST_TRI_UPPER, d), fill=st.ST_FILL_SYMMETRIC).cpu().numpy().reshape(d, d)
+    # oracle: dense second moment of all samples, scaled, times the symmetric expansion of W
+    T, S = oracle.moment2(np.concatenate(batches))
+    Wd = oracle.unpack(W, oracle.KIND_TRI, d, fill=oracle.FILL_SYMMETRIC).astype(np.float64)
+    assert oracle.rel_err(full, T / total * Wd, S / total * np.abs(Wd)) <= 2 * TOL_F32
+    # third moments of two batches added in packed space equal the third moment of their union
+    Xa, Xb = workloads.draw((900, 16), "normal", 1251), workloads.draw((333, 16), "normal", 1252)
+    m3 = st.st_packed_axpby(1.0, st.st_sym_moment3(dev(Xa)), 1.0, st.st_sym_moment3(dev(Xb)))
+    T3, S3 = oracle.moment3(np.concatenate([Xa, Xb]))
+    assert oracle.rel_err(expand3(st, m3, 16), T3, S3) <= TOL_F32
+    # odd sizes and aliasing
+    a, b = dev(workloads.draw((1003,), "normal", 1)), dev(workloads.draw((1003,), "normal", 2))
+    want = (2.0 * a.double() - 0.5 * b.double()).float()
+    assert torch.allclose(st.st_packed_axpby(2.0, a, -0.5, b), want, rtol=1e-6, atol=1e-6)
+    assert torch.equal(st.st_packed_mul(a, b, out=a.clone()), a * b)
