@@ -26,7 +26,7 @@ namespace m4 {
 
 constexpr int MAX_D = 64;
 constexpr int EXP_ROWS = 32;        // sample rows per pass of a block
-constexpr int EXP_THREADS = 256;
+constexpr int EXP_THREADS = 192;
 
 struct Plan {
     int64_t dP, p_bytes, m2_elems, m2_ws;
@@ -53,48 +53,54 @@ static Plan plan(int64_t N, int64_t d, unsigned flags)
     return p;
 }
 
-__device__ __forceinline__ void store_pair(float *P, int64_t at, float a, float b)
+__device__ __forceinline__ void store4(float *dst, float a, float b, float c, float e)
 {
-    *reinterpret_cast<float2 *>(P + at) = make_float2(a, b);
+    *reinterpret_cast<float4 *>(dst) = make_float4(a, b, c, e);
 }
-__device__ __forceinline__ void store_pair(__nv_bfloat16 *P, int64_t at, float a, float b)
+__device__ __forceinline__ void store4(__nv_bfloat16 *dst, float a, float b, float c, float e)
 {
-    *reinterpret_cast<__nv_bfloat162 *>(P + at) = __floats2bfloat162_rn(a, b);
+    const __nv_bfloat162 lo = __floats2bfloat162_rn(a, b), hi = __floats2bfloat162_rn(c, e);
+    *reinterpret_cast<uint2 *>(dst) = make_uint2(*reinterpret_cast<const uint32_t *>(&lo), *reinterpret_cast<const uint32_t *>(&hi));
 }
 
 // P[n, p(i,j)] = X[n,i] X[n,j] for the unique pairs in packed order, zeros in the padding
-// columns.  A block stages EXP_ROWS rows of X per pass; a thread owns two adjacent columns of P
-// (their index pairs are decoded once) and writes them for every staged row, so a warp writes
-// 256 (fp32) or 128 (bf16) contiguous bytes per row.  HBM bound: the write of P.
+// columns.  A block stages EXP_ROWS rows of X per pass (one extra column holds zero); a thread owns
+// four adjacent columns of P, decodes their index pairs once and writes them for every staged
+// row with one 8- or 16-byte store.  HBM bound: the write of P.
 template <typename OutT>
 __global__ void __launch_bounds__(EXP_THREADS)
 pair_expand_kernel(const float *__restrict__ X, int64_t N, int d, int64_t ldx, OutT *__restrict__ P, int dP, int npairs)
 {
-    extern __shared__ __align__(16) float xs[];                       // [EXP_ROWS][d]
-    const int half = dP / 2;
-    const int cols_per_block = 2 * EXP_THREADS;
+    extern __shared__ __align__(16) float xs[];                       // [EXP_ROWS][d + 1], column d is zero
+    const int pitch = d + 1;
     // gridDim.x = column groups, gridDim.y = row groups
-    const int p = blockIdx.x * cols_per_block + 2 * threadIdx.x;      // this thread's columns p, p+1
-    int i0 = 0, j0 = 0, i1 = 0, j1 = 0;
-    const bool have0 = p < npairs, have1 = p + 1 < npairs, inside = p < 2 * half;
-    if (have0) { int64_t a, b; tri_decode(d, p, a, b); i0 = (int)a; j0 = (int)b; }
-    if (have1) { int64_t a, b; tri_decode(d, p + 1, a, b); i1 = (int)a; j1 = (int)b; }
+    const int p = (blockIdx.x * EXP_THREADS + threadIdx.x) * 4;       // this thread's columns p .. p+3
+    int ci[4], cj[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+        ci[u] = cj[u] = d;                                            // padding column: 0 * 0
+        if (p + u < npairs) {
+            int64_t a, b;
+            tri_decode(d, p + u, a, b);
+            ci[u] = (int)a;
+            cj[u] = (int)b;
+        }
+    }
+    const bool inside = p < dP;
     for (int64_t row0 = (int64_t)blockIdx.y * EXP_ROWS; row0 < N; row0 += (int64_t)gridDim.y * EXP_ROWS) {
+        const int nrows = N - row0 < EXP_ROWS ? (int)(N - row0) : EXP_ROWS;
         __syncthreads();
-        for (int e = threadIdx.x; e < EXP_ROWS * d; e += EXP_THREADS) {
-            const int r = e / d, c = e - r * d;
-            xs[e] = row0 + r < N ? X[(row0 + r) * ldx + c] : 0.f;
+        for (int e = threadIdx.x; e < nrows * pitch; e += EXP_THREADS) {
+            const int r = e / pitch, c = e - r * pitch;
+            xs[e] = c < d ? X[(row0 + r) * ldx + c] : 0.f;
         }
         __syncthreads();
         if (!inside) continue;
-#pragma unroll 8
-        for (int r = 0; r < EXP_ROWS; ++r) {
-            if (row0 + r >= N) break;
-            const float *x = xs + r * d;
-            const float a = have0 ? x[i0] * x[j0] : 0.f;
-            const float b = have1 ? x[i1] * x[j1] : 0.f;
-            store_pair(P, (row0 + r) * dP + p, a, b);
-        }
+        OutT *dst = P + row0 * dP + p;
+        const float *x = xs;
+#pragma unroll 4
+        for (int r = 0; r < nrows; ++r, dst += dP, x += pitch)
+            store4(dst, x[ci[0]] * x[cj[0]], x[ci[1]] * x[cj[1]], x[ci[2]] * x[cj[2]], x[ci[3]] * x[cj[3]]);
     }
 }
 
@@ -139,8 +145,8 @@ extern "C" st_status st_sym_moment4(const float *X, int64_t N, int64_t d, int64_
     unsigned char *w = (unsigned char *)ws;
     float *M2 = (float *)(w + p.off_m2);
     const int npairs = (int)tri_rows(d);
-    const size_t smem = (size_t)EXP_ROWS * d * sizeof(float);
-    const unsigned col_groups = (unsigned)((p.dP + 2 * EXP_THREADS - 1) / (2 * EXP_THREADS));
+    const size_t smem = (size_t)EXP_ROWS * (d + 1) * sizeof(float);
+    const unsigned col_groups = (unsigned)((p.dP + 4 * EXP_THREADS - 1) / (4 * EXP_THREADS));
     const int64_t passes = (N + EXP_ROWS - 1) / EXP_ROWS;
     const int64_t cap = ((int64_t)sm_count_or_default() * 8 + col_groups - 1) / col_groups;
     const dim3 grid(col_groups, (unsigned)(passes < cap ? passes : cap));
