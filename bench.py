@@ -355,6 +355,36 @@ def dense_controls(w, torch, reps=5):
     return out
 
 
+def moment2_sample_sweep(w, torch, reps=7):
+    """The small second moment (d = 64) from the named size up to 4M samples: the named size is bound by
+    launch and memory latency, the sweep shows where the kernel reaches its fp32 roofline."""
+    st = w.st
+    dev = w.ws.device
+    d = w.cfg["moment2"]["d"]
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+    out = torch.empty(tri(d), dtype=torch.float32, device=dev)
+    res = []
+    for N in (4096, 32768, 262144, 1048576, 4194304):
+        X = torch.empty((N, d), dtype=torch.float32, device=dev).uniform_(-1.0, 1.0)
+        ws = torch.empty(max(st.st_workspace_bytes(st.ST_OP_SYM_MOMENT2, N, d, st.ST_F32), 256), dtype=torch.uint8, device=dev)
+        for _ in range(2):
+            st.st_sym_moment2(X, out=out, ws=ws)
+        ts = []
+        for _ in range(reps):
+            flush.zero_()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(); st.st_sym_moment2(X, out=out, ws=ws); e1.record()
+            torch.cuda.synchronize()
+            ts.append(e0.elapsed_time(e1) * 1e3)
+        us = float(np.median(ts))
+        flops, nbytes = 2 * N * tri(d), 4 * (N * d + tri(d))
+        roof = max(flops / (FP32_PEAK_TFLOPS * 1e12), nbytes / (load_peaks()["hbm_gbs"] * 1e9)) * 1e6
+        res.append({"N": N, "us": round(us, 2), "tflops": round(flops / us / 1e6, 2), "gbs": round(nbytes / us / 1e3, 1),
+                    "roofline_us": round(roof, 2), "frac": round(roof / us, 4)})
+        del X, ws
+    return res
+
+
 def max_over_ranks(values, dist, device):
     """Element-wise maximum of a list of floats over all ranks (the slowest rank sets the time)."""
     import torch
@@ -506,6 +536,7 @@ def run_ours(args):
     }
     if world == 1 and not args.no_controls:
         line["dense_control"] = dense_controls(w, torch)
+        line["sym_moment2_sample_sweep"] = moment2_sample_sweep(w, torch)
     if rank == 0:
         if world == 1 and not args.no_cpu_baseline:
             line["cpu_baseline"] = cpu_baseline(budget_s=args.cpu_budget)
