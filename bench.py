@@ -187,7 +187,7 @@ class ClockSampler:
 
 def bench_config():
     cfg = {k: dict(v) for k, v in workloads.CONFIGS.items()}
-    cfg["band"] = dict(d=2048, kl=64, ku=63, inner=16)
+    cfg["band"] = dict(d=2048, kl=512, ku=511, inner=16)
     cfg["moment4"] = dict(N=cfg["moment3"]["N"], d=32)
     cfg["m2_large_dtype"] = "bf16"
     cfg["ttm_tc"] = True
