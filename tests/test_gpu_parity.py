@@ -672,3 +672,20 @@ def test_chain_in_packed_space_with_one_reconstruction_at_the_end(st):
     want = (2.0 * a.double() - 0.5 * b.double()).float()
     assert torch.allclose(st.st_packed_axpby(2.0, a, -0.5, b), want, rtol=1e-6, atol=1e-6)
     assert torch.equal(st.st_packed_mul(a, b, out=a.clone()), a * b)
+
+
+def test_thp_and_ttm_packed_at_the_benchmark_size(st):
+    # the packed upper-half-cube operand of the benchmark (131,328 fibres of 512) times its own dense expansion
+    Bp, _, _ = workloads.mttkrp_inputs()
+    I, K = 512, 512
+    lay = st.Layout(st.ST_TRI_UPPER, I, inner=K)
+    Bd = oracle.unpack(Bp.reshape(-1), oracle.KIND_TRI, I, inner=K)
+    got = st.st_thp(dev(Bp).view(-1), dev(Bd).view(-1), lay).cpu().numpy()
+    assert np.array_equal(got, (Bp.astype(np.float64) ** 2).astype(np.float32).reshape(-1))
+    # TTM of the same operand on sampled fibres (first, last, row starts, seeded random)
+    U = workloads.draw((K, 64), "normal", 1300)
+    A = st.st_ttm_packed(dev(Bp), dev(U), lay, flags=st.ST_FLAG_TC_TF32).cpu().numpy()
+    rng = np.random.default_rng(5)
+    rows = np.unique(np.concatenate([[0, 511, 512, Bp.shape[0] - 1], rng.integers(0, Bp.shape[0], 300)]))
+    T, S = oracle.ttm(Bp[rows], U)
+    assert oracle.rel_err(A[rows], T, S) <= 5e-3
