@@ -137,6 +137,28 @@ structured_copy_kernel(const U *__restrict__ src, U *__restrict__ dst, LayoutArg
     }
 }
 
+// Symmetric fill of a plain matrix / order-3 tensor of 4-byte elements (the reconstruction of a moment
+// output): one thread per dense element, indices from the thread coordinates, 32-bit arithmetic only.
+template <int KIND>
+__global__ void __launch_bounds__(256)
+sym_unpack32_kernel(const uint32_t *__restrict__ packed, uint32_t *__restrict__ dense, unsigned d)
+{
+    const unsigned x = blockIdx.x * blockDim.x + threadIdx.x, y = blockIdx.y * blockDim.y + threadIdx.y;
+    if (x >= d || y >= d) return;
+    if (KIND == ST_TRI_UPPER) {
+        const unsigned i = y < x ? y : x, j = y < x ? x : y;             // representative (min, max): T_R of the symmetric structure
+        dense[y * d + x] = packed[i * (2 * d - i + 1) / 2 + (j - i)];
+    } else {
+        unsigned a = blockIdx.z, b = y, c = x, t;                        // dense (i, j, k) = (z, y, x); sort to a <= b <= c
+        if (a > b) { t = a; a = b; b = t; }
+        if (b > c) { t = b; b = c; c = t; }
+        if (a > b) { t = a; a = b; b = t; }
+        const unsigned m = d - a, jj = b - a, kk = c - a;
+        const unsigned slab = d * (d + 1) / 2 * (d + 2) / 3 - m * (m + 1) / 2 * (m + 2) / 3;
+        dense[(blockIdx.z * d + y) * d + x] = packed[slab + jj * (2 * m - jj + 1) / 2 + (kk - jj)];
+    }
+}
+
 // Run of unique columns of slice s, in rows of `chunks` units: dense columns [lo,hi) of the
 // slice map to packed rows prow.. (contiguous).  For ST_BAND also the extent of the fixed-width
 // packed row [band0, band1) whose slots outside the run are zero-filled by pack.
@@ -278,6 +300,12 @@ template <int KIND, typename U, bool PACK>
 static st_status launch_copy(const void *src, void *dst, const LayoutArgs &a, cudaStream_t s, const void *mul)
 {
     const int64_t cap = (int64_t)sm_count_or_default() * 16;
+    if (!PACK && a.fill == ST_FILL_SYMMETRIC && sizeof(U) == 4 && a.chunks == 1 &&
+        ((KIND == ST_TRI_UPPER && a.d <= 32768) || (KIND == ST_TET && a.d <= 1024))) {
+        const dim3 block(32, 8), grid((unsigned)((a.d + 31) / 32), (unsigned)((a.d + 7) / 8), KIND == ST_TET ? (unsigned)a.d : 1u);
+        sym_unpack32_kernel<(KIND == ST_TET ? ST_TET : ST_TRI_UPPER)><<<grid, block, 0, s>>>((const uint32_t *)src, (uint32_t *)dst, (unsigned)a.d);
+        return launch_status();
+    }
     if (!PACK && a.fill == ST_FILL_SYMMETRIC) {
         // redundancy map: one lane group per dense row
         int shift = 0;

@@ -136,6 +136,18 @@ def test_pack_unpack_at_config_sizes(st):
     assert torch.equal(st.st_pack(dense_t.view(-1), lay), Pt)
 
 
+def test_pack_unpack_blockdiag_midsize(st):
+    # 16 blocks of 64 x 64 fibres of 64 floats: 16.8 MB packed, 268 MB dense (larger than L2); full comparison
+    lay = st.Layout(st.ST_BLOCKDIAG, 1024, inner=64, nblocks=16, bs=64)
+    n = st.st_packed_elems(lay)
+    P = np.random.default_rng(3).integers(0, 2 ** 32, size=n, dtype=np.uint32)
+    Pt = torch.from_numpy(P.view(np.int32)).cuda()
+    dense = st.st_unpack(Pt, lay)
+    want = oracle.unpack(P, oracle.KIND_BLOCKDIAG, 1024, inner=64, nb=16, bs=64).reshape(-1)
+    assert np.array_equal(dense.cpu().numpy().view(np.uint32), want)
+    assert torch.equal(st.st_pack(dense, lay), Pt)
+
+
 # ------------------------------------------------------------------------------ moments
 
 def expand2(st, packed, d):
