@@ -594,7 +594,7 @@ st_status moment2_bf16_tc(const void *X, int64_t N, int64_t d, int64_t ldx, floa
             (void)cudaGetLastError();
             return ST_ERR_CUDA;
         }
-        moment2_tc_pair_reduce_kernel<<<dim3(q.tab.ntiles, 16), 256, 0, stream>>>(part2, out, (int)d, q.tab);
+        moment2_tc_pair_reduce_kernel<<<dim3(q.tab.ntiles, 64), 256, 0, stream>>>(part2, out, (int)d, q.tab);
         return launch_status();
     }
     const M2TcPlan p = m2tc_plan(N, d, flags);
@@ -611,7 +611,7 @@ st_status moment2_bf16_tc(const void *X, int64_t N, int64_t d, int64_t ldx, floa
     moment2_tc_kernel<<<p.tab.nblocks, THREADS, SMEM_BYTES, stream>>>(tmap, partials, (unsigned *)ws, p.chunks_total,
                                                                       p.tab);
     if (cudaGetLastError() != cudaSuccess) return ST_ERR_CUDA;
-    moment2_tc_reduce_kernel<<<dim3(p.tab.ntiles, 8), 256, 0, stream>>>(partials, out, (int)d, p.tab);
+    moment2_tc_reduce_kernel<<<dim3(p.tab.ntiles, 32), 256, 0, stream>>>(partials, out, (int)d, p.tab);
     return launch_status();
 }
 
