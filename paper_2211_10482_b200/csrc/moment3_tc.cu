@@ -1,12 +1,12 @@
-// st_sym_moment3, tensor-core path (ST_FLAG_TC_TF32):
+// st_sym_moment3, tensor-core path (ST_FLAG_TC_TF32 / ST_FLAG_TC_BF16):
 //     out[q(i,j,k)] = sum_n X[n,i] X[n,j] X[n,k]   for 0 <= i <= j <= k < d
 // (Section 3, M2 = f (x) vec(f (x) f) summed over samples; unique elements i<=j<=k, Section 2
 // "Tensor Structures").  With the pair product hoisted out of the k loop (loop-invariant code
 // motion, Section 5.5) the sum is a contraction over the samples,
 //     out[(i,j), k] = sum_n P[n,(i,j)] X[n,k],      P[n,(i,j)] = X[n,i] X[n,j]   (i <= j),
 // that is a GEMM [pairs x samples] x [samples x d] whose left operand exists nowhere in memory.
-// This kernel makes P on the fly.  A loader warp writes slices of 32 samples of X^T, rounded to
-// TF32, into shared memory in the K-major 128-byte-swizzled form the tensor core reads (lane =
+// This kernel makes P on the fly.  A loader warp writes slices of 32 (TF32) or 64 (bf16) samples of X^T,
+// rounded, into shared memory in the K-major 128-byte-swizzled form the tensor core reads (lane =
 // sample).  Producer warps read their lane's x_i and x_j back from that slice, multiply the
 // pairs of one tile (8 values of i x 16 values of j) and store the products, rounded to TF32, in
 // the same form as the left operand of the tile's MMA.  A tile with j >= 16*JB needs the
@@ -15,8 +15,11 @@
 // Accumulators of all tiles of a block stay in tensor memory for the block's whole sample
 // range; at d = 64 they need 640 columns, so two blocks ("groups") share one sample range.
 //
-// Bound by the shared-memory stores of P (one 4-byte store per pair and sample), not by the
-// tensor pipe.  TF32 products, fp32 accumulation: 5e-3 tolerance.
+// What bounds it: an MMA of M = 128 takes about 49 ns whatever N <= 128 is, and N <= d <= 64 here, so the
+// time goes with the number of MMAs (4 per tile and slice) and with the shared-memory traffic around them
+// (P is stored once and read once by the tensor core), not with the tensor arithmetic.  bf16 halves both
+// (64 samples per slice instead of 32).  Products and x_k rounded to TF32 / bf16, fp32 accumulation: 5e-3
+// tolerance (bf16: for N >= 1000).
 #include "tc_common.cuh"
 #include "st_index.cuh"
 
