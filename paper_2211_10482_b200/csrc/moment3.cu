@@ -73,10 +73,14 @@ __device__ __forceinline__ uint64_t ffma2(uint64_t a, uint64_t b, uint64_t c)
 }
 
 // One stage of rows for one tile.  acc[a][c] holds the sums for j = a, k = 2c and 2c+1.
-template <int J0, bool DIAG>
-__device__ __forceinline__ void m3_stage(const float *__restrict__ xs, int d, int pi, int oj, int ok, int half,
+// DC > 0: the row length is the compile-time constant DC, so that every shared-memory address of
+// the loop is "row base + immediate" (integer multiply-adds share the FMA pipe: with run-time strides
+// the kernel was 9 % slower at d = 64).
+template <int J0, bool DIAG, int DC>
+__device__ __forceinline__ void m3_stage(const float *__restrict__ xs, int d_, int pi, int oj, int ok, int half_,
                                          uint64_t (&acc)[8][4])
 {
+    const int d = DC > 0 ? DC : d_, half = DC > 0 ? DC / 2 : half_;
 #pragma unroll 2
     for (int r = 0; r < M3_STAGE_ROWS; ++r) {
         const float *row = xs + r * d;
@@ -103,7 +107,7 @@ __device__ __forceinline__ void m3_stage(const float *__restrict__ xs, int d, in
     }
 }
 
-template <int WARPS>
+template <int WARPS, int DC>
 __global__ void __launch_bounds__(M3_THREADS, 1)
 moment3_kernel(const float *__restrict__ X, int64_t N, int d, int64_t ldx, float *__restrict__ partials,
                int64_t rows_per_slice, int out_elems, const __grid_constant__ M3Table<WARPS> tab)
@@ -163,15 +167,15 @@ moment3_kernel(const float *__restrict__ X, int64_t N, int d, int64_t ldx, float
             cp_async_commit();
         const float *xs = smem + (int)(s % M3_BUFFERS) * stage_floats;
         switch (variant) {
-        case 0: m3_stage<0, false>(xs, d, pi, oj, ok, half, acc); break;
-        case 1: m3_stage<0, true>(xs, d, pi, oj, ok, half, acc); break;
-        case 2: m3_stage<1, false>(xs, d, pi, oj, ok, half, acc); break;
-        case 3: m3_stage<2, false>(xs, d, pi, oj, ok, half, acc); break;
-        case 4: m3_stage<3, false>(xs, d, pi, oj, ok, half, acc); break;
-        case 5: m3_stage<4, false>(xs, d, pi, oj, ok, half, acc); break;
-        case 6: m3_stage<5, false>(xs, d, pi, oj, ok, half, acc); break;
-        case 7: m3_stage<6, false>(xs, d, pi, oj, ok, half, acc); break;
-        case 8: m3_stage<7, false>(xs, d, pi, oj, ok, half, acc); break;
+        case 0: m3_stage<0, false, DC>(xs, d, pi, oj, ok, half, acc); break;
+        case 1: m3_stage<0, true, DC>(xs, d, pi, oj, ok, half, acc); break;
+        case 2: m3_stage<1, false, DC>(xs, d, pi, oj, ok, half, acc); break;
+        case 3: m3_stage<2, false, DC>(xs, d, pi, oj, ok, half, acc); break;
+        case 4: m3_stage<3, false, DC>(xs, d, pi, oj, ok, half, acc); break;
+        case 5: m3_stage<4, false, DC>(xs, d, pi, oj, ok, half, acc); break;
+        case 6: m3_stage<5, false, DC>(xs, d, pi, oj, ok, half, acc); break;
+        case 7: m3_stage<6, false, DC>(xs, d, pi, oj, ok, half, acc); break;
+        case 8: m3_stage<7, false, DC>(xs, d, pi, oj, ok, half, acc); break;
         default: break;
         }
     }
@@ -391,10 +395,16 @@ static st_status moment3_launch(const float *X, int64_t N, int64_t d, int64_t ld
     if (!aligned256(ws)) return ST_ERR_ALIGN;
     float *partials = (float *)((unsigned char *)ws + kWsHeaderBytes);
     const size_t smem = (size_t)M3_BUFFERS * M3_STAGE_ROWS * d * sizeof(float);
-    if (!ensure_dynamic_smem(moment3_kernel<WARPS>, smem)) return ST_ERR_CUDA;
     dim3 grid(p.groups, p.slices);
-    moment3_kernel<WARPS><<<grid, M3_THREADS, smem, stream>>>(X, N, (int)d, ldx, partials, p.rows_per_slice,
-                                                              (int)p.out_elems, local);
+    if (d == M3_MAX_D) {      // the largest side has its own instance with compile-time strides
+        if (!ensure_dynamic_smem(moment3_kernel<WARPS, M3_MAX_D>, smem)) return ST_ERR_CUDA;
+        moment3_kernel<WARPS, M3_MAX_D><<<grid, M3_THREADS, smem, stream>>>(X, N, (int)d, ldx, partials, p.rows_per_slice,
+                                                                           (int)p.out_elems, local);
+    } else {
+        if (!ensure_dynamic_smem(moment3_kernel<WARPS, 0>, smem)) return ST_ERR_CUDA;
+        moment3_kernel<WARPS, 0><<<grid, M3_THREADS, smem, stream>>>(X, N, (int)d, ldx, partials, p.rows_per_slice,
+                                                                    (int)p.out_elems, local);
+    }
     if (cudaGetLastError() != cudaSuccess) return ST_ERR_CUDA;
     return sum_slices_launch(partials, out, p.out_elems, p.slices, stream);
 }
