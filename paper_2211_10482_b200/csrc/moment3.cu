@@ -180,6 +180,7 @@ moment3_kernel(const float *__restrict__ X, int64_t N, int d, int64_t ldx, float
         }
     }
     cp_async_wait<0>();
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // the slice sums may be launched; they wait for this grid to end
 
     if (!valid || variant == 255) return;
     float *mine = partials + (size_t)blockIdx.y * out_elems;
@@ -207,6 +208,9 @@ __global__ void __launch_bounds__(32 * SUM_GROUPS)
 sum_slices_kernel(const float *__restrict__ partials, float *__restrict__ out, int64_t elems, int slices)
 {
     __shared__ float part[SUM_GROUPS][32];
+    // launched as a programmatic dependent of the kernel that writes the partial sums: the launch itself
+    // overlaps that kernel's tail, and nothing is read before that kernel has completed
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     const int lane = threadIdx.x & 31, g = threadIdx.x >> 5;
     const int64_t e = (int64_t)blockIdx.x * 32 + lane;
     float s = 0.f;
@@ -235,8 +239,21 @@ sum_slices_kernel(const float *__restrict__ partials, float *__restrict__ out, i
 
 st_status sum_slices_launch(const float *partials, float *out, int64_t elems, int slices, cudaStream_t stream)
 {
-    sum_slices_kernel<<<(unsigned)((elems + 31) / 32), 32 * SUM_GROUPS, 0, stream>>>(partials, out, elems, slices);
-    return launch_status();
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)((elems + 31) / 32));
+    cfg.blockDim = dim3(32 * SUM_GROUPS);
+    cfg.dynamicSmemBytes = 0;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    if (cudaLaunchKernelEx(&cfg, sum_slices_kernel, partials, out, elems, slices) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return ST_ERR_CUDA;
+    }
+    return ST_OK;
 }
 
 // ---- host side: tile table ------------------------------------------------------------

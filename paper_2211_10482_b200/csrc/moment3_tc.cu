@@ -204,6 +204,7 @@ moment3_tc_kernel(const __grid_constant__ Args a)
             if (lane == 0) mbar_arrive(&a_full[as]);
         }
 
+        asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // the slice sums may be launched; they wait for this grid to end
         // ---- epilogue: tensor memory -> this slice's partial sums ---------------------------------
         if (nstages > 0 && mbar_wait(acc_full, 0u, abort_flag, a.status, 13)) {
             tc_fence_after();
