@@ -34,11 +34,11 @@ constexpr int BM = TI * TJ;                  // 128 pairs = rows of the MMA
 constexpr int ROW_BYTES = 128;               // one swizzled row: 32 TF32 or 64 bf16 samples
 constexpr int A_STAGE_BYTES = BM * ROW_BYTES; // 16 KiB
 constexpr int B_STAGE_BYTES = DP * ROW_BYTES; // 8 KiB
-constexpr int NA_MAX = 10;                   // A stages in flight (TF32: 10, bf16: 8)
+constexpr int NA_MAX = 10;                   // A stages in flight (TF32: 10, bf16: 8; even: see the issuers)
 constexpr int NB = 4;                        // X^T slices in flight
 constexpr int X32_STAGE_BYTES = DP * 64 * 4; // bf16 path: fp32 copy of a slice of X^T for the producers (16 KiB)
 constexpr int PRODUCERS = 8;                 // producer warps (also the epilogue warps)
-constexpr int MMA_WARPS = 1;                 // one issuer: stages are consumed in the order they are produced
+constexpr int MMA_WARPS = 2;                 // issuer w takes the stages q = w (mod 2): while one polls, the other's MMAs run
 constexpr int MMA_WARP = PRODUCERS, LOAD_WARP = PRODUCERS + MMA_WARPS;
 constexpr int LOAD_WARPS = 1;                // one loader: slices are filled in order
 constexpr int THREADS = 32 * (PRODUCERS + MMA_WARPS + LOAD_WARPS);
@@ -96,7 +96,8 @@ moment3_tc_kernel(const __grid_constant__ Args a)
     uint64_t *bars = (uint64_t *)(x32_stage0 + (BF16 ? (size_t)NB * X32_STAGE_BYTES : 0));
     uint64_t *a_full = bars, *a_empty = bars + NA_MAX, *b_full = bars + 2 * NA_MAX, *b_empty = bars + 2 * NA_MAX + NB,
              *acc_full = bars + 2 * NA_MAX + 2 * NB;
-    uint32_t *tmem_slot = (uint32_t *)(acc_full + 1);
+    uint64_t *iss_sync = acc_full + 1;
+    uint32_t *tmem_slot = (uint32_t *)(acc_full + 2);
     volatile int *abort_flag = (volatile int *)(tmem_slot + 1);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -114,6 +115,7 @@ moment3_tc_kernel(const __grid_constant__ Args a)
             mbar_init(&b_empty[s], MMA_WARPS);
         }
         mbar_init(acc_full, MMA_WARPS);
+        mbar_init(iss_sync, MMA_WARPS);
         *abort_flag = 0;
         if (blockIdx.x == 0 && blockIdx.y == 0) {
             a.status[kWsStatusWord] = 0;
@@ -265,15 +267,21 @@ moment3_tc_kernel(const __grid_constant__ Args a)
             }
         }
     } else if (warp < LOAD_WARP) {
-        // ---- MMA issuer --------------------------------------------------------------------------
+        // ---- MMA issuers: two warps.  A barrier poll issued behind tcgen05.mma instructions of the same thread
+        // returns only as they drain, so one issuer alone leaves the tensor pipe idle while it polls.
+        // A ring slot q % NA has the parity of q (NA is even), so every slot has one issuer and its uses are polled in
+        // order.  The MMAs of slice 0 overwrite the accumulators: both issuers wait until all of them are complete
+        // before either adds slice 1, after which the order of the additions into a tile is free.
+        const int iw = warp - MMA_WARP;
         if (elect_one()) {
             bool ok = true;
-            int64_t q = 0;
             for (int slice = 0; slice < nslices && ok; ++slice) {
                 const int bs = slice % NB;
                 if (!mbar_wait(&b_full[bs], (uint32_t)((slice / NB) & 1), abort_flag, a.status, 14)) break;
                 const uint32_t sb = smem_u32(b_stage0 + (size_t)bs * B_STAGE_BYTES);
-                for (int ti = 0; ti < tg; ++ti, ++q) {
+                for (int ti = 0; ti < tg; ++ti) {
+                    const int64_t q = (int64_t)slice * tg + ti;
+                    if ((int)(q & 1) != iw) continue;
                     const Tile t = tiles[ti];
                     const int kstart = TJ * t.jb, ncols = a.dcols - kstart;
                     const int as = (int)(q % NA);
@@ -293,9 +301,15 @@ moment3_tc_kernel(const __grid_constant__ Args a)
                     }
                     tc_commit(&a_empty[as]);
                 }
-                if (ok) tc_commit(&b_empty[bs]);
+                if (!ok) break;
+                tc_commit(&b_empty[bs]);
+                if (slice == 0 && nslices > 1) {
+                    tc_commit(iss_sync);
+                    if (!mbar_wait(iss_sync, 0u, abort_flag, a.status, 17)) break;
+                    tc_fence_after();
+                }
+                if (slice == nslices - 1) tc_commit(acc_full);
             }
-            if (ok) tc_commit(acc_full);
         }
     } else {
         // ---- loader: slices of X^T (row = column c of X), rounded to TF32 or bf16.  A lane owns one
