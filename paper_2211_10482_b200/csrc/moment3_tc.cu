@@ -16,8 +16,9 @@
 // range; at d = 64 they need 640 columns, so two blocks ("groups") share one sample range.
 //
 // What bounds it: an MMA of M = 128 takes about 49 ns whatever N <= 128 is, and N <= d <= 64 here, so the
-// time goes with the number of MMAs (4 per tile and slice) and with the shared-memory traffic around them
-// (P is stored once and read once by the tensor core), not with the tensor arithmetic.  bf16 halves both
+// time goes with the number of MMAs (4 per tile and slice) and with what the issuing threads do between them
+// (a barrier poll behind tcgen05.mma instructions of the same thread returns only as they drain: two issuer
+// warps take alternate stages), not with the tensor arithmetic.  bf16 halves the number of MMAs
 // (64 samples per slice instead of 32).  Products and x_k rounded to TF32 / bf16, fp32 accumulation: 5e-3
 // tolerance (bf16: for N >= 1000).
 #include "tc_common.cuh"
