@@ -270,6 +270,44 @@ def test_ttm_keeps_block_diagonal_structure():
                 assert np.all(A1[i, j] == 0)
 
 
+def test_thp_brute_force_and_closed_forms():
+    """THP of Table 1: A(i,j,k) = B(i,j,k) * C(i,j,k).  Pinned by a pure-Python triple loop on a tensor
+    with three different extents, by B = 1 (the product is C itself), and by a B that is non-zero on
+    the diagonal plane i = j only (the unique set of a product is the intersection of the operands'
+    unique sets, Section 5.1: the result is zero off the plane and b_i * C(i,i,k) on it)."""
+    I, J, K = 3, 4, 5
+    B, C = rnd((I, J, K), 21), rnd((I, J, K), 22, "uniform")
+    A, S = oracle.thp(B, C)
+    assert A.dtype == np.float64 and A.shape == (I, J, K)
+    for i in range(I):
+        for j in range(J):
+            for k in range(K):
+                want = float(B[i, j, k]) * float(C[i, j, k])      # exact in fp64: two 24-bit significands
+                assert A[i, j, k] == want and S[i, j, k] == abs(want)
+    # the operands are not interchangeable with their transposes: a reshaped or transposed C fails this
+    assert not np.array_equal(A, oracle.thp(B, np.ascontiguousarray(C.transpose(0, 2, 1)).reshape(I, J, K))[0])
+    A1, _ = oracle.thp(np.ones((I, J, K), np.float32), C)
+    assert np.array_equal(A1, C.astype(np.float64))
+    d = 4
+    b = rnd((d,), 23)
+    Bd = np.zeros((d, d, K), np.float32)
+    for i in range(d):
+        Bd[i, i, :] = b[i]
+    Cd = rnd((d, d, K), 24)
+    Ad, Sd = oracle.thp(Bd, Cd)
+    for i in range(d):
+        for j in range(d):
+            if i == j:
+                assert np.array_equal(Ad[i, i], np.float64(b[i]) * Cd[i, i].astype(np.float64))
+            else:
+                assert np.all(Ad[i, j] == 0) and np.all(Sd[i, j] == 0)
+    # widening happens before the product: the fp64 product of two fp32 numbers is not the fp32 one
+    x = np.array([[[1.0 + 2.0 ** -23]]], np.float32)
+    assert oracle.thp(x, x)[0][0, 0, 0] == (1.0 + 2.0 ** -23) ** 2 != float(np.float32(x[0, 0, 0] * x[0, 0, 0]))
+    with pytest.raises(AssertionError):
+        oracle.thp(B, C[:, :, :4])
+
+
 # --------------------------------------------------------------------------- layouts
 
 def test_unique_set_counts_closed_forms():
