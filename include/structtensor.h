@@ -121,7 +121,7 @@ size_t st_workspace_bytes(st_op op, int64_t a, int64_t b, int64_t c, int64_t e, 
  * summed over samples; Section 5.5, "Vector Self-Outer-Product": y_U = 0<=i<=j<n):
  *     out[p(i,j)] = sum_n X[n,i] * X[n,j]      for 0 <= i <= j < d
  * X: [N, ldx] with ldx >= d, dtype ST_F32 (fp32 FMA path, any d) or ST_BF16 (tensor-core
- * path: bf16 products, fp32 accumulation; needs d % 64 == 0, ldx % 8 == 0).
+ * path: bf16 products, fp32 accumulation; needs d % 8 == 0, ldx % 8 == 0).
  * out_packed: d(d+1)/2 floats in ST_TRI_UPPER order.
  * ST_FLAG_DENSE_CONTROL: all d*d products are computed (lower-triangle tiles too) and
  * the lower results discarded; the output is the same. */
@@ -220,7 +220,8 @@ st_status st_mttkrp_slice(const float *Bp, int64_t I, int64_t J, int64_t K, int6
  * The output keeps the structure of the input (A_U(i,j,r) = B_U(i,j,.)).
  * Bp: packed [nblocks*bs*bs, K] fp32; U: [K,R] fp32; Ap: packed [nblocks*bs*bs, R] fp32.
  * Needs K % 4 == 0 and R % 4 == 0.  ST_FLAG_TC_TF32 selects the tensor-core path
- * (operands truncated to TF32, fp32 accumulation; needs K % 32 == 0, R % 16 == 0, R <= 256).
+ * (Bp truncated and U rounded to TF32, fp32 accumulation; 5e-3 tolerance; needs K % 4 == 0,
+ * R % 16 == 0, R <= 256).
  * ST_FLAG_DENSE_CONTROL: Bp is a dense [d,d,K] tensor and Ap a dense [d,d,R] one,
  * d = nblocks*bs; all d*d fibres are multiplied. */
 st_status st_ttm_blockdiag(const float *Bp, int64_t nblocks, int64_t bs, int64_t K,

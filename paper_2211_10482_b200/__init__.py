@@ -160,11 +160,33 @@ def st_workspace_bytes(op: int, a: int, b: int, c: int = 0, e: int = 0, flags: i
     return int(lib().st_workspace_bytes(op, a, b, c, e, flags))
 
 
+_allocator = None          # callable (numel, dtype, device) -> tensor, or None for torch.empty
+_last_ws: dict = {}        # device index -> the workspace of the most recent compute call on that device
+
+
+def set_allocator(fn) -> None:
+    """Device memory for the outputs and workspaces that a caller does not pass comes from
+    ``fn(numel, dtype, device)`` (a 1-d tensor whose data pointer is 256-byte aligned); ``None``
+    restores ``torch.empty``.  For callers that manage their own pool, and for tests that
+    surround every buffer with guard bands."""
+    global _allocator
+    _allocator = fn
+
+
+def _alloc(numel: int, dtype, device) -> torch.Tensor:
+    if _allocator is not None:
+        return _allocator(int(numel), dtype, device)
+    return torch.empty(int(numel), dtype=dtype, device=device)
+
+
 def _workspace(query, device, ws: torch.Tensor | None) -> torch.Tensor:
-    """The caller's workspace, or a fresh one of the size that `query()` reports."""
-    if ws is not None:
-        return ws
-    return torch.empty(max(int(query()), 256), dtype=torch.uint8, device=device)
+    """The caller's workspace, or a fresh one of the size that `query()` reports.  Either way it is
+    remembered as the device's last workspace, so that st_check_status() can read the status word
+    that the call's kernels may have written."""
+    if ws is None:
+        ws = _alloc(max(int(query()), 256), torch.uint8, device)
+    _last_ws[ws.device.index] = ws
+    return ws
 
 
 def st_pack(dense: torch.Tensor, layout: Layout, out: torch.Tensor | None = None) -> torch.Tensor:
@@ -174,7 +196,7 @@ def st_pack(dense: torch.Tensor, layout: Layout, out: torch.Tensor | None = None
     if dense.numel() != st_dense_elems(layout):
         raise ValueError("dense has %d elements, layout needs %d" % (dense.numel(), st_dense_elems(layout)))
     if out is None:
-        out = torch.empty(n, dtype=dense.dtype, device=dense.device)
+        out = _alloc(n, dense.dtype, dense.device)
     _check(lib().st_pack(ctypes.byref(layout.c()), _dtype(dense), _dev(dense, "dense"), _dev(out, "out"),
                          _stream()), "st_pack")
     return out
@@ -188,7 +210,7 @@ def st_unpack(packed: torch.Tensor, layout: Layout, fill: int = ST_FILL_ZERO,
     if packed.numel() != st_packed_elems(layout):
         raise ValueError("packed has %d elements, layout needs %d" % (packed.numel(), st_packed_elems(layout)))
     if out is None:
-        out = torch.empty(n, dtype=packed.dtype, device=packed.device)
+        out = _alloc(n, packed.dtype, packed.device)
     _check(lib().st_unpack(ctypes.byref(layout.c()), _dtype(packed), _dev(packed, "packed"), _dev(out, "out"),
                            int(fill), _stream()), "st_unpack")
     return out
@@ -198,9 +220,11 @@ def st_sym_moment2(X: torch.Tensor, out: torch.Tensor | None = None, ws: torch.T
                    flags: int = 0) -> torch.Tensor:
     """Packed upper triangle of X^T X; X is [N, d] float32 or bfloat16."""
     N, d = X.shape
-    xdt = _dtype(X)
+    if X.dtype not in (torch.float32, torch.bfloat16):
+        raise TypeError("X must be float32 or bfloat16")
+    xdt = _DTYPES[X.dtype]
     if out is None:
-        out = torch.empty(d * (d + 1) // 2, dtype=torch.float32, device=X.device)
+        out = _alloc(d * (d + 1) // 2, torch.float32, X.device)
     ws = _workspace(lambda: st_workspace_bytes(ST_OP_SYM_MOMENT2, N, d, xdt, 0, flags), X.device, ws)
     _check(lib().st_sym_moment2(_dev(X, "X"), xdt, N, d, X.stride(0), _dev(out, "out"), ws.data_ptr(),
                                 ws.numel() * ws.element_size(), flags, _stream()), "st_sym_moment2")
@@ -214,7 +238,7 @@ def st_sym_moment3(X: torch.Tensor, out: torch.Tensor | None = None, ws: torch.T
     if X.dtype != torch.float32:
         raise TypeError("X must be float32")
     if out is None:
-        out = torch.empty(d * (d + 1) * (d + 2) // 6, dtype=torch.float32, device=X.device)
+        out = _alloc(d * (d + 1) * (d + 2) // 6, torch.float32, X.device)
     ws = _workspace(lambda: st_workspace_bytes(ST_OP_SYM_MOMENT3, N, d, 0, 0, flags), X.device, ws)
     _check(lib().st_sym_moment3(_dev(X, "X"), N, d, X.stride(0), _dev(out, "out"), ws.data_ptr(),
                                 ws.numel() * ws.element_size(), flags, _stream()), "st_sym_moment3")
@@ -228,7 +252,7 @@ def st_sym_moment4(X: torch.Tensor, out: torch.Tensor | None = None, ws: torch.T
     if X.dtype != torch.float32:
         raise TypeError("X must be float32")
     if out is None:
-        out = torch.empty(d * (d + 1) * (d + 2) * (d + 3) // 24, dtype=torch.float32, device=X.device)
+        out = _alloc(d * (d + 1) * (d + 2) * (d + 3) // 24, torch.float32, X.device)
     ws = _workspace(lambda: st_workspace_bytes(ST_OP_SYM_MOMENT4, N, d, 0, 0, flags), X.device, ws)
     _check(lib().st_sym_moment4(_dev(X, "X"), N, d, X.stride(0), _dev(out, "out"), ws.data_ptr(),
                                 ws.numel() * ws.element_size(), flags, _stream()), "st_sym_moment4")
@@ -262,7 +286,7 @@ def st_mttkrp_tri(Bp: torch.Tensor, C: torch.Tensor, D: torch.Tensor, out: torch
     if Bp.numel() != want or D.shape[1] != R:
         raise ValueError("shape mismatch")
     if out is None:
-        out = torch.empty((I, R), dtype=torch.float32, device=Bp.device)
+        out = _alloc(I * R, torch.float32, Bp.device).view(I, R)
     ws = _workspace(lambda: st_workspace_bytes(ST_OP_MTTKRP_TRI, I, K, R, 0, flags), Bp.device, ws)
     _check(lib().st_mttkrp_tri(_dev(Bp, "Bp"), I, K, _dev(C, "C"), _dev(D, "D"), R, _dev(out, "out"),
                                ws.data_ptr(), ws.numel() * ws.element_size(), flags, _stream()),
@@ -282,7 +306,7 @@ def st_mttkrp_slice(Bp: torch.Tensor, C: torch.Tensor, D: torch.Tensor, I: int, 
     if Bp.numel() != rows * K or D.shape[1] != R:
         raise ValueError("shape mismatch")
     if out is None:
-        out = torch.empty((I, R), dtype=torch.float32, device=Bp.device)
+        out = _alloc(I * R, torch.float32, Bp.device).view(I, R)
     ws = _workspace(lambda: st_workspace_bytes(ST_OP_MTTKRP_TRI, I, K, R, 0, flags), Bp.device, ws)
     _check(lib().st_mttkrp_slice(_dev(Bp, "Bp"), I, J, K, fixed_i, fixed_j, _dev(C, "C"), _dev(D, "D"), R,
                                  _dev(out, "out"), ws.data_ptr(), ws.numel() * ws.element_size(), flags, _stream()),
@@ -302,7 +326,7 @@ def st_ttm_blockdiag(Bp: torch.Tensor, U: torch.Tensor, nblocks: int, bs: int,
     if Bp.numel() != rows * K:
         raise ValueError("shape mismatch")
     if out is None:
-        out = torch.empty((rows, R), dtype=torch.float32, device=Bp.device)
+        out = _alloc(rows * R, torch.float32, Bp.device).view(rows, R)
     ws = _workspace(lambda: st_workspace_bytes(ST_OP_TTM_BLOCKDIAG, nblocks, bs, K, R, flags), Bp.device, ws)
     _check(lib().st_ttm_blockdiag(_dev(Bp, "Bp"), nblocks, bs, K, _dev(U, "U"), R, _dev(out, "out"),
                                   ws.data_ptr(), ws.numel() * ws.element_size(), flags, _stream()),
@@ -320,7 +344,7 @@ def st_ttm_packed(Bp: torch.Tensor, U: torch.Tensor, layout: Layout, out: torch.
         raise ValueError("shape mismatch")
     rows = Bp.numel() // K
     if out is None:
-        out = torch.empty((rows, R), dtype=torch.float32, device=Bp.device)
+        out = _alloc(rows * R, torch.float32, Bp.device).view(rows, R)
     ws = _workspace(lambda: st_workspace_bytes(ST_OP_TTM_BLOCKDIAG, rows, 1, K, R, flags), Bp.device, ws)
     _check(lib().st_ttm_packed(ctypes.byref(layout.c()), _dev(Bp, "Bp"), _dev(U, "U"), R, _dev(out, "out"),
                                ws.data_ptr(), ws.numel() * ws.element_size(), flags, _stream()), "st_ttm_packed")
@@ -334,7 +358,7 @@ def st_thp(Bp: torch.Tensor, C: torch.Tensor, layout: Layout, out: torch.Tensor 
     if Bp.numel() != st_packed_elems(layout) or C.numel() != st_dense_elems(layout):
         raise ValueError("shape mismatch")
     if out is None:
-        out = torch.empty_like(Bp)
+        out = _alloc(Bp.numel(), torch.float32, Bp.device).view(Bp.shape)
     _check(lib().st_thp(ctypes.byref(layout.c()), _dev(Bp, "Bp"), _dev(C, "C"), _dev(out, "out"), _stream()), "st_thp")
     return out
 
@@ -345,7 +369,7 @@ def st_packed_axpby(alpha: float, a: torch.Tensor, beta: float, b: torch.Tensor,
     if a.dtype != torch.float32 or b.dtype != torch.float32 or a.numel() != b.numel():
         raise ValueError("two float32 arrays of the same size are needed")
     if out is None:
-        out = torch.empty_like(a)
+        out = _alloc(a.numel(), torch.float32, a.device).view(a.shape)
     _check(lib().st_packed_axpby(a.numel(), alpha, _dev(a, "a"), beta, _dev(b, "b"), _dev(out, "out"), _stream()),
            "st_packed_axpby")
     return out
@@ -356,10 +380,14 @@ def st_packed_mul(a: torch.Tensor, b: torch.Tensor, out: torch.Tensor | None = N
     if a.dtype != torch.float32 or b.dtype != torch.float32 or a.numel() != b.numel():
         raise ValueError("two float32 arrays of the same size are needed")
     if out is None:
-        out = torch.empty_like(a)
+        out = _alloc(a.numel(), torch.float32, a.device).view(a.shape)
     _check(lib().st_packed_mul(a.numel(), _dev(a, "a"), _dev(b, "b"), _dev(out, "out"), _stream()), "st_packed_mul")
     return out
 
 
 def st_check_status(ws: torch.Tensor | None = None) -> int:
+    """Synchronises the current stream and returns the device-side status of `ws`; without an
+    argument, of the workspace used by the most recent compute call on the current device."""
+    if ws is None:
+        ws = _last_ws.get(torch.cuda.current_device())
     return int(lib().st_check_status(ws.data_ptr() if ws is not None else None, _stream()))

@@ -32,12 +32,12 @@ def _deps_mtime():
     return m
 
 
-def _compile(src: str, verbose: bool, objdir: str = OBJDIR, defines=()) -> str:
-    obj = os.path.join(objdir, src[:-3] + ".o")
+def _compile(src: str, verbose: bool) -> str:
+    obj = os.path.join(OBJDIR, src[:-3] + ".o")
     spath = os.path.join(CSRC, src)
     if os.path.exists(obj) and os.path.getmtime(obj) >= max(os.path.getmtime(spath), _deps_mtime()):
         return obj
-    cmd = ["nvcc", *NVCC_FLAGS, *["-D" + d for d in defines], "-c", spath, "-o", obj]
+    cmd = ["nvcc", *NVCC_FLAGS, "-c", spath, "-o", obj]
     if verbose:
         cmd.insert(1, "-Xptxas=-v")
     res = subprocess.run(cmd, capture_output=True, text=True)
@@ -48,11 +48,8 @@ def _compile(src: str, verbose: bool, objdir: str = OBJDIR, defines=()) -> str:
     return obj
 
 
-def build(force: bool = False, verbose: bool = False, out: str = LIB, objdir: str = OBJDIR, defines=()) -> str:
-    """Compiles every .cu under csrc/ and links the shared library.  `out`, `objdir` and `defines`
-    build a variant (extra -D macros) beside the default library."""
-    LIB = out
-    OBJDIR = objdir
+def build(force: bool = False, verbose: bool = False) -> str:
+    """Compiles every .cu under csrc/ and links the shared library."""
     os.makedirs(OBJDIR, exist_ok=True)
     if force:
         for f in os.listdir(OBJDIR):
@@ -60,7 +57,7 @@ def build(force: bool = False, verbose: bool = False, out: str = LIB, objdir: st
                 os.remove(os.path.join(OBJDIR, f))
     srcs = _sources()
     with concurrent.futures.ThreadPoolExecutor(max_workers=min(8, len(srcs))) as ex:
-        objs = list(ex.map(lambda s: _compile(s, verbose, OBJDIR, defines), srcs))
+        objs = list(ex.map(lambda s: _compile(s, verbose), srcs))
     if force or not os.path.exists(LIB) or any(os.path.getmtime(o) > os.path.getmtime(LIB) for o in objs):
         tmp = LIB + ".%d.tmp" % os.getpid()
         cmd = ["nvcc", "-shared", "-gencode", "arch=compute_100a,code=sm_100a", "-o", tmp, *objs]

@@ -22,9 +22,16 @@ namespace st {
 st_status ttm_tf32_tc(const float *Bp, int64_t rows, int64_t K, const float *U, int64_t R, float *Ap, void *ws,
                       size_t ws_bytes, cudaStream_t stream);
 st_status mttkrp_slice_tf32_tc(const float *Bp, int64_t rows, int64_t div, int64_t K, const float *C, const float *D,
-                               int64_t R, float *A, void *ws, size_t ws_bytes, cudaStream_t stream);
+                               int64_t R, float *A, void *zero, size_t zero_bytes, void *ws, size_t ws_bytes,
+                               cudaStream_t stream);
 st_status mttkrp_tf32_tc(const float *Bp, int64_t I, int64_t K, const float *C, const float *D, int64_t R, float *A,
                          bool dense, void *ws, size_t ws_bytes, cudaStream_t stream);
+
+// The fp32 kernels need no workspace; when the caller passes one anyway its status word is set to "ok".
+static inline unsigned *ws_status(void *ws, size_t ws_bytes)
+{
+    return (ws && ws_bytes >= kWsHeaderBytes && aligned256(ws)) ? (unsigned *)ws : nullptr;
+}
 
 constexpr int RG_THREADS = 256;
 constexpr int RG_KC = 32;         // k-values per stage
@@ -49,6 +56,7 @@ struct RgArgs {
     int K, R, I;         // I: rows of A reachable from `out`
     int64_t div;         // RG_MTTKRP_DENSE: fibre `row` belongs to (i, j) = (row / div, row % div)
     int tiles, ksplit, kchunks_per_split, kchunks;
+    unsigned *status;    // workspace header, or NULL
 };
 
 // TM rows x 8 columns per thread, CT column threads (R = 8*CT), RG_ROWS = 256/CT*TM fibres per tile.
@@ -65,6 +73,10 @@ __global__ void __launch_bounds__(RG_THREADS, 1) rowgemm_kernel(const RgArgs a)
     const int tid = threadIdx.x;
     const int tc = tid % CT, tr = tid / CT;
 
+    if (a.status && blockIdx.x == 0 && tid == 0) {      // no bounded waits in this kernel: the status is "ok"
+        a.status[kWsStatusWord] = 0;
+        a.status[kWsDetailWord] = 0;
+    }
     for (int e = tid; e < a.kchunks * RG_KC * a.R / 4; e += RG_THREADS)
         reinterpret_cast<float4 *>(Ws)[e] =
             (e < a.K * a.R / 4) ? reinterpret_cast<const float4 *>(a.W)[e] : make_float4(0.f, 0.f, 0.f, 0.f);
@@ -237,8 +249,10 @@ static size_t rowgemm_smem(int64_t K, int64_t R)
     return (kpad * R + (size_t)stages * rows * RG_LD + (size_t)RG_NI * R) * sizeof(float);
 }
 
+// `zero` (MTTKRP: the output A, which the kernel adds into) is cleared right before the launch, after
+// every check that can still reject the call.
 template <int MODE>
-static st_status rowgemm_launch(const RgArgs &a0, cudaStream_t stream)
+static st_status rowgemm_launch(const RgArgs &a0, cudaStream_t stream, void *zero = nullptr, size_t zero_bytes = 0)
 {
     RgArgs a = a0;
     const DeviceInfo di = device_info();
@@ -267,6 +281,7 @@ static st_status rowgemm_launch(const RgArgs &a0, cudaStream_t stream)
     const int grid = (int)(items < di.sm_count ? items : di.sm_count);
     auto run = [&](auto kernel) -> st_status {
         if (!ensure_dynamic_smem(kernel, smem)) return ST_ERR_CUDA;
+        if (zero && cudaMemsetAsync(zero, 0, zero_bytes, stream) != cudaSuccess) return ST_ERR_CUDA;
         kernel<<<grid, RG_THREADS, smem, stream>>>(a);
         return launch_status();
     };
@@ -300,6 +315,7 @@ st_status st_ttm_blockdiag(const float *Bp, int64_t nblocks, int64_t bs, int64_t
     if (R != 8 && R != 16 && R != 32 && R != 64) return ST_ERR_UNSUPPORTED;
     RgArgs a{};
     a.B = Bp; a.W = U; a.C = nullptr; a.out = Ap; a.rows = rows; a.K = (int)K; a.R = (int)R; a.I = 0;
+    a.status = ws_status(ws, ws_bytes);
     return rowgemm_launch<RG_TTM>(a, (cudaStream_t)stream);
 }
 
@@ -321,6 +337,7 @@ st_status st_ttm_packed(const st_layout *layout, const float *Bp, const float *U
     if (R != 8 && R != 16 && R != 32 && R != 64) return ST_ERR_UNSUPPORTED;
     RgArgs a{};
     a.B = Bp; a.W = U; a.C = nullptr; a.out = Ap; a.rows = rows; a.K = (int)K; a.R = (int)R; a.I = 0;
+    a.status = ws_status(ws, ws_bytes);
     return rowgemm_launch<RG_TTM>(a, (cudaStream_t)stream);
 }
 
@@ -342,9 +359,10 @@ st_status st_mttkrp_tri(const float *Bp, int64_t I, int64_t K, const float *C, c
     a.B = Bp; a.W = D; a.C = C; a.out = A; a.K = (int)K; a.R = (int)R; a.I = (int)I;
     a.rows = dense ? I * I : tri_rows(I);
     a.div = I;
-    if (cudaMemsetAsync(A, 0, (size_t)I * R * sizeof(float), (cudaStream_t)stream) != cudaSuccess) return ST_ERR_CUDA;
-    return dense ? rowgemm_launch<RG_MTTKRP_DENSE>(a, (cudaStream_t)stream)
-                 : rowgemm_launch<RG_MTTKRP_PACKED>(a, (cudaStream_t)stream);
+    a.status = ws_status(ws, ws_bytes);
+    const size_t a_bytes = (size_t)I * R * sizeof(float);
+    return dense ? rowgemm_launch<RG_MTTKRP_DENSE>(a, (cudaStream_t)stream, A, a_bytes)
+                 : rowgemm_launch<RG_MTTKRP_PACKED>(a, (cudaStream_t)stream, A, a_bytes);
 }
 
 st_status st_mttkrp_slice(const float *Bp, int64_t I, int64_t J, int64_t K, int64_t fixed_i, int64_t fixed_j,
@@ -367,15 +385,16 @@ st_status st_mttkrp_slice(const float *Bp, int64_t I, int64_t J, int64_t K, int6
     const float *Cs = fixed_j >= 0 ? C + fixed_j * R : C;
     float *As = fixed_i >= 0 ? A + fixed_i * R : A;
     cudaStream_t s = (cudaStream_t)stream;
-    if (cudaMemsetAsync(A, 0, (size_t)I * R * sizeof(float), s) != cudaSuccess) return ST_ERR_CUDA;
-    if (flags & ST_FLAG_TC_TF32) return mttkrp_slice_tf32_tc(Bp, rows, div, K, Cs, D, R, As, ws, ws_bytes, s);
+    const size_t a_bytes = (size_t)I * R * sizeof(float);
+    if (flags & ST_FLAG_TC_TF32) return mttkrp_slice_tf32_tc(Bp, rows, div, K, Cs, D, R, As, A, a_bytes, ws, ws_bytes, s);
     if (R != 8 && R != 16 && R != 32 && R != 64) return ST_ERR_UNSUPPORTED;
     RgArgs a{};
     a.B = Bp; a.W = D; a.C = Cs; a.out = As; a.K = (int)K; a.R = (int)R;
     a.I = (int)(fixed_i >= 0 ? 1 : I);
     a.rows = rows;
     a.div = div;
-    return rowgemm_launch<RG_MTTKRP_DENSE>(a, s);
+    a.status = ws_status(ws, ws_bytes);
+    return rowgemm_launch<RG_MTTKRP_DENSE>(a, s, A, a_bytes);
 }
 
 }  // extern "C"

@@ -54,8 +54,12 @@ static M2Plan moment2_plan(int64_t N, int64_t d, unsigned flags)
 template <bool DENSE>
 __global__ void __launch_bounds__(256)
 moment2_f32_kernel(const float *__restrict__ X, int64_t N, int d, int64_t ldx, float *__restrict__ out,
-                   float *__restrict__ partials, int nt, int nsplit, int64_t rows_per_split)
+                   float *__restrict__ partials, int nt, int nsplit, int64_t rows_per_split, unsigned *status)
 {
+    if (blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0) {   // no bounded waits here: the status is "ok"
+        status[kWsStatusWord] = 0;
+        status[kWsDetailWord] = 0;
+    }
     __shared__ __align__(16) float As[M2_KC][M2_T];
     __shared__ __align__(16) float Bs[M2_KC][M2_T];
 
@@ -192,10 +196,10 @@ static st_status moment2_f32(const float *X, int64_t N, int64_t d, int64_t ldx, 
     const int dense = (flags & ST_FLAG_DENSE_CONTROL) ? 1 : 0;
     if (dense)
         moment2_f32_kernel<true><<<grid, 256, 0, stream>>>(X, N, (int)d, ldx, out, partials, p.nt, p.nsplit,
-                                                           p.rows_per_split);
+                                                           p.rows_per_split, (unsigned *)ws);
     else
         moment2_f32_kernel<false><<<grid, 256, 0, stream>>>(X, N, (int)d, ldx, out, partials, p.nt, p.nsplit,
-                                                            p.rows_per_split);
+                                                            p.rows_per_split, (unsigned *)ws);
     if (cudaGetLastError() != cudaSuccess) return ST_ERR_CUDA;
     moment2_f32_reduce_kernel<<<dim3(p.ntiles, 16), 256, 0, stream>>>(partials, out, (int)d, p.nt, p.nsplit, dense);
     return launch_status();

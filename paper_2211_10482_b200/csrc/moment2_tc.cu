@@ -251,16 +251,10 @@ moment2_tc_reduce_kernel(const float *__restrict__ partials, float *__restrict__
 namespace m2tc2 {
 constexpr int BM = 256, BN = 256;               // tile of the pair
 constexpr int HALF = 128;                       // rows / B columns staged per block
-#ifndef ST_M2PAIR_KROWS
-#define ST_M2PAIR_KROWS 64
-#endif
-constexpr int KROWS = ST_M2PAIR_KROWS, BOXC = m2tc::BOXC, BOX_BYTES = BOXC * KROWS * 2;
+constexpr int KROWS = 64, BOXC = m2tc::BOXC, BOX_BYTES = BOXC * KROWS * 2;
 constexpr int NBOX = HALF / BOXC;               // 2 boxes per operand per block
 constexpr int STAGE_BYTES = 2 * NBOX * BOX_BYTES;   // 32 KiB
-#ifndef ST_M2PAIR_STAGES
-#define ST_M2PAIR_STAGES 4
-#endif
-constexpr int STAGES = ST_M2PAIR_STAGES;
+constexpr int STAGES = 4;
 constexpr int THREADS = 192;
 constexpr int MAX_TILES = 160;
 constexpr uint32_t TMEM_COLS = 512;

@@ -110,8 +110,12 @@ __device__ __forceinline__ void m3_stage(const float *__restrict__ xs, int d_, i
 template <int WARPS, int DC>
 __global__ void __launch_bounds__(M3_THREADS, 1)
 moment3_kernel(const float *__restrict__ X, int64_t N, int d, int64_t ldx, float *__restrict__ partials,
-               int64_t rows_per_slice, int out_elems, const __grid_constant__ M3Table<WARPS> tab)
+               int64_t rows_per_slice, int out_elems, unsigned *status, const __grid_constant__ M3Table<WARPS> tab)
 {
+    if (blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0) {   // this kernel has no bounded waits: the status is "ok"
+        status[kWsStatusWord] = 0;
+        status[kWsDetailWord] = 0;
+    }
     extern __shared__ __align__(16) float smem[];   // M3_BUFFERS stages of M3_STAGE_ROWS x d floats
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int group = blockIdx.x;
@@ -416,11 +420,11 @@ static st_status moment3_launch(const float *X, int64_t N, int64_t d, int64_t ld
     if (d == M3_MAX_D) {      // the largest side has its own instance with compile-time strides
         if (!ensure_dynamic_smem(moment3_kernel<WARPS, M3_MAX_D>, smem)) return ST_ERR_CUDA;
         moment3_kernel<WARPS, M3_MAX_D><<<grid, M3_THREADS, smem, stream>>>(X, N, (int)d, ldx, partials, p.rows_per_slice,
-                                                                           (int)p.out_elems, local);
+                                                                           (int)p.out_elems, (unsigned *)ws, local);
     } else {
         if (!ensure_dynamic_smem(moment3_kernel<WARPS, 0>, smem)) return ST_ERR_CUDA;
         moment3_kernel<WARPS, 0><<<grid, M3_THREADS, smem, stream>>>(X, N, (int)d, ldx, partials, p.rows_per_slice,
-                                                                    (int)p.out_elems, local);
+                                                                    (int)p.out_elems, (unsigned *)ws, local);
     }
     if (cudaGetLastError() != cudaSuccess) return ST_ERR_CUDA;
     return sum_slices_launch(partials, out, p.out_elems, p.slices, stream);

@@ -107,8 +107,14 @@ pair_expand_kernel(const float *__restrict__ X, int64_t N, int d, int64_t ldx, O
 // One block per row (i,j,k) of the 4-simplex: out[s(i,j,k,l)], l = k..d-1, is the run of row (i,j),
 // columns (k,k)..(k,d-1) of the packed pair-by-pair triangle.
 __global__ void __launch_bounds__(64)
-simplex_gather_kernel(const float *__restrict__ M2, float *__restrict__ out, int d, int64_t dP)
+simplex_gather_kernel(const float *__restrict__ M2, float *__restrict__ out, int d, int64_t dP, unsigned *status,
+                      const unsigned *inner_status)
 {
+    // the second-moment step ran on its own part of the workspace: its status becomes the call's
+    if (blockIdx.x == 0 && threadIdx.x == 0) {
+        status[kWsStatusWord] = inner_status[kWsStatusWord];
+        status[kWsDetailWord] = inner_status[kWsDetailWord];
+    }
     int64_t i, j, k;
     tet_decode(d, blockIdx.x, i, j, k);
     const int64_t p = tri_encode(d, i, j), q = tri_encode(d, k, k);       // p <= q because j <= k
@@ -160,6 +166,7 @@ extern "C" st_status st_sym_moment4(const float *X, int64_t N, int64_t d, int64_
     const st_status rc = st_sym_moment2(w + p.off_p, p.bf16 ? ST_BF16 : ST_F32, N, p.dP, p.dP, M2, w + p.off_ws,
                                         (size_t)p.m2_ws, 0, stream_);
     if (rc != ST_OK) return rc;
-    simplex_gather_kernel<<<(unsigned)tet_rows(d), 64, 0, stream>>>(M2, out_packed, (int)d, p.dP);
+    simplex_gather_kernel<<<(unsigned)tet_rows(d), 64, 0, stream>>>(M2, out_packed, (int)d, p.dP, (unsigned *)w,
+                                                                    (const unsigned *)(w + p.off_ws));
     return launch_status();
 }

@@ -236,11 +236,12 @@ slice_copy_kernel(const U *__restrict__ src, U *__restrict__ dst, LayoutArgs a, 
     }
 }
 
-// out = alpha * a + beta * b (OP 0) or out = a * b (OP 1) over packed arrays of the same layout
+// out = alpha * a + beta * b (OP 0) or out = a * b (OP 1) over packed arrays of the same layout.
+// `out` may be `a` or `b` (a thread reads the elements it later writes, and nobody else's), so none of
+// the pointers is declared restrict.
 template <int OP>
 __global__ void __launch_bounds__(256)
-packed_binary_kernel(const float *__restrict__ a, const float *__restrict__ b, float *__restrict__ out, int64_t n,
-                     float alpha, float beta)
+packed_binary_kernel(const float *a, const float *b, float *out, int64_t n, float alpha, float beta)
 {
     const int64_t n4 = n >> 2;
     const int64_t stride = (int64_t)gridDim.x * blockDim.x;

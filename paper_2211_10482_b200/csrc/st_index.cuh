@@ -23,14 +23,16 @@ ST_HD int64_t tet_rows(int64_t d) { return (d * (d + 1) / 2) * (d + 2) / 3; }  /
 ST_HD int64_t tri_row_start(int64_t d, int64_t i) { return i * (2 * d - i + 1) / 2; }
 ST_HD int64_t tri_encode(int64_t d, int64_t i, int64_t j) { return tri_row_start(d, i) + (j - i); }
 
-// Inverse of tri_encode: the largest i with tri_row_start(d,i) <= p.  The square-root
-// estimate is corrected with integer comparisons, so it is exact for every p.
+// Inverse of tri_encode: the largest i with tri_row_start(d,i) <= p.  The discriminant is an exact
+// integer; only its square root is taken in floating point -- single precision, which the GPU
+// evaluates at full rate -- and the estimate is corrected with integer comparisons, so the result is
+// exact for every p.
 ST_HD void tri_decode(int64_t d, int64_t p, int64_t &i, int64_t &j)
 {
-    const double b = 2.0 * (double)d + 1.0;
-    double disc = b * b - 8.0 * (double)p;
-    if (disc < 0.0) disc = 0.0;
-    int64_t ii = (int64_t)((b - sqrt(disc)) * 0.5);
+    const int64_t b = 2 * d + 1;
+    int64_t disc = b * b - 8 * p;
+    if (disc < 0) disc = 0;
+    int64_t ii = (b - (int64_t)sqrtf((float)disc)) >> 1;
     if (ii < 0) ii = 0;
     if (ii > d - 1) ii = d - 1;
     while (ii > 0 && tri_row_start(d, ii) > p) --ii;
@@ -51,7 +53,7 @@ ST_HD int64_t tet_encode(int64_t d, int64_t i, int64_t j, int64_t k)
 ST_HD void tet_decode(int64_t d, int64_t q, int64_t &i, int64_t &j, int64_t &k)
 {
     const int64_t r = tet_rows(d) - q;          // positions left, 1 <= r <= tet(d)
-    int64_t m = (int64_t)cbrt(6.0 * (double)r); // slab i has side m = d-i: tet(m-1) < r <= tet(m)
+    int64_t m = (int64_t)cbrtf(6.0f * (float)r); // slab i has side m = d-i: tet(m-1) < r <= tet(m)
     if (m < 1) m = 1;
     if (m > d) m = d;
     while (m > 1 && tet_rows(m - 1) >= r) --m;

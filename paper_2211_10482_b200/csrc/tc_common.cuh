@@ -193,10 +193,6 @@ inline EncodeTiledFn encode_tiled_fn()
     return fn;
 }
 
-#ifndef ST_TMA_L2_PROMOTION
-#define ST_TMA_L2_PROMOTION CU_TENSOR_MAP_L2_PROMOTION_L2_256B
-#endif
-
 // Row-major [rows, cols] matrix with a row pitch of `pitch_bytes`; box of box_cols x box_rows,
 // 128-byte swizzle, out-of-range elements read as zero.
 inline bool make_tmap_2d(CUtensorMap *m, CUtensorMapDataType dt, const void *base, uint64_t rows, uint64_t cols,
@@ -209,7 +205,7 @@ inline bool make_tmap_2d(CUtensorMap *m, CUtensorMapDataType dt, const void *bas
     cuuint32_t box[2] = {box_cols, box_rows};
     cuuint32_t estr[2] = {1, 1};
     return fn(m, dt, 2, const_cast<void *>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-              CU_TENSOR_MAP_SWIZZLE_128B, ST_TMA_L2_PROMOTION,
+              CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 

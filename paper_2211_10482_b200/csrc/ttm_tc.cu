@@ -274,8 +274,10 @@ static TtmTcPlan ttm_tc_plan(int64_t K, int64_t R)
     p.ok = false;
     if (K <= 0 || R <= 0 || K % 4 != 0 || R % 16 != 0 || R > 256 || K > (1 << 20)) return p;
     p.kchunks = (int)((K + KC - 1) / KC);
+    // two accumulators of R columns; the epilogue reads them with 32-column loads, so the second one
+    // (which starts at column R) needs R rounded up to 32 columns behind it: 64 columns for R = 16
     uint32_t cols = 32;
-    while (cols < 2 * (uint32_t)R) cols *= 2;
+    while (cols < (uint32_t)R + ((uint32_t)R + 31u) / 32u * 32u) cols *= 2;
     p.tmem_cols = cols;
     const size_t u_bytes = (size_t)p.kchunks * R * 128;
     const size_t fixed = 1024 + u_bytes + 512;
@@ -297,7 +299,7 @@ size_t ttm_tf32_tc_workspace(int64_t rows, int64_t K, int64_t R)
 
 static st_status tc_rows_launch(const float *Bp, int64_t rows, int64_t K, const float *U, int64_t R, float *Ap,
                                 const float *C, int64_t I, int mode, void *ws, size_t ws_bytes, cudaStream_t stream,
-                                int64_t div = 0);
+                                int64_t div = 0, void *zero = nullptr, size_t zero_bytes = 0);
 
 st_status ttm_tf32_tc(const float *Bp, int64_t rows, int64_t K, const float *U, int64_t R, float *Ap, void *ws,
                       size_t ws_bytes, cudaStream_t stream)
@@ -311,23 +313,24 @@ st_status mttkrp_tf32_tc(const float *Bp, int64_t I, int64_t K, const float *C, 
                          bool dense, void *ws, size_t ws_bytes, cudaStream_t stream)
 {
     if (R % 32 != 0) return ST_ERR_UNSUPPORTED;
-    if (cudaMemsetAsync(A, 0, (size_t)I * R * sizeof(float), stream) != cudaSuccess) return ST_ERR_CUDA;
     const int64_t rows = dense ? I * I : tri_rows(I);
-    return tc_rows_launch(Bp, rows, K, D, R, A, C, I, dense ? TC_MTTKRP_DENSE : TC_MTTKRP_PACKED, ws, ws_bytes, stream);
+    return tc_rows_launch(Bp, rows, K, D, R, A, C, I, dense ? TC_MTTKRP_DENSE : TC_MTTKRP_PACKED, ws, ws_bytes, stream,
+                          0, A, (size_t)I * R * sizeof(float));
 }
 
 // MTTKRP on a slice of B (fixed i and / or fixed j): the fibres of the slice are the rows, A and C arrive
-// already shifted to the fixed row (A is zeroed by the caller).
+// already shifted to the fixed row; `zero` is the whole of A, cleared right before the launch.
 st_status mttkrp_slice_tf32_tc(const float *Bp, int64_t rows, int64_t div, int64_t K, const float *C, const float *D,
-                               int64_t R, float *A, void *ws, size_t ws_bytes, cudaStream_t stream)
+                               int64_t R, float *A, void *zero, size_t zero_bytes, void *ws, size_t ws_bytes,
+                               cudaStream_t stream)
 {
     if (R % 32 != 0) return ST_ERR_UNSUPPORTED;
-    return tc_rows_launch(Bp, rows, K, D, R, A, C, 1, TC_MTTKRP_DENSE, ws, ws_bytes, stream, div);
+    return tc_rows_launch(Bp, rows, K, D, R, A, C, 1, TC_MTTKRP_DENSE, ws, ws_bytes, stream, div, zero, zero_bytes);
 }
 
 static st_status tc_rows_launch(const float *Bp, int64_t rows, int64_t K, const float *U, int64_t R, float *Ap,
                                 const float *C, int64_t I, int mode, void *ws, size_t ws_bytes, cudaStream_t stream,
-                                int64_t div)
+                                int64_t div, void *zero, size_t zero_bytes)
 {
     using namespace ttmtc;
     const TtmTcPlan p = ttm_tc_plan(K, R);
@@ -352,6 +355,8 @@ static st_status tc_rows_launch(const float *Bp, int64_t rows, int64_t K, const 
     a.reverse = mode != TC_TTM ? 1 : 0;
     if (!ensure_dynamic_smem(ttm_tc_kernel, p.smem)) return ST_ERR_CUDA;
     const int grid = a.ntiles < di.sm_count ? a.ntiles : di.sm_count;
+    // the MTTKRP epilogue adds into A: cleared here, after every check that can still reject the call
+    if (zero && cudaMemsetAsync(zero, 0, zero_bytes, stream) != cudaSuccess) return ST_ERR_CUDA;
     ttm_tc_kernel<<<grid, THREADS, p.smem, stream>>>(tmap, a);
     return launch_status();
 }

@@ -13,6 +13,8 @@ import workloads
 torch = pytest.importorskip("torch")
 pytestmark = pytest.mark.gpu
 
+import oracle
+
 TOL = 1e-4   # the fp32 tolerance of the parity tests: |a - b| <= TOL * sum |terms|
 
 
@@ -41,6 +43,10 @@ def test_static_entry_point_matches_the_workspace_one_on_two_calls_in_a_row():
         assert torch.cuda.memory_allocated() == before             # nothing went through torch's allocator
         assert bool(torch.all(torch.isfinite(got)))
         assert bool(torch.all((got - want).abs() <= TOL * scale)), (N, d)
+        # and against the CPU oracle, entry by entry in the packed order i <= j <= k
+        ii, jj, kk = (np.array(v) for v in zip(*[(i, j, k) for i in range(d) for j in range(i, d) for k in range(j, d)]))
+        T, S = oracle.moment3_at(Xh, ii, jj, kk)
+        assert oracle.rel_err(got.cpu().numpy(), T, S) <= TOL, (N, d)
     # the binding of the same name reaches the same entry point
     X = torch.from_numpy(cases[0][0]).cuda()
     out = torch.empty(64 * 65 * 66 // 6, dtype=torch.float32, device="cuda")
