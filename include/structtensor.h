@@ -65,7 +65,7 @@ typedef enum { ST_F32 = 0, ST_BF16 = 1, ST_F64 = 2 } st_dtype;
 typedef enum { ST_TRI_UPPER = 0, ST_TET = 1, ST_BAND = 2, ST_BLOCKDIAG = 3 } st_kind;
 typedef enum { ST_FILL_ZERO = 0, ST_FILL_SYMMETRIC = 1 } st_fill;
 typedef enum { ST_OP_SYM_MOMENT2 = 0, ST_OP_SYM_MOMENT3 = 1, ST_OP_MTTKRP_TRI = 2,
-               ST_OP_TTM_BLOCKDIAG = 3, ST_OP_SYM_MOMENT4 = 4 } st_op;
+               ST_OP_TTM_BLOCKDIAG = 3, ST_OP_SYM_MOMENT4 = 4, ST_OP_MTTKRP_SLICE = 5 } st_op;
 
 /* flags (bit mask) */
 #define ST_FLAG_DENSE_CONTROL 1u /* run the same kernel over the dense, unstructured iteration
@@ -111,7 +111,8 @@ st_status st_unpack(const st_layout *layout, st_dtype dtype, const void *packed,
  *   ST_OP_SYM_MOMENT2   a=N, b=d, c=st_dtype of X, e unused
  *   ST_OP_SYM_MOMENT3   a=N, b=d (flags select the kernel: they change the size)
  *   ST_OP_SYM_MOMENT4   a=N, b=d (flags as for the call)
- *   ST_OP_MTTKRP_TRI    a=I, b=K, c=R
+ *   ST_OP_MTTKRP_TRI    a=I, b=K, c=R (flags as for the call: they change the size)
+ *   ST_OP_MTTKRP_SLICE  a=I, b=J, c=K, e=R (enough for any fixed_i / fixed_j; flags as for the call)
  *   ST_OP_TTM_BLOCKDIAG a=nblocks, b=bs, c=K, e=R
  * Returns 0 for an invalid request (the call itself reports the error).  The current
  * device is queried for its SM count. */
@@ -195,7 +196,9 @@ st_status st_sym_moment3_static(const float *X, int64_t N, int64_t d, int64_t ld
  * A: [I,R] fp32 (dense: its unique set is every (i,r)).  Needs K % 4 == 0, R in {8,16,32,64},
  * I <= 32768.  ST_FLAG_TC_TF32 selects the tensor-core path (Bp truncated and D rounded to TF32,
  * fp32 accumulation, the product with C in fp32; 5e-3 tolerance; needs R % 32 == 0, R <= 256).
- * ST_FLAG_DENSE_CONTROL: Bp is instead a dense [I,I,K] tensor and all j are visited. */
+ * ST_FLAG_DENSE_CONTROL: Bp is instead a dense [I,I,K] tensor and all j are visited.
+ * The sum over j is taken in a fixed order (per-warp partial sums in the workspace, added by a second
+ * kernel): no atomics, every element of A written once, the same bits on every call. */
 st_status st_mttkrp_tri(const float *Bp, int64_t I, int64_t K, const float *C, const float *D,
                         int64_t R, float *A, void *ws, size_t ws_bytes, unsigned flags,
                         void *stream);
@@ -209,7 +212,7 @@ st_status st_mttkrp_tri(const float *Bp, int64_t I, int64_t K, const float *C, c
  * C: [J,R]; D: [K,R]; A: dense [I,R], every element written (with fixed i only row fixed_i is
  * non-zero: A_U(i,r) = (i = fixed_i)).  K % 4 == 0; fp32 path R in {8,16,32,64};
  * ST_FLAG_TC_TF32 as for st_mttkrp_tri (R % 32 == 0, R <= 256, 5e-3 tolerance).
- * Workspace: that of ST_OP_MTTKRP_TRI. */
+ * Workspace: ST_OP_MTTKRP_SLICE.  Fixed-order sum over j as in st_mttkrp_tri. */
 st_status st_mttkrp_slice(const float *Bp, int64_t I, int64_t J, int64_t K, int64_t fixed_i,
                           int64_t fixed_j, const float *C, const float *D, int64_t R, float *A,
                           void *ws, size_t ws_bytes, unsigned flags, void *stream);

@@ -28,7 +28,8 @@ ST_TRI_UPPER, ST_TET, ST_BAND, ST_BLOCKDIAG = 0, 1, 2, 3
 # st_fill
 ST_FILL_ZERO, ST_FILL_SYMMETRIC = 0, 1
 # st_op
-ST_OP_SYM_MOMENT2, ST_OP_SYM_MOMENT3, ST_OP_MTTKRP_TRI, ST_OP_TTM_BLOCKDIAG, ST_OP_SYM_MOMENT4 = 0, 1, 2, 3, 4
+ST_OP_SYM_MOMENT2, ST_OP_SYM_MOMENT3, ST_OP_MTTKRP_TRI, ST_OP_TTM_BLOCKDIAG, ST_OP_SYM_MOMENT4, \
+    ST_OP_MTTKRP_SLICE = 0, 1, 2, 3, 4, 5
 # flags
 ST_FLAG_DENSE_CONTROL = 1
 ST_FLAG_TC_TF32 = 2
@@ -307,7 +308,7 @@ def st_mttkrp_slice(Bp: torch.Tensor, C: torch.Tensor, D: torch.Tensor, I: int, 
         raise ValueError("shape mismatch")
     if out is None:
         out = _alloc(I * R, torch.float32, Bp.device).view(I, R)
-    ws = _workspace(lambda: st_workspace_bytes(ST_OP_MTTKRP_TRI, I, K, R, 0, flags), Bp.device, ws)
+    ws = _workspace(lambda: st_workspace_bytes(ST_OP_MTTKRP_SLICE, I, J, K, R, flags), Bp.device, ws)
     _check(lib().st_mttkrp_slice(_dev(Bp, "Bp"), I, J, K, fixed_i, fixed_j, _dev(C, "C"), _dev(D, "D"), R,
                                  _dev(out, "out"), ws.data_ptr(), ws.numel() * ws.element_size(), flags, _stream()),
            "st_mttkrp_slice")

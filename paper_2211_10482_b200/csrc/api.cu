@@ -6,6 +6,7 @@ size_t moment2_workspace(int64_t N, int64_t d, int xdt, unsigned flags);
 size_t moment3_workspace(int64_t N, int64_t d, unsigned flags);
 size_t moment4_workspace(int64_t N, int64_t d, unsigned flags);
 size_t ttm_tf32_tc_workspace(int64_t rows, int64_t K, int64_t R);
+size_t mttkrp_workspace(int64_t rows, int64_t I, int64_t K, int64_t R, unsigned flags);
 }  // namespace st
 
 extern "C" {
@@ -16,7 +17,17 @@ size_t st_workspace_bytes(st_op op, int64_t a, int64_t b, int64_t c, int64_t e, 
     case ST_OP_SYM_MOMENT2: return st::moment2_workspace(a, b, (int)c, flags);
     case ST_OP_SYM_MOMENT3: return st::moment3_workspace(a, b, flags);
     case ST_OP_SYM_MOMENT4: return st::moment4_workspace(a, b, flags);
-    case ST_OP_MTTKRP_TRI: return (a > 0 && b > 0 && c > 0) ? st::kWsHeaderBytes : 0;
+    case ST_OP_MTTKRP_TRI:
+        if (a <= 0 || a > (1 << 15)) return 0;
+        return st::mttkrp_workspace((flags & ST_FLAG_DENSE_CONTROL) ? a * a : a * (a + 1) / 2, a, b, c, flags);
+    case ST_OP_MTTKRP_SLICE: {
+        // enough for any choice of the fixed indices: the longest slice, reaching every row of A
+        if (a <= 0 || b <= 0) return 0;
+        const size_t x = st::mttkrp_workspace(a, a, c, e, flags), y = st::mttkrp_workspace(b, 1, c, e, flags),
+                     z = st::mttkrp_workspace(1, 1, c, e, flags);
+        if (x == 0 || y == 0 || z == 0) return 0;
+        return x > y ? (x > z ? x : z) : (y > z ? y : z);
+    }
     case ST_OP_TTM_BLOCKDIAG:
         if (a <= 0 || b <= 0 || c <= 0 || e <= 0) return 0;
         if (flags & ST_FLAG_TC_TF32) {

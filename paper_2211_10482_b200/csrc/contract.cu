@@ -12,20 +12,20 @@
 // threads each keep TM x 8 sums in registers (TM = 8 for R >= 32).  Fibres are streamed through
 // a cp.async pipeline in slices of 32 k-values; work items (tile, k-split) are walked in one flattened loop so the
 // pipeline never drains between tiles.  MTTKRP splits k over work items when that evens out
-// the load (its output is a sum over k anyway) and reduces over j with shared-memory
-// accumulators per tile followed by one global atomic per (i,r).
+// the load (its output is a sum over k anyway); the sum over j is taken in a fixed order: every
+// warp writes the sums of its runs of fibres with equal i to partial slots and a second kernel
+// adds the slots of every row of A (mttkrp_common.cuh).
 #include "st_common.cuh"
 #include "st_index.cuh"
+#include "mttkrp_common.cuh"
 
 namespace st {
 
 st_status ttm_tf32_tc(const float *Bp, int64_t rows, int64_t K, const float *U, int64_t R, float *Ap, void *ws,
                       size_t ws_bytes, cudaStream_t stream);
-st_status mttkrp_slice_tf32_tc(const float *Bp, int64_t rows, int64_t div, int64_t K, const float *C, const float *D,
-                               int64_t R, float *A, void *zero, size_t zero_bytes, void *ws, size_t ws_bytes,
-                               cudaStream_t stream);
-st_status mttkrp_tf32_tc(const float *Bp, int64_t I, int64_t K, const float *C, const float *D, int64_t R, float *A,
-                         bool dense, void *ws, size_t ws_bytes, cudaStream_t stream);
+st_status mttkrp_tf32_tc(const float *Bp, const MttkrpRows &m, int64_t K, const float *C, const float *D, int64_t R,
+                         float *A_full, int64_t I_full, int64_t i_off, void *ws, size_t ws_bytes, cudaStream_t stream);
+size_t mttkrp_tf32_tc_workspace(int64_t rows, int64_t I, int64_t K, int64_t R);
 
 // The fp32 kernels need no workspace; when the caller passes one anyway its status word is set to "ok".
 static inline unsigned *ws_status(void *ws, size_t ws_bytes)
@@ -36,7 +36,6 @@ static inline unsigned *ws_status(void *ws, size_t ws_bytes)
 constexpr int RG_THREADS = 256;
 constexpr int RG_KC = 32;         // k-values per stage
 constexpr int RG_LD = RG_KC + 4;  // padded row stride (floats) of a stage
-constexpr int RG_NI = 40;         // rows of A accumulated in shared memory per tile
 
 enum { RG_TTM = 0, RG_MTTKRP_PACKED = 1, RG_MTTKRP_DENSE = 2 };
 
@@ -51,7 +50,7 @@ struct RgArgs {
     const float *B;      // [rows, K]
     const float *W;      // [K, R]
     const float *C;      // MTTKRP: [I, R]
-    float *out;          // TTM: [rows, R];  MTTKRP: A [I, R] (zeroed before the launch)
+    float *out;          // TTM: [rows, R];  MTTKRP: partial slots [slots, R]
     int64_t rows;
     int K, R, I;         // I: rows of A reachable from `out`
     int64_t div;         // RG_MTTKRP_DENSE: fibre `row` belongs to (i, j) = (row / div, row % div)
@@ -67,7 +66,6 @@ __global__ void __launch_bounds__(RG_THREADS, 1) rowgemm_kernel(const RgArgs a)
     extern __shared__ __align__(16) float smem[];
     float *Ws = smem;                                   // [kchunks*RG_KC][R], rows >= K are zero
     float *Bs = Ws + (size_t)a.kchunks * RG_KC * a.R;   // RG_STAGES x [RG_ROWS][RG_LD]
-    float *As = Bs + RG_STAGES * RG_ROWS * RG_LD;       // MTTKRP: [RG_NI][R]
     constexpr int R_ = CT * 8;
     constexpr int RT = RG_THREADS / CT;                 // row threads; thread rows = tr + a*RT
     const int tid = threadIdx.x;
@@ -161,18 +159,12 @@ __global__ void __launch_bounds__(RG_THREADS, 1) rowgemm_kernel(const RgArgs a)
                     }
                 }
             } else {
-                // first row of A touched by this tile
-                int64_t i_first, j_first;
-                if (MODE == RG_MTTKRP_PACKED) tri_decode(a.I, row0, i_first, j_first);
-                else { i_first = row0 / a.div; j_first = 0; }
-                (void)j_first;
-                for (int e = tid; e < RG_NI * R_; e += RG_THREADS) As[e] = 0.f;
-                __syncthreads();
-                // A warp holds, for each i, 32/CT consecutive fibres (8 columns per lane).  When they
-                // all belong to one row of A (the usual case: a row of A owns I-i consecutive fibres)
-                // they are summed with shuffles and one lane per column group adds the result to the
-                // shared accumulator; otherwise every lane adds its own fibre.
+                // A warp holds, for each i-slot, US = 32/CT consecutive fibres (8 columns per lane): one unit.
+                // Every run of fibres of the unit that share the row of A is summed with a shuffle butterfly
+                // (masked when the unit holds several runs) and written to partial slot (unit + row of A).
+                constexpr int US = 32 / CT;
                 const int lane = tid & 31;
+                const int fib = lane / CT;                 // fibre of this lane within the unit
 #pragma unroll
                 for (int i = 0; i < TM; ++i) {
                     const int64_t row = row0 + tr + i * RT;
@@ -194,33 +186,45 @@ __global__ void __launch_bounds__(RG_THREADS, 1) rowgemm_kernel(const RgArgs a)
                         for (int j = 0; j < 8; ++j) v[j] = 0.f;
                     }
                     const int gi32 = (int)gi;
-                    const int gi_first = __shfl_sync(0xffffffffu, gi32, 0);
-                    const int gi_last = __shfl_sync(0xffffffffu, gi32, 31);
-                    const bool uniform = (gi_first == gi_last) && gi_first >= 0;
-                    if (uniform) {
+                    const int prev = __shfl_up_sync(0xffffffffu, gi32, CT);
+                    // one bit per fibre (taken from the lanes with tc == 0)
+                    const unsigned heads = __ballot_sync(0xffffffffu, valid && tc == 0 && (fib == 0 || prev != gi32));
+                    const unsigned vmask = __ballot_sync(0xffffffffu, valid && tc == 0);
+                    if (heads == 0u) continue;             // no fibre of this unit exists
+                    const int64_t unit = (row - fib) / US; // the unit's first row is a multiple of US
+                    const int64_t unit0 = __shfl_sync(0xffffffffu, (long long)unit, 0);
+                    auto store = [&](int64_t slot, const float (&w)[8]) {
+                        float4 *dst = reinterpret_cast<float4 *>(a.out + (slot * a.ksplit + ks) * R_ + tc * 8);
+                        dst[0] = make_float4(w[0], w[1], w[2], w[3]);
+                        dst[1] = make_float4(w[4], w[5], w[6], w[7]);
+                    };
+                    const int gi0 = __shfl_sync(0xffffffffu, gi32, 0);
+                    if (heads == 1u) {
 #pragma unroll
                         for (int off = CT; off < 32; off <<= 1)
 #pragma unroll
                             for (int j = 0; j < 8; ++j) v[j] += __shfl_xor_sync(0xffffffffu, v[j], off);
-                    }
-                    if (valid && (!uniform || lane < CT)) {
-                        const int li = (int)(gi - i_first);
-                        if (li < RG_NI) {
-                            float *dst = As + li * R_ + tc * 8;
+                        if (lane < CT) store(unit0 + gi0, v);
+                    } else if (heads == vmask) {
+                        if (valid) store(unit0 + gi, v);
+                    } else {
+                        unsigned h = heads;
+                        while (h) {
+                            const int l0 = __ffs(h) - 1;
+                            h &= h - 1;
+                            const int l1 = h ? __ffs(h) - 1 : 32;
+                            const bool in = lane >= l0 && lane < l1;
+                            float w[8];
 #pragma unroll
-                            for (int j = 0; j < 8; ++j) atomicAdd(dst + j, v[j]);
-                        } else {
-                            float *dst = a.out + gi * R_ + tc * 8;
+                            for (int j = 0; j < 8; ++j) w[j] = in ? v[j] : 0.f;
 #pragma unroll
-                            for (int j = 0; j < 8; ++j) atomicAdd(dst + j, v[j]);
+                            for (int off = CT; off < 32; off <<= 1)
+#pragma unroll
+                                for (int j = 0; j < 8; ++j) w[j] += __shfl_xor_sync(0xffffffffu, w[j], off);
+                            const int gis = __shfl_sync(0xffffffffu, gi32, l0);
+                            if (lane < CT) store(unit0 + gis, w);
                         }
                     }
-                }
-                __syncthreads();
-                for (int e = tid; e < RG_NI * R_; e += RG_THREADS) {
-                    const int li = e / R_;
-                    const float v = As[e];
-                    if (i_first + li < a.I && v != 0.f) atomicAdd(a.out + (i_first + li) * R_ + (e - li * R_), v);
                 }
             }
 #pragma unroll
@@ -230,6 +234,67 @@ __global__ void __launch_bounds__(RG_THREADS, 1) rowgemm_kernel(const RgArgs a)
         }
     }
     asm volatile("cp.async.wait_group 0;\n" ::);
+    if (MODE != RG_TTM) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // the row sums may be launched
+}
+
+// Second pass of MTTKRP: one warp per row of A adds the partial slots of that row in increasing
+// order (units, then k-splits) and writes the row; rows the fibres do not reach are zero.
+__global__ void __launch_bounds__(256)
+mttkrp_rowsum_kernel(const float *__restrict__ part, float *__restrict__ A, int64_t I_full, int64_t i_off, MttkrpRows m,
+                     int R, int unit_rows, int ksplit)
+{
+    asm volatile("griddepcontrol.wait;" ::: "memory");      // launched early: wait for the kernel that wrote the partials
+    const int lane = threadIdx.x & 31;
+    const int64_t ii = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    if (ii >= I_full) return;
+    const int64_t i = ii - i_off;
+    float *dst = A + ii * R;
+    if (i < 0 || i >= m.I) {
+        for (int r = lane; r < R; r += 32) dst[r] = 0.f;
+        return;
+    }
+    int64_t s, e;
+    if (m.mode == MK_PACKED) { s = tri_row_start(m.I, i); e = s + (m.I - i); }
+    else { s = i * m.div; e = s + m.div; }
+    if (e > m.rows) e = m.rows;
+    const int64_t u0 = s / unit_rows, u1 = (e - 1) / unit_rows;
+    for (int r = lane; r < R; r += 32) {
+        float sum = 0.f;
+        if (e > s) {
+            const float *p = part + ((u0 + i) * ksplit) * R + r;
+            const int64_t n = (u1 - u0 + 1) * ksplit;
+            int64_t k = 0;
+            for (; k + 8 <= n; k += 8) {               // eight independent loads in flight
+                float t[8];
+#pragma unroll
+                for (int u = 0; u < 8; ++u) t[u] = __ldcg(p + (k + u) * R);
+#pragma unroll
+                for (int u = 0; u < 8; ++u) sum += t[u];
+            }
+            for (; k < n; ++k) sum += __ldcg(p + k * R);
+        }
+        dst[r] = sum;
+    }
+}
+
+st_status mttkrp_rowsum_launch(const float *part, float *A_full, int64_t I_full, int64_t i_off, const MttkrpRows &m,
+                               int R, int unit_rows, int ksplit, cudaStream_t stream)
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)((I_full + 7) / 8));
+    cfg.blockDim = dim3(256);
+    cfg.dynamicSmemBytes = 0;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    if (cudaLaunchKernelEx(&cfg, mttkrp_rowsum_kernel, part, A_full, I_full, i_off, m, R, unit_rows, ksplit) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return ST_ERR_CUDA;
+    }
+    return ST_OK;
 }
 
 // tile shape by R: {TM, stages}; rows per tile = 256 / (R/8) * TM
@@ -246,42 +311,55 @@ static size_t rowgemm_smem(int64_t K, int64_t R)
     rowgemm_shape(R, tm, stages);
     const size_t rows = (size_t)RG_THREADS / (R / 8) * tm;
     const size_t kpad = (size_t)((K + RG_KC - 1) / RG_KC) * RG_KC;
-    return (kpad * R + (size_t)stages * rows * RG_LD + (size_t)RG_NI * R) * sizeof(float);
+    return (kpad * R + (size_t)stages * rows * RG_LD) * sizeof(float);
 }
 
-// `zero` (MTTKRP: the output A, which the kernel adds into) is cleared right before the launch, after
-// every check that can still reject the call.
+struct RgPlan {
+    int tiles, ksplit, kchunks, unit_rows;
+};
+
+// Tiles and, for MTTKRP, the k-split that wastes the fewest SM slots in the last wave.
+static RgPlan rowgemm_plan(int64_t rows, int64_t K, int64_t R, bool mttkrp)
+{
+    RgPlan p;
+    int tm, stages;
+    rowgemm_shape(R, tm, stages);
+    const int64_t tile_rows = (int64_t)RG_THREADS / (R / 8) * tm;
+    p.tiles = (int)((rows + tile_rows - 1) / tile_rows);
+    p.kchunks = (int)((K + RG_KC - 1) / RG_KC);
+    p.unit_rows = (int)(32 / (R / 8));
+    p.ksplit = 1;
+    if (mttkrp) {
+        const int sms = sm_count_or_default();
+        double best = -1.0;
+        for (int ks = 1; ks <= 4; ks *= 2) {
+            if (p.kchunks % ks) continue;
+            const int64_t items = (int64_t)p.tiles * ks;
+            const int64_t waves = (items + sms - 1) / sms;
+            const double eff = (double)items / (double)(waves * sms);
+            if (eff > best + 0.02) { best = eff; p.ksplit = ks; }
+        }
+    }
+    return p;
+}
+
 template <int MODE>
-static st_status rowgemm_launch(const RgArgs &a0, cudaStream_t stream, void *zero = nullptr, size_t zero_bytes = 0)
+static st_status rowgemm_launch(const RgArgs &a0, cudaStream_t stream)
 {
     RgArgs a = a0;
     const DeviceInfo di = device_info();
     if (!di.ok) return ST_ERR_CUDA;
     const size_t smem = rowgemm_smem(a.K, a.R);
     if (smem > (size_t)di.max_smem_optin) return ST_ERR_UNSUPPORTED;
-    a.kchunks = (a.K + RG_KC - 1) / RG_KC;
-    int tm, stages;
-    rowgemm_shape(a.R, tm, stages);
-    const int64_t tile_rows = (int64_t)RG_THREADS / (a.R / 8) * tm;
-    a.tiles = (int)((a.rows + tile_rows - 1) / tile_rows);
-    a.ksplit = 1;
-    if (MODE != RG_TTM) {
-        // pick the k-split that wastes the fewest SM slots in the last wave
-        double best = -1.0;
-        for (int ks = 1; ks <= 4; ks *= 2) {
-            if (a.kchunks % ks) continue;
-            const int64_t items = (int64_t)a.tiles * ks;
-            const int64_t waves = (items + di.sm_count - 1) / di.sm_count;
-            const double eff = (double)items / (double)(waves * di.sm_count);
-            if (eff > best + 0.02) { best = eff; a.ksplit = ks; }
-        }
-    }
+    const RgPlan p = rowgemm_plan(a.rows, a.K, a.R, MODE != RG_TTM);
+    a.kchunks = p.kchunks;
+    a.tiles = p.tiles;
+    a.ksplit = p.ksplit;
     a.kchunks_per_split = a.kchunks / a.ksplit;
     const int64_t items = (int64_t)a.tiles * a.ksplit;
     const int grid = (int)(items < di.sm_count ? items : di.sm_count);
     auto run = [&](auto kernel) -> st_status {
         if (!ensure_dynamic_smem(kernel, smem)) return ST_ERR_CUDA;
-        if (zero && cudaMemsetAsync(zero, 0, zero_bytes, stream) != cudaSuccess) return ST_ERR_CUDA;
         kernel<<<grid, RG_THREADS, smem, stream>>>(a);
         return launch_status();
     };
@@ -292,6 +370,40 @@ static st_status rowgemm_launch(const RgArgs &a0, cudaStream_t stream, void *zer
     case 64: return run(rowgemm_kernel<8, 8, 3, MODE>);
     default: return ST_ERR_UNSUPPORTED;
     }
+}
+
+static bool rowgemm_r_ok(int64_t R) { return R == 8 || R == 16 || R == 32 || R == 64; }
+
+// Workspace of MTTKRP over `rows` fibres that reach `I` rows of A: the header and the partial slots.
+size_t mttkrp_workspace(int64_t rows, int64_t I, int64_t K, int64_t R, unsigned flags)
+{
+    if (rows <= 0 || I <= 0 || K <= 0 || R <= 0 || K % 4 != 0) return 0;
+    if (flags & ST_FLAG_TC_TF32) return mttkrp_tf32_tc_workspace(rows, I, K, R);
+    if (!rowgemm_r_ok(R)) return 0;
+    const RgPlan p = rowgemm_plan(rows, K, R, true);
+    return kWsHeaderBytes + (size_t)mttkrp_slots(rows, p.unit_rows, I, p.ksplit) * R * sizeof(float);
+}
+
+// Both passes of MTTKRP; `m` says how a row maps to (i, j), the fibres reach rows i_off .. of A_full.
+static st_status mttkrp_run(const float *Bp, const MttkrpRows &m, int64_t K, const float *C, const float *D, int64_t R,
+                            float *A_full, int64_t I_full, int64_t i_off, void *ws, size_t ws_bytes, unsigned flags,
+                            cudaStream_t stream)
+{
+    if (flags & ST_FLAG_TC_TF32)
+        return mttkrp_tf32_tc(Bp, m, K, C, D, R, A_full, I_full, i_off, ws, ws_bytes, stream);
+    if (!rowgemm_r_ok(R)) return ST_ERR_UNSUPPORTED;
+    const size_t need = mttkrp_workspace(m.rows, m.I, K, R, flags);
+    if (!ws || ws_bytes < need) return ST_ERR_WORKSPACE;
+    if (!aligned256(ws)) return ST_ERR_ALIGN;
+    const RgPlan p = rowgemm_plan(m.rows, K, R, true);
+    RgArgs a{};
+    a.B = Bp; a.W = D; a.C = C; a.out = (float *)((unsigned char *)ws + kWsHeaderBytes);
+    a.K = (int)K; a.R = (int)R; a.I = m.I; a.rows = m.rows; a.div = m.div;
+    a.status = (unsigned *)ws;
+    const st_status rc = m.mode == MK_PACKED ? rowgemm_launch<RG_MTTKRP_PACKED>(a, stream)
+                                             : rowgemm_launch<RG_MTTKRP_DENSE>(a, stream);
+    if (rc != ST_OK) return rc;
+    return mttkrp_rowsum_launch(a.out, A_full, I_full, i_off, m, (int)R, p.unit_rows, p.ksplit, stream);
 }
 
 }  // namespace st
@@ -350,19 +462,13 @@ st_status st_mttkrp_tri(const float *Bp, int64_t I, int64_t K, const float *C, c
     if (flags & ~(ST_FLAG_DENSE_CONTROL | ST_FLAG_TC_TF32)) return ST_ERR_UNSUPPORTED;
     if (!aligned16(Bp) || !aligned16(C) || !aligned16(D) || !aligned16(A)) return ST_ERR_ALIGN;
     if (I > (1 << 15) || K > (1 << 20) || K % 4 != 0) return ST_ERR_UNSUPPORTED;
-    if (flags & ST_FLAG_TC_TF32)
-        return mttkrp_tf32_tc(Bp, I, K, C, D, R, A, (flags & ST_FLAG_DENSE_CONTROL) != 0, ws, ws_bytes,
-                              (cudaStream_t)stream);
-    if (R != 8 && R != 16 && R != 32 && R != 64) return ST_ERR_UNSUPPORTED;
     const bool dense = (flags & ST_FLAG_DENSE_CONTROL) != 0;
-    RgArgs a{};
-    a.B = Bp; a.W = D; a.C = C; a.out = A; a.K = (int)K; a.R = (int)R; a.I = (int)I;
-    a.rows = dense ? I * I : tri_rows(I);
-    a.div = I;
-    a.status = ws_status(ws, ws_bytes);
-    const size_t a_bytes = (size_t)I * R * sizeof(float);
-    return dense ? rowgemm_launch<RG_MTTKRP_DENSE>(a, (cudaStream_t)stream, A, a_bytes)
-                 : rowgemm_launch<RG_MTTKRP_PACKED>(a, (cudaStream_t)stream, A, a_bytes);
+    MttkrpRows m;
+    m.mode = dense ? MK_DENSE : MK_PACKED;
+    m.I = (int)I;
+    m.div = I;
+    m.rows = dense ? I * I : tri_rows(I);
+    return mttkrp_run(Bp, m, K, C, D, R, A, I, 0, ws, ws_bytes, flags, (cudaStream_t)stream);
 }
 
 st_status st_mttkrp_slice(const float *Bp, int64_t I, int64_t J, int64_t K, int64_t fixed_i, int64_t fixed_j,
@@ -383,18 +489,13 @@ st_status st_mttkrp_slice(const float *Bp, int64_t I, int64_t J, int64_t K, int6
     const int64_t rows = fixed_i >= 0 ? (fixed_j >= 0 ? 1 : J) : I;
     const int64_t div = fixed_i >= 0 ? (fixed_j >= 0 ? 1 : J) : 1;
     const float *Cs = fixed_j >= 0 ? C + fixed_j * R : C;
-    float *As = fixed_i >= 0 ? A + fixed_i * R : A;
-    cudaStream_t s = (cudaStream_t)stream;
-    const size_t a_bytes = (size_t)I * R * sizeof(float);
-    if (flags & ST_FLAG_TC_TF32) return mttkrp_slice_tf32_tc(Bp, rows, div, K, Cs, D, R, As, A, a_bytes, ws, ws_bytes, s);
-    if (R != 8 && R != 16 && R != 32 && R != 64) return ST_ERR_UNSUPPORTED;
-    RgArgs a{};
-    a.B = Bp; a.W = D; a.C = Cs; a.out = As; a.K = (int)K; a.R = (int)R;
-    a.I = (int)(fixed_i >= 0 ? 1 : I);
-    a.rows = rows;
-    a.div = div;
-    a.status = ws_status(ws, ws_bytes);
-    return rowgemm_launch<RG_MTTKRP_DENSE>(a, s, A, a_bytes);
+    MttkrpRows m;
+    m.mode = MK_DENSE;
+    m.I = (int)(fixed_i >= 0 ? 1 : I);
+    m.div = div;
+    m.rows = rows;
+    // the fibres reach row fixed_i of A only (fixed i), or every row; the second pass writes the others as zero
+    return mttkrp_run(Bp, m, K, Cs, D, R, A, I, fixed_i >= 0 ? fixed_i : 0, ws, ws_bytes, flags, (cudaStream_t)stream);
 }
 
 }  // extern "C"

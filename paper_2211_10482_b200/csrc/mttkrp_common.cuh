@@ -1,0 +1,59 @@
+// Fixed-order reduction over j of MTTKRP (Table 1): A[i,r] = sum_j C[j,r] * Y[(i,j), r], where
+// Y = sum_k B[(i,j),k] D[k,r] is what the fibre kernels compute.
+//
+// The fibres (i,j) are the rows of a tall matrix in which i never decreases (packed upper half
+// cube: row p(i,j); dense and slice forms: row = i * div + j).  The fibre kernels cut the rows into
+// units of `unit_rows` consecutive rows (the rows one warp reduces with shuffles) and, for every
+// maximal run of rows of one unit that share i, write the sum of the run to partial slot
+//     slot(unit, i) = unit + i        (times ksplit, plus the k-split index, when k is split).
+// Walking the rows, every new run increments unit, i or both, so unit + i is strictly increasing:
+// the slots of different runs differ, and the runs of one i occupy consecutive slots.  The second
+// pass adds the slots of every i in increasing order and writes A, every element exactly once:
+// no atomics, no zeroing of A, and the same bits on every call.
+#pragma once
+#include "st_common.cuh"
+#include "st_index.cuh"
+
+namespace st {
+
+enum { MK_PACKED = 1, MK_DENSE = 2 };      // how a row maps to (i, j)
+
+struct MttkrpRows {
+    int mode;            // MK_PACKED: row = p(i,j) of a triangle of side I;  MK_DENSE: (i, j) = (row / div, row % div)
+    int I;               // rows of A that the fibres reach (MK_PACKED: side of the triangle)
+    int64_t div;
+    int64_t rows;
+};
+
+__host__ __device__ inline int64_t mttkrp_slots(int64_t rows, int unit_rows, int64_t I, int ksplit)
+{
+    return ((rows + unit_rows - 1) / unit_rows + I) * ksplit;
+}
+
+// Second pass.  A_full has I_full rows; the fibres reach rows i_off .. i_off + m.I - 1 of it, the
+// other rows are written as zero.
+st_status mttkrp_rowsum_launch(const float *part, float *A_full, int64_t I_full, int64_t i_off, const MttkrpRows &m,
+                               int R, int unit_rows, int ksplit, cudaStream_t stream);
+
+#if defined(__CUDACC__)
+// Transposing shuffle reduction of 32 columns held by every lane (one fibre per lane): after the
+// step with offset o a lane keeps the half of its columns selected by bit o of its lane index; at
+// the end lane l holds the sum of column l over the warp.  The order of the additions is fixed.
+__device__ __forceinline__ float warp_transpose_sum32(float (&v)[32], int lane)
+{
+#define ST_TR_STEP(OFF)                                                                       \
+    {                                                                                         \
+        const bool up = (lane & OFF) != 0;                                                    \
+        _Pragma("unroll") for (int j = 0; j < OFF; ++j) {                                     \
+            const float send = up ? v[j] : v[j + OFF];                                        \
+            const float keep = up ? v[j + OFF] : v[j];                                        \
+            v[j] = keep + __shfl_xor_sync(0xffffffffu, send, OFF);                            \
+        }                                                                                     \
+    }
+    ST_TR_STEP(16) ST_TR_STEP(8) ST_TR_STEP(4) ST_TR_STEP(2) ST_TR_STEP(1)
+#undef ST_TR_STEP
+    return v[0];
+}
+#endif
+
+}  // namespace st

@@ -11,6 +11,7 @@
 // next.  Warp roles: warp 0 TMA producer, warp 1 MMA issuer / TMEM owner, warps 2..5 epilogue.
 #include "tc_common.cuh"
 #include "st_index.cuh"
+#include "mttkrp_common.cuh"
 
 namespace st {
 
@@ -196,9 +197,10 @@ ttm_tc_kernel(const __grid_constant__ CUtensorMap tmap, const TtmTcArgs a)
                     }
                 }
             } else {
-                // MTTKRP: this lane's fibre is packed row p(i,j); scale by C[j,:] and add into A[i,:].
-                // The 32 fibres of a warp are consecutive, so they usually share i: then the warp sums
-                // them with a transposing shuffle reduction and issues one atomic per column.
+                // MTTKRP: this lane's fibre is row (i,j); scale by C[j,:], then sum every run of fibres of
+                // the warp that share i and write it to partial slot (unit + i), unit = row / 32 (see
+                // mttkrp_common.cuh).  The 32 fibres of a warp are consecutive, so they usually share i:
+                // one transposing shuffle reduction and one coalesced store per 32 columns.
                 const bool valid = row < a.rows;
                 int64_t gi = -1, gj = 0;
                 if (valid) {
@@ -206,8 +208,11 @@ ttm_tc_kernel(const __grid_constant__ CUtensorMap tmap, const TtmTcArgs a)
                     else { gi = row / a.div; gj = row - gi * a.div; }
                 }
                 const int gi32 = (int)gi;
-                const bool uniform = __shfl_sync(0xffffffffu, gi32, 0) == __shfl_sync(0xffffffffu, gi32, 31) && gi32 >= 0;
-                for (int c0 = 0; c0 < a.R; c0 += 32) {
+                const int prev = __shfl_up_sync(0xffffffffu, gi32, 1);
+                const unsigned heads = __ballot_sync(0xffffffffu, valid && (lane == 0 || prev != gi32));
+                const unsigned vmask = __ballot_sync(0xffffffffu, valid);
+                const int64_t unit = tile * (BM / 32) + q;
+                for (int c0 = 0; c0 < a.R && heads != 0u; c0 += 32) {
                     uint32_t r[32];
                     tmem_ld_32x32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * a.R + c0), r);
                     tmem_ld_wait();
@@ -226,24 +231,28 @@ ttm_tc_kernel(const __grid_constant__ CUtensorMap tmap, const TtmTcArgs a)
 #pragma unroll
                         for (int e = 0; e < 32; ++e) v[e] = 0.f;
                     }
-                    if (uniform) {
-                        // after the step with offset o a lane keeps the half of its columns selected by
-                        // bit o of its lane index; at the end lane l holds the sum of column l
-#define ST_TR_STEP(OFF)                                                                       \
-    {                                                                                         \
-        const bool up = (lane & OFF) != 0;                                                    \
-        _Pragma("unroll") for (int j = 0; j < OFF; ++j) {                                     \
-            const float send = up ? v[j] : v[j + OFF];                                        \
-            const float keep = up ? v[j + OFF] : v[j];                                        \
-            v[j] = keep + __shfl_xor_sync(0xffffffffu, send, OFF);                            \
-        }                                                                                     \
-    }
-                        ST_TR_STEP(16) ST_TR_STEP(8) ST_TR_STEP(4) ST_TR_STEP(2) ST_TR_STEP(1)
-#undef ST_TR_STEP
-                        atomicAdd(a.out + (int64_t)gi32 * a.R + c0 + lane, v[0]);
-                    } else if (valid) {
+                    if (heads == 1u) {                     // one run: the whole warp
+                        const float sum = warp_transpose_sum32(v, lane);
+                        a.out[(unit + __shfl_sync(0xffffffffu, gi32, 0)) * a.R + c0 + lane] = sum;
+                    } else if (heads == vmask) {           // every fibre is a run of its own
+                        if (valid) {
+                            float4 *dst = reinterpret_cast<float4 *>(a.out + (unit + gi) * a.R + c0);
 #pragma unroll
-                        for (int e = 0; e < 32; ++e) atomicAdd(a.out + gi * a.R + c0 + e, v[e]);
+                            for (int e = 0; e < 8; ++e) dst[e] = make_float4(v[4 * e], v[4 * e + 1], v[4 * e + 2], v[4 * e + 3]);
+                        }
+                    } else {                               // several runs: one masked reduction per run
+                        unsigned h = heads;
+                        while (h) {
+                            const int s0 = __ffs(h) - 1;
+                            h &= h - 1;
+                            const int s1 = h ? __ffs(h) - 1 : 32;
+                            const bool in = lane >= s0 && lane < s1;
+                            float w[32];
+#pragma unroll
+                            for (int e = 0; e < 32; ++e) w[e] = in ? v[e] : 0.f;
+                            const float sum = warp_transpose_sum32(w, lane);
+                            a.out[(unit + __shfl_sync(0xffffffffu, gi32, s0)) * a.R + c0 + lane] = sum;
+                        }
                     }
                 }
             }
@@ -252,6 +261,8 @@ ttm_tc_kernel(const __grid_constant__ CUtensorMap tmap, const TtmTcArgs a)
             if (lane == 0) mbar_arrive(&acc_empty[buf]);
         }
     }
+    // MTTKRP: the kernel that adds the partial sums may be launched now (it waits for this grid to end)
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     tc_fence_before();
     __syncthreads();
     if (warp == 1) {
@@ -299,7 +310,7 @@ size_t ttm_tf32_tc_workspace(int64_t rows, int64_t K, int64_t R)
 
 static st_status tc_rows_launch(const float *Bp, int64_t rows, int64_t K, const float *U, int64_t R, float *Ap,
                                 const float *C, int64_t I, int mode, void *ws, size_t ws_bytes, cudaStream_t stream,
-                                int64_t div = 0, void *zero = nullptr, size_t zero_bytes = 0);
+                                int64_t div = 0);
 
 st_status ttm_tf32_tc(const float *Bp, int64_t rows, int64_t K, const float *U, int64_t R, float *Ap, void *ws,
                       size_t ws_bytes, cudaStream_t stream)
@@ -307,30 +318,33 @@ st_status ttm_tf32_tc(const float *Bp, int64_t rows, int64_t K, const float *U, 
     return tc_rows_launch(Bp, rows, K, U, R, Ap, nullptr, 0, TC_TTM, ws, ws_bytes, stream);
 }
 
-// MTTKRP on tensor cores: the same streaming kernel with W = D; the epilogue scales every fibre's
-// result by C[j,:] and adds it into A[i,:] (A is zeroed first).  TF32 operands, 5e-3 tolerance.
-st_status mttkrp_tf32_tc(const float *Bp, int64_t I, int64_t K, const float *C, const float *D, int64_t R, float *A,
-                         bool dense, void *ws, size_t ws_bytes, cudaStream_t stream)
+size_t mttkrp_tf32_tc_workspace(int64_t rows, int64_t I, int64_t K, int64_t R)
 {
-    if (R % 32 != 0) return ST_ERR_UNSUPPORTED;
-    const int64_t rows = dense ? I * I : tri_rows(I);
-    return tc_rows_launch(Bp, rows, K, D, R, A, C, I, dense ? TC_MTTKRP_DENSE : TC_MTTKRP_PACKED, ws, ws_bytes, stream,
-                          0, A, (size_t)I * R * sizeof(float));
+    if (rows <= 0 || R % 32 != 0 || !ttm_tc_plan(K, R).ok) return 0;
+    return kWsHeaderBytes + (size_t)mttkrp_slots(rows, 32, I, 1) * R * sizeof(float);
 }
 
-// MTTKRP on a slice of B (fixed i and / or fixed j): the fibres of the slice are the rows, A and C arrive
-// already shifted to the fixed row; `zero` is the whole of A, cleared right before the launch.
-st_status mttkrp_slice_tf32_tc(const float *Bp, int64_t rows, int64_t div, int64_t K, const float *C, const float *D,
-                               int64_t R, float *A, void *zero, size_t zero_bytes, void *ws, size_t ws_bytes,
-                               cudaStream_t stream)
+// MTTKRP on tensor cores: the same streaming kernel with W = D; the epilogue scales every fibre's result
+// by C[j,:] and writes the sums of the runs of equal i to the workspace, a second kernel adds them in a
+// fixed order (mttkrp_common.cuh).  `m` says how a row maps to (i, j); the fibres reach rows
+// i_off .. i_off + m.I - 1 of A_full, which has I_full rows.  TF32 operands, 5e-3 tolerance.
+st_status mttkrp_tf32_tc(const float *Bp, const MttkrpRows &m, int64_t K, const float *C, const float *D, int64_t R,
+                         float *A_full, int64_t I_full, int64_t i_off, void *ws, size_t ws_bytes, cudaStream_t stream)
 {
     if (R % 32 != 0) return ST_ERR_UNSUPPORTED;
-    return tc_rows_launch(Bp, rows, K, D, R, A, C, 1, TC_MTTKRP_DENSE, ws, ws_bytes, stream, div, zero, zero_bytes);
+    const size_t need = mttkrp_tf32_tc_workspace(m.rows, m.I, K, R);
+    if (need == 0) return ST_ERR_UNSUPPORTED;
+    if (!ws || ws_bytes < need) return ST_ERR_WORKSPACE;
+    float *part = (float *)((unsigned char *)ws + kWsHeaderBytes);
+    const st_status rc = tc_rows_launch(Bp, m.rows, K, D, R, part, C, m.I, m.mode == MK_PACKED ? TC_MTTKRP_PACKED : TC_MTTKRP_DENSE,
+                                        ws, ws_bytes, stream, m.div);
+    if (rc != ST_OK) return rc;
+    return mttkrp_rowsum_launch(part, A_full, I_full, i_off, m, (int)R, 32, 1, stream);
 }
 
 static st_status tc_rows_launch(const float *Bp, int64_t rows, int64_t K, const float *U, int64_t R, float *Ap,
                                 const float *C, int64_t I, int mode, void *ws, size_t ws_bytes, cudaStream_t stream,
-                                int64_t div, void *zero, size_t zero_bytes)
+                                int64_t div)
 {
     using namespace ttmtc;
     const TtmTcPlan p = ttm_tc_plan(K, R);
@@ -355,8 +369,6 @@ static st_status tc_rows_launch(const float *Bp, int64_t rows, int64_t K, const 
     a.reverse = mode != TC_TTM ? 1 : 0;
     if (!ensure_dynamic_smem(ttm_tc_kernel, p.smem)) return ST_ERR_CUDA;
     const int grid = a.ntiles < di.sm_count ? a.ntiles : di.sm_count;
-    // the MTTKRP epilogue adds into A: cleared here, after every check that can still reject the call
-    if (zero && cudaMemsetAsync(zero, 0, zero_bytes, stream) != cudaSuccess) return ST_ERR_CUDA;
     ttm_tc_kernel<<<grid, THREADS, p.smem, stream>>>(tmap, a);
     return launch_status();
 }
