@@ -72,6 +72,12 @@ typedef enum { ST_OP_SYM_MOMENT2 = 0, ST_OP_SYM_MOMENT3 = 1, ST_OP_MTTKRP_TRI = 
                                     space (a control for measurements; see each call) */
 #define ST_FLAG_TC_TF32       2u /* st_ttm_blockdiag, st_mttkrp_tri, st_sym_moment3: tensor cores, operands read as TF32 */
 #define ST_FLAG_TC_BF16       4u /* st_sym_moment3, st_sym_moment4: tensor cores, operands rounded to bf16 */
+#define ST_FLAG_TC_SPLIT      8u /* st_ttm_blockdiag, st_ttm_packed, st_mttkrp_tri, st_mttkrp_slice: tensor cores with
+                                    both operands split into two bf16 parts and three of the four partial products
+                                    kept: meets the 1e-4 tolerance of the fp32 path, at the speed of the HBM stream
+                                    (needs K % 4 == 0, R % 32 == 0, R <= 128, and the split factor, 4*K*R bytes rounded up to
+                                    whole chunks of 64 k-values, in shared memory: K*R <= 40960; not with
+                                    ST_FLAG_TC_TF32) */
 
 typedef struct {
     int32_t kind;      /* st_kind */
@@ -196,6 +202,7 @@ st_status st_sym_moment3_static(const float *X, int64_t N, int64_t d, int64_t ld
  * A: [I,R] fp32 (dense: its unique set is every (i,r)).  Needs K % 4 == 0, R in {8,16,32,64},
  * I <= 32768.  ST_FLAG_TC_TF32 selects the tensor-core path (Bp truncated and D rounded to TF32,
  * fp32 accumulation, the product with C in fp32; 5e-3 tolerance; needs R % 32 == 0, R <= 256).
+ * ST_FLAG_TC_SPLIT: tensor cores with split bf16 operands, 1e-4 tolerance (see the flag).
  * ST_FLAG_DENSE_CONTROL: Bp is instead a dense [I,I,K] tensor and all j are visited.
  * The sum over j is taken in a fixed order (per-warp partial sums in the workspace, added by a second
  * kernel): no atomics, every element of A written once, the same bits on every call. */
@@ -211,7 +218,7 @@ st_status st_mttkrp_tri(const float *Bp, int64_t I, int64_t K, const float *C, c
  * Bp: the packed slice, fp32: [J, K] (fixed i; row = j), [I, K] (fixed j; row = i), [K] (both).
  * C: [J,R]; D: [K,R]; A: dense [I,R], every element written (with fixed i only row fixed_i is
  * non-zero: A_U(i,r) = (i = fixed_i)).  K % 4 == 0; fp32 path R in {8,16,32,64};
- * ST_FLAG_TC_TF32 as for st_mttkrp_tri (R % 32 == 0, R <= 256, 5e-3 tolerance).
+ * ST_FLAG_TC_TF32 as for st_mttkrp_tri (R % 32 == 0, R <= 256, 5e-3 tolerance), ST_FLAG_TC_SPLIT likewise.
  * Workspace: ST_OP_MTTKRP_SLICE.  Fixed-order sum over j as in st_mttkrp_tri. */
 st_status st_mttkrp_slice(const float *Bp, int64_t I, int64_t J, int64_t K, int64_t fixed_i,
                           int64_t fixed_j, const float *C, const float *D, int64_t R, float *A,
@@ -224,7 +231,8 @@ st_status st_mttkrp_slice(const float *Bp, int64_t I, int64_t J, int64_t K, int6
  * Bp: packed [nblocks*bs*bs, K] fp32; U: [K,R] fp32; Ap: packed [nblocks*bs*bs, R] fp32.
  * Needs K % 4 == 0 and R % 4 == 0.  ST_FLAG_TC_TF32 selects the tensor-core path
  * (Bp truncated and U rounded to TF32, fp32 accumulation; 5e-3 tolerance; needs K % 4 == 0,
- * R % 16 == 0, R <= 256).
+ * R % 16 == 0, R <= 256).  ST_FLAG_TC_SPLIT: tensor cores with split bf16 operands, 1e-4 tolerance
+ * (see the flag).
  * ST_FLAG_DENSE_CONTROL: Bp is a dense [d,d,K] tensor and Ap a dense [d,d,R] one,
  * d = nblocks*bs; all d*d fibres are multiplied. */
 st_status st_ttm_blockdiag(const float *Bp, int64_t nblocks, int64_t bs, int64_t K,
@@ -237,7 +245,7 @@ st_status st_ttm_blockdiag(const float *Bp, int64_t nblocks, int64_t bs, int64_t
  * ST_BLOCKDIAG with bs = 1 (or ST_BAND with kl = ku = 0) its "diagonal plane" (i = j), ST_TET a
  * 4-mode tensor with i <= j <= k.  The output has the structure of the input with inner = R
  * (the unique set of the product, projected over k, keeps B's (i,j) part: Section 5.1).
- * Same kernels, flags (ST_FLAG_TC_TF32 only) and shape limits as st_ttm_blockdiag; the
+ * Same kernels, flags (ST_FLAG_TC_TF32 or ST_FLAG_TC_SPLIT) and shape limits as st_ttm_blockdiag; the
  * workspace is that of ST_OP_TTM_BLOCKDIAG. */
 st_status st_ttm_packed(const st_layout *layout, const float *Bp, const float *U, int64_t R,
                         float *Ap, void *ws, size_t ws_bytes, unsigned flags, void *stream);

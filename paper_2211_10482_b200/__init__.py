@@ -34,6 +34,7 @@ ST_OP_SYM_MOMENT2, ST_OP_SYM_MOMENT3, ST_OP_MTTKRP_TRI, ST_OP_TTM_BLOCKDIAG, ST_
 ST_FLAG_DENSE_CONTROL = 1
 ST_FLAG_TC_TF32 = 2
 ST_FLAG_TC_BF16 = 4
+ST_FLAG_TC_SPLIT = 8
 
 EXPORTS = [
     "st_packed_elems", "st_dense_elems", "st_pack", "st_unpack", "st_workspace_bytes", "st_sym_moment2",

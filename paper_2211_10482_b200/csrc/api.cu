@@ -6,6 +6,7 @@ size_t moment2_workspace(int64_t N, int64_t d, int xdt, unsigned flags);
 size_t moment3_workspace(int64_t N, int64_t d, unsigned flags);
 size_t moment4_workspace(int64_t N, int64_t d, unsigned flags);
 size_t ttm_tf32_tc_workspace(int64_t rows, int64_t K, int64_t R);
+size_t ttm_split_workspace(int64_t rows, int64_t K, int64_t R);
 size_t mttkrp_workspace(int64_t rows, int64_t I, int64_t K, int64_t R, unsigned flags);
 }  // namespace st
 
@@ -30,9 +31,11 @@ size_t st_workspace_bytes(st_op op, int64_t a, int64_t b, int64_t c, int64_t e, 
     }
     case ST_OP_TTM_BLOCKDIAG:
         if (a <= 0 || b <= 0 || c <= 0 || e <= 0) return 0;
-        if (flags & ST_FLAG_TC_TF32) {
+        if ((flags & ST_FLAG_TC_TF32) && (flags & ST_FLAG_TC_SPLIT)) return 0;
+        if (flags & (ST_FLAG_TC_TF32 | ST_FLAG_TC_SPLIT)) {
             const int64_t d = a * b;
-            return st::ttm_tf32_tc_workspace((flags & ST_FLAG_DENSE_CONTROL) ? d * d : a * b * b, c, e);
+            const int64_t rows = (flags & ST_FLAG_DENSE_CONTROL) ? d * d : a * b * b;
+            return (flags & ST_FLAG_TC_TF32) ? st::ttm_tf32_tc_workspace(rows, c, e) : st::ttm_split_workspace(rows, c, e);
         }
         return st::kWsHeaderBytes;
     default: return 0;

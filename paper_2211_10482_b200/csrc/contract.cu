@@ -26,6 +26,11 @@ st_status ttm_tf32_tc(const float *Bp, int64_t rows, int64_t K, const float *U, 
 st_status mttkrp_tf32_tc(const float *Bp, const MttkrpRows &m, int64_t K, const float *C, const float *D, int64_t R,
                          float *A_full, int64_t I_full, int64_t i_off, void *ws, size_t ws_bytes, cudaStream_t stream);
 size_t mttkrp_tf32_tc_workspace(int64_t rows, int64_t I, int64_t K, int64_t R);
+st_status ttm_split(const float *Bp, int64_t rows, int64_t K, const float *U, int64_t R, float *Ap, void *ws,
+                    size_t ws_bytes, cudaStream_t stream);
+st_status mttkrp_split(const float *Bp, const MttkrpRows &m, int64_t K, const float *C, const float *D, int64_t R,
+                       float *A_full, int64_t I_full, int64_t i_off, void *ws, size_t ws_bytes, cudaStream_t stream);
+size_t mttkrp_split_workspace(int64_t rows, int64_t I, int64_t K, int64_t R);
 
 // The fp32 kernels need no workspace; when the caller passes one anyway its status word is set to "ok".
 static inline unsigned *ws_status(void *ws, size_t ws_bytes)
@@ -378,7 +383,9 @@ static bool rowgemm_r_ok(int64_t R) { return R == 8 || R == 16 || R == 32 || R =
 size_t mttkrp_workspace(int64_t rows, int64_t I, int64_t K, int64_t R, unsigned flags)
 {
     if (rows <= 0 || I <= 0 || K <= 0 || R <= 0 || K % 4 != 0) return 0;
+    if ((flags & ST_FLAG_TC_TF32) && (flags & ST_FLAG_TC_SPLIT)) return 0;
     if (flags & ST_FLAG_TC_TF32) return mttkrp_tf32_tc_workspace(rows, I, K, R);
+    if (flags & ST_FLAG_TC_SPLIT) return mttkrp_split_workspace(rows, I, K, R);
     if (!rowgemm_r_ok(R)) return 0;
     const RgPlan p = rowgemm_plan(rows, K, R, true);
     return kWsHeaderBytes + (size_t)mttkrp_slots(rows, p.unit_rows, I, p.ksplit) * R * sizeof(float);
@@ -391,6 +398,8 @@ static st_status mttkrp_run(const float *Bp, const MttkrpRows &m, int64_t K, con
 {
     if (flags & ST_FLAG_TC_TF32)
         return mttkrp_tf32_tc(Bp, m, K, C, D, R, A_full, I_full, i_off, ws, ws_bytes, stream);
+    if (flags & ST_FLAG_TC_SPLIT)
+        return mttkrp_split(Bp, m, K, C, D, R, A_full, I_full, i_off, ws, ws_bytes, stream);
     if (!rowgemm_r_ok(R)) return ST_ERR_UNSUPPORTED;
     const size_t need = mttkrp_workspace(m.rows, m.I, K, R, flags);
     if (!ws || ws_bytes < need) return ST_ERR_WORKSPACE;
@@ -416,13 +425,15 @@ st_status st_ttm_blockdiag(const float *Bp, int64_t nblocks, int64_t bs, int64_t
     using namespace st;
     if (!Bp || !U || !Ap) return ST_ERR_NULL;
     if (nblocks <= 0 || bs <= 0 || K <= 0 || R <= 0) return ST_ERR_SHAPE;
-    if (flags & ~(ST_FLAG_DENSE_CONTROL | ST_FLAG_TC_TF32)) return ST_ERR_UNSUPPORTED;
+    if (flags & ~(ST_FLAG_DENSE_CONTROL | ST_FLAG_TC_TF32 | ST_FLAG_TC_SPLIT)) return ST_ERR_UNSUPPORTED;
+    if ((flags & ST_FLAG_TC_TF32) && (flags & ST_FLAG_TC_SPLIT)) return ST_ERR_UNSUPPORTED;
     if (!aligned16(Bp) || !aligned16(U) || !aligned16(Ap)) return ST_ERR_ALIGN;
     if (nblocks > (int64_t(1) << 24) || bs > (int64_t(1) << 15) || K > (1 << 20)) return ST_ERR_UNSUPPORTED;
     const int64_t d = nblocks * bs;
     const int64_t rows = (flags & ST_FLAG_DENSE_CONTROL) ? d * d : nblocks * bs * bs;
     if (rows / 256 + 1 > (int64_t(1) << 28)) return ST_ERR_UNSUPPORTED;
     if (flags & ST_FLAG_TC_TF32) return ttm_tf32_tc(Bp, rows, K, U, R, Ap, ws, ws_bytes, (cudaStream_t)stream);
+    if (flags & ST_FLAG_TC_SPLIT) return ttm_split(Bp, rows, K, U, R, Ap, ws, ws_bytes, (cudaStream_t)stream);
     if (K % 4 != 0) return ST_ERR_UNSUPPORTED;
     if (R != 8 && R != 16 && R != 32 && R != 64) return ST_ERR_UNSUPPORTED;
     RgArgs a{};
@@ -437,7 +448,8 @@ st_status st_ttm_packed(const st_layout *layout, const float *Bp, const float *U
     using namespace st;
     if (!layout || !Bp || !U || !Ap) return ST_ERR_NULL;
     if (R <= 0) return ST_ERR_SHAPE;
-    if (flags & ~(ST_FLAG_TC_TF32)) return ST_ERR_UNSUPPORTED;
+    if (flags & ~(ST_FLAG_TC_TF32 | ST_FLAG_TC_SPLIT)) return ST_ERR_UNSUPPORTED;
+    if ((flags & ST_FLAG_TC_TF32) && (flags & ST_FLAG_TC_SPLIT)) return ST_ERR_UNSUPPORTED;
     if (!aligned16(Bp) || !aligned16(U) || !aligned16(Ap)) return ST_ERR_ALIGN;
     const int64_t K = layout->inner;
     const int64_t elems = st_packed_elems(layout);      // validates the layout
@@ -445,6 +457,7 @@ st_status st_ttm_packed(const st_layout *layout, const float *Bp, const float *U
     const int64_t rows = elems / K;                      // one fibre along k per packed position
     if (K > (1 << 20) || rows / 256 + 1 > (int64_t(1) << 28)) return ST_ERR_UNSUPPORTED;
     if (flags & ST_FLAG_TC_TF32) return ttm_tf32_tc(Bp, rows, K, U, R, Ap, ws, ws_bytes, (cudaStream_t)stream);
+    if (flags & ST_FLAG_TC_SPLIT) return ttm_split(Bp, rows, K, U, R, Ap, ws, ws_bytes, (cudaStream_t)stream);
     if (K % 4 != 0) return ST_ERR_UNSUPPORTED;
     if (R != 8 && R != 16 && R != 32 && R != 64) return ST_ERR_UNSUPPORTED;
     RgArgs a{};
@@ -459,7 +472,8 @@ st_status st_mttkrp_tri(const float *Bp, int64_t I, int64_t K, const float *C, c
     using namespace st;
     if (!Bp || !C || !D || !A) return ST_ERR_NULL;
     if (I <= 0 || K <= 0 || R <= 0) return ST_ERR_SHAPE;
-    if (flags & ~(ST_FLAG_DENSE_CONTROL | ST_FLAG_TC_TF32)) return ST_ERR_UNSUPPORTED;
+    if (flags & ~(ST_FLAG_DENSE_CONTROL | ST_FLAG_TC_TF32 | ST_FLAG_TC_SPLIT)) return ST_ERR_UNSUPPORTED;
+    if ((flags & ST_FLAG_TC_TF32) && (flags & ST_FLAG_TC_SPLIT)) return ST_ERR_UNSUPPORTED;
     if (!aligned16(Bp) || !aligned16(C) || !aligned16(D) || !aligned16(A)) return ST_ERR_ALIGN;
     if (I > (1 << 15) || K > (1 << 20) || K % 4 != 0) return ST_ERR_UNSUPPORTED;
     const bool dense = (flags & ST_FLAG_DENSE_CONTROL) != 0;
@@ -479,7 +493,8 @@ st_status st_mttkrp_slice(const float *Bp, int64_t I, int64_t J, int64_t K, int6
     if (!Bp || !C || !D || !A) return ST_ERR_NULL;
     if (I <= 0 || J <= 0 || K <= 0 || R <= 0) return ST_ERR_SHAPE;
     if (fixed_i >= I || fixed_j >= J || (fixed_i < 0 && fixed_j < 0)) return ST_ERR_SHAPE;
-    if (flags & ~(ST_FLAG_TC_TF32)) return ST_ERR_UNSUPPORTED;
+    if (flags & ~(ST_FLAG_TC_TF32 | ST_FLAG_TC_SPLIT)) return ST_ERR_UNSUPPORTED;
+    if ((flags & ST_FLAG_TC_TF32) && (flags & ST_FLAG_TC_SPLIT)) return ST_ERR_UNSUPPORTED;
     if (!aligned16(Bp) || !aligned16(C) || !aligned16(D) || !aligned16(A)) return ST_ERR_ALIGN;
     if (I > (1 << 24) || J > (1 << 24) || K > (1 << 20) || K % 4 != 0 || R % 4 != 0) return ST_ERR_UNSUPPORTED;
     // The fibres of the slice are the packed rows.  With (i, j) = (row / div, row % div):

@@ -54,6 +54,51 @@ __device__ __forceinline__ float warp_transpose_sum32(float (&v)[32], int lane)
 #undef ST_TR_STEP
     return v[0];
 }
+
+// How the fibres of a warp (one per lane, consecutive rows) fall into runs of equal i.
+struct WarpRuns {
+    unsigned heads;      // lanes that start a run
+    unsigned vmask;      // lanes that hold a fibre
+};
+__device__ __forceinline__ WarpRuns warp_runs(bool valid, int gi32, int lane)
+{
+    WarpRuns w;
+    const int prev = __shfl_up_sync(0xffffffffu, gi32, 1);
+    w.heads = __ballot_sync(0xffffffffu, valid && (lane == 0 || prev != gi32));
+    w.vmask = __ballot_sync(0xffffffffu, valid);
+    return w;
+}
+
+// Writes the sums of the warp's runs for the 32 columns c0.. held in v (v[c] = C[j,c0+c] * Y[fibre,c0+c],
+// zeros in lanes without a fibre) to the partial slots (unit + i).  Call with all 32 lanes.
+__device__ __forceinline__ void warp_store_runs(float (&v)[32], const WarpRuns &w, bool valid, int gi32, int64_t unit,
+                                                int lane, float *part, int R, int c0)
+{
+    if (w.heads == 0u) return;                 // no fibre in this warp
+    if (w.heads == 1u) {                       // one run: the whole warp
+        const float sum = warp_transpose_sum32(v, lane);
+        part[(unit + __shfl_sync(0xffffffffu, gi32, 0)) * R + c0 + lane] = sum;
+    } else if (w.heads == w.vmask) {           // every fibre is a run of its own
+        if (valid) {
+            float4 *dst = reinterpret_cast<float4 *>(part + (unit + gi32) * R + c0);
+#pragma unroll
+            for (int e = 0; e < 8; ++e) dst[e] = make_float4(v[4 * e], v[4 * e + 1], v[4 * e + 2], v[4 * e + 3]);
+        }
+    } else {                                   // several runs: one masked reduction per run
+        unsigned h = w.heads;
+        while (h) {
+            const int s0 = __ffs(h) - 1;
+            h &= h - 1;
+            const int s1 = h ? __ffs(h) - 1 : 32;
+            const bool in = lane >= s0 && lane < s1;
+            float t[32];
+#pragma unroll
+            for (int e = 0; e < 32; ++e) t[e] = in ? v[e] : 0.f;
+            const float sum = warp_transpose_sum32(t, lane);
+            part[(unit + __shfl_sync(0xffffffffu, gi32, s0)) * R + c0 + lane] = sum;
+        }
+    }
+}
 #endif
 
 }  // namespace st

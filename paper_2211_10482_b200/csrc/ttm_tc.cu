@@ -208,11 +208,9 @@ ttm_tc_kernel(const __grid_constant__ CUtensorMap tmap, const TtmTcArgs a)
                     else { gi = row / a.div; gj = row - gi * a.div; }
                 }
                 const int gi32 = (int)gi;
-                const int prev = __shfl_up_sync(0xffffffffu, gi32, 1);
-                const unsigned heads = __ballot_sync(0xffffffffu, valid && (lane == 0 || prev != gi32));
-                const unsigned vmask = __ballot_sync(0xffffffffu, valid);
+                const WarpRuns runs = warp_runs(valid, gi32, lane);
                 const int64_t unit = tile * (BM / 32) + q;
-                for (int c0 = 0; c0 < a.R && heads != 0u; c0 += 32) {
+                for (int c0 = 0; c0 < a.R && runs.heads != 0u; c0 += 32) {
                     uint32_t r[32];
                     tmem_ld_32x32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * a.R + c0), r);
                     tmem_ld_wait();
@@ -231,29 +229,7 @@ ttm_tc_kernel(const __grid_constant__ CUtensorMap tmap, const TtmTcArgs a)
 #pragma unroll
                         for (int e = 0; e < 32; ++e) v[e] = 0.f;
                     }
-                    if (heads == 1u) {                     // one run: the whole warp
-                        const float sum = warp_transpose_sum32(v, lane);
-                        a.out[(unit + __shfl_sync(0xffffffffu, gi32, 0)) * a.R + c0 + lane] = sum;
-                    } else if (heads == vmask) {           // every fibre is a run of its own
-                        if (valid) {
-                            float4 *dst = reinterpret_cast<float4 *>(a.out + (unit + gi) * a.R + c0);
-#pragma unroll
-                            for (int e = 0; e < 8; ++e) dst[e] = make_float4(v[4 * e], v[4 * e + 1], v[4 * e + 2], v[4 * e + 3]);
-                        }
-                    } else {                               // several runs: one masked reduction per run
-                        unsigned h = heads;
-                        while (h) {
-                            const int s0 = __ffs(h) - 1;
-                            h &= h - 1;
-                            const int s1 = h ? __ffs(h) - 1 : 32;
-                            const bool in = lane >= s0 && lane < s1;
-                            float w[32];
-#pragma unroll
-                            for (int e = 0; e < 32; ++e) w[e] = in ? v[e] : 0.f;
-                            const float sum = warp_transpose_sum32(w, lane);
-                            a.out[(unit + __shfl_sync(0xffffffffu, gi32, s0)) * a.R + c0 + lane] = sum;
-                        }
-                    }
+                    warp_store_runs(v, runs, valid, gi32, unit, lane, a.out, a.R, c0);
                 }
             }
             tc_fence_before();

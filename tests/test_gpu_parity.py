@@ -267,6 +267,8 @@ def test_fixed_order_calls_give_the_same_bits_twenty_times(st):
         "ttm_tf32": lambda: st.st_ttm_blockdiag(Bq, U, 3, 16, flags=st.ST_FLAG_TC_TF32),
         "mttkrp": lambda: st.st_mttkrp_tri(Bp, C, D),
         "mttkrp_tf32": lambda: st.st_mttkrp_tri(Bp, C, D, flags=st.ST_FLAG_TC_TF32),
+        "ttm_split": lambda: st.st_ttm_blockdiag(Bq, U, 3, 16, flags=st.ST_FLAG_TC_SPLIT),
+        "mttkrp_split": lambda: st.st_mttkrp_tri(Bp, C, D, flags=st.ST_FLAG_TC_SPLIT),
     }
     for name, fn in calls.items():
         first = fn().clone()
@@ -664,6 +666,71 @@ def test_ttm_tf32_sixteen_columns_many_tiles(st):
     assert st.st_check_status() == st.ST_OK
 
 
+# split-bf16 tensor-core path of TTM and MTTKRP: both operands as hi + lo bf16 parts, three partial
+# products: held to the fp32 tolerance
+
+@pytest.mark.parametrize("nb,bs,K,R", [(1, 1, 4, 32), (3, 2, 8, 32), (2, 5, 36, 32), (4, 8, 64, 64), (7, 3, 32, 96),
+                                       (2, 17, 100, 128), (5, 12, 256, 64), (3, 9, 520, 32), (1, 40, 1024, 32)])
+def test_ttm_split_tensor_core_small(st, nb, bs, K, R):
+    Bp, U = workloads.ttm_inputs(nb, bs, K, R)
+    A, S = oracle.ttm(Bp.reshape(-1, K), U)
+    got = st.st_ttm_blockdiag(dev(Bp), dev(U), nb, bs, flags=st.ST_FLAG_TC_SPLIT).cpu().numpy()
+    assert st.st_check_status() == st.ST_OK
+    assert oracle.rel_err(got, A, S) <= TOL_F32
+
+
+def test_ttm_split_many_tiles_both_accumulators_and_limits(st):
+    nb, bs, K, R = 5, 72, 96, 32          # 25,920 fibres = 203 tiles: every block uses both accumulator buffers
+    Bp, U = workloads.ttm_inputs(nb, bs, K, R)
+    A, S = oracle.ttm(Bp.reshape(-1, K), U)
+    got = st.st_ttm_blockdiag(dev(Bp), dev(U), nb, bs, flags=st.ST_FLAG_TC_SPLIT).cpu().numpy()
+    assert st.st_check_status() == st.ST_OK
+    assert oracle.rel_err(got, A, S) <= TOL_F32
+    # all-positive operands: the worst case for a rounding bias of the accumulation
+    Bpos, Upos = np.abs(Bp) + 0.5, np.abs(U) + 0.5
+    A, S = oracle.ttm(Bpos.reshape(-1, K), Upos)
+    got = st.st_ttm_blockdiag(dev(Bpos), dev(Upos), nb, bs, flags=st.ST_FLAG_TC_SPLIT).cpu().numpy()
+    assert oracle.rel_err(got, A, S) <= TOL_F32
+    # shapes the path does not take, and the two tensor-core flags together
+    L, s = st.lib(), torch.cuda.current_stream().cuda_stream
+    x = torch.zeros(1 << 20, device="cuda")
+    ws = guarded(st, 4096, torch.uint8)
+    SP = st.ST_FLAG_TC_SPLIT
+    assert L.st_ttm_blockdiag(x.data_ptr(), 2, 2, 8, x.data_ptr(), 48, x.data_ptr(), ws.data_ptr(), 4096, SP, s) == st.ST_ERR_UNSUPPORTED
+    assert L.st_ttm_blockdiag(x.data_ptr(), 2, 2, 4096, x.data_ptr(), 32, x.data_ptr(), ws.data_ptr(), 4096, SP, s) == st.ST_ERR_UNSUPPORTED
+    assert L.st_ttm_blockdiag(x.data_ptr(), 2, 2, 8, x.data_ptr(), 32, x.data_ptr(), ws.data_ptr(), 4096,
+                              SP | st.ST_FLAG_TC_TF32, s) == st.ST_ERR_UNSUPPORTED
+    assert st.st_workspace_bytes(st.ST_OP_TTM_BLOCKDIAG, 2, 2, 8, 48, SP) == 0
+
+
+def test_ttm_split_config(st, ttm_config_oracle):
+    Bp, U, A, S = ttm_config_oracle
+    got = st.st_ttm_blockdiag(dev(Bp), dev(U), 64, 64, flags=st.ST_FLAG_TC_SPLIT).cpu().numpy()
+    assert st.st_check_status() == st.ST_OK
+    assert oracle.rel_err(got, A, S) <= TOL_F32          # every fibre, every column, at the fp32 tolerance
+
+
+@pytest.mark.parametrize("I,K,R", [(1, 4, 32), (5, 36, 32), (16, 64, 64), (40, 100, 32), (70, 32, 96), (33, 68, 64),
+                                   (130, 8, 128)])
+def test_mttkrp_split_tensor_core_small(st, I, K, R):
+    Bp, C, D = workloads.mttkrp_inputs(I, K, R)
+    Bd = oracle.unpack(Bp.reshape(-1), oracle.KIND_TRI, I, inner=K)
+    A, S = oracle.mttkrp(Bd, C, D)
+    got = st.st_mttkrp_tri(dev(Bp), dev(C), dev(D), flags=st.ST_FLAG_TC_SPLIT).cpu().numpy()
+    assert st.st_check_status() == st.ST_OK
+    assert oracle.rel_err(got, A, S) <= TOL_F32
+    ctl = st.st_mttkrp_tri(dev(Bd), dev(C), dev(D), flags=st.ST_FLAG_TC_SPLIT | st.ST_FLAG_DENSE_CONTROL).cpu().numpy()
+    assert oracle.rel_err(ctl, A, S) <= TOL_F32
+
+
+def test_mttkrp_split_config(st, mttkrp_config_oracle):
+    Bp, C, D, A, S = mttkrp_config_oracle
+    got = st.st_mttkrp_tri(dev(Bp), dev(C), dev(D), flags=st.ST_FLAG_TC_SPLIT)
+    assert st.st_check_status() == st.ST_OK
+    assert oracle.rel_err(got.cpu().numpy(), A, S) <= TOL_F32      # every (i, r), at the fp32 tolerance
+    assert torch.equal(got, st.st_mttkrp_tri(dev(Bp), dev(C), dev(D), flags=st.ST_FLAG_TC_SPLIT))
+
+
 def test_moment2_bf16_all_tiles_midsize(st):
     """d = 1024 (all 20 launched tiles, both diagonal and off-diagonal kinds) at a sample count
     the oracle can still check on sampled entries quickly; input 256 MiB, larger than L2."""
@@ -715,9 +782,10 @@ def _okind(st, lay):
             st.ST_BLOCKDIAG: oracle.KIND_BLOCKDIAG}[lay.kind]
 
 
-@pytest.mark.parametrize("flag_name,K,R", [("f32", 36, 32), ("f32", 64, 8), ("tf32", 64, 32), ("tf32", 36, 48)])
+@pytest.mark.parametrize("flag_name,K,R", [("f32", 36, 32), ("f32", 64, 8), ("tf32", 64, 32), ("tf32", 36, 48),
+                                           ("split", 36, 32), ("split", 64, 64)])
 def test_ttm_on_every_structure_of_the_first_two_modes(st, flag_name, K, R):
-    flags = st.ST_FLAG_TC_TF32 if flag_name == "tf32" else 0
+    flags = {"tf32": st.ST_FLAG_TC_TF32, "split": st.ST_FLAG_TC_SPLIT, "f32": 0}[flag_name]
     for n, lay in enumerate(_table1_layouts(st, K)):
         rows = st.st_packed_elems(lay) // K
         Bp = workloads.draw((rows, K), "normal", 800 + n)
@@ -733,7 +801,7 @@ def test_ttm_on_every_structure_of_the_first_two_modes(st, flag_name, K, R):
         scale = oracle.pack(S, _okind(st, lay), lay.d, inner=R, **okw(lay)).reshape(rows, R)
         got = st.st_ttm_packed(dev(Bp), dev(U), lay, flags=flags).cpu().numpy()
         assert st.st_check_status() == st.ST_OK
-        assert oracle.rel_err(got, want, scale) <= (5e-3 if flags else TOL_F32), (flag_name, n)
+        assert oracle.rel_err(got, want, scale) <= (5e-3 if flag_name == "tf32" else TOL_F32), (flag_name, n)
         # everything outside the structure of the dense result is exactly zero (output keeps B's structure)
         mask = oracle.unpack(np.ones(rows * R, np.float32), _okind(st, lay), lay.d, inner=R, **okw(lay))
         assert np.all(A[mask == 0] == 0)
@@ -760,10 +828,11 @@ def test_thp_structured_times_dense(st):
 
 
 @pytest.mark.parametrize("flag_name,I,J,K,R", [("f32", 5, 7, 36, 32), ("f32", 300, 40, 64, 8), ("f32", 33, 700, 32, 64),
-                                               ("tf32", 5, 7, 36, 32), ("tf32", 300, 260, 64, 64), ("tf32", 1, 1, 4, 32)])
+                                               ("tf32", 5, 7, 36, 32), ("tf32", 300, 260, 64, 64), ("tf32", 1, 1, 4, 32),
+                                               ("split", 5, 7, 36, 32), ("split", 300, 260, 64, 64)])
 def test_mttkrp_on_slice_structures(st, flag_name, I, J, K, R):
-    flags = st.ST_FLAG_TC_TF32 if flag_name == "tf32" else 0
-    tol = 5e-3 if flags else TOL_F32
+    flags = {"tf32": st.ST_FLAG_TC_TF32, "split": st.ST_FLAG_TC_SPLIT, "f32": 0}[flag_name]
+    tol = 5e-3 if flag_name == "tf32" else TOL_F32
     C = workloads.draw((J, R), "uniform", 1100)
     D = workloads.draw((K, R), "uniform", 1101)
     i0, j0 = I // 2, J - 1
