@@ -76,7 +76,7 @@ typedef enum { ST_OP_SYM_MOMENT2 = 0, ST_OP_SYM_MOMENT3 = 1, ST_OP_MTTKRP_TRI = 
                                     both operands split into two bf16 parts and three of the four partial products
                                     kept: meets the 1e-4 tolerance of the fp32 path, at the speed of the HBM stream
                                     (needs K % 4 == 0, R % 32 == 0, R <= 128, and the split factor, 4*K*R bytes rounded up to
-                                    whole chunks of 64 k-values, in shared memory: K*R <= 40960; not with
+                                    whole chunks of 64 k-values, in shared memory: K*R <= 24576; not with
                                     ST_FLAG_TC_TF32) */
 
 typedef struct {

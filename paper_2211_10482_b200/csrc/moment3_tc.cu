@@ -71,17 +71,6 @@ struct Args {
 // index has (row & 7) == m
 __device__ __forceinline__ uint32_t swz(int lane, int m) { return (uint32_t)((((lane >> 2) ^ m) << 4) + ((lane & 3) << 2)); }
 
-__device__ __forceinline__ void tmem_ld_32x16(uint32_t taddr, uint32_t *r)
-{
-    asm volatile(
-        "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
-        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
-        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
-          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
-        : "r"(taddr)
-        : "memory");
-}
-
 template <bool BF16>
 __global__ void __launch_bounds__(THREADS, 1)
 moment3_tc_kernel(const __grid_constant__ Args a)

@@ -55,6 +55,23 @@ __device__ __forceinline__ float warp_transpose_sum32(float (&v)[32], int lane)
     return v[0];
 }
 
+// The same for 16 columns: every lane ends with the sum of column (lane % 16) over the warp.
+__device__ __forceinline__ float warp_transpose_sum16(float (&v)[16], int lane)
+{
+#define ST_TR_STEP(OFF)                                                                       \
+    {                                                                                         \
+        const bool up = (lane & OFF) != 0;                                                    \
+        _Pragma("unroll") for (int j = 0; j < OFF; ++j) {                                     \
+            const float send = up ? v[j] : v[j + OFF];                                        \
+            const float keep = up ? v[j + OFF] : v[j];                                        \
+            v[j] = keep + __shfl_xor_sync(0xffffffffu, send, OFF);                            \
+        }                                                                                     \
+    }
+    ST_TR_STEP(8) ST_TR_STEP(4) ST_TR_STEP(2) ST_TR_STEP(1)
+#undef ST_TR_STEP
+    return v[0] + __shfl_xor_sync(0xffffffffu, v[0], 16);
+}
+
 // How the fibres of a warp (one per lane, consecutive rows) fall into runs of equal i.
 struct WarpRuns {
     unsigned heads;      // lanes that start a run
@@ -96,6 +113,38 @@ __device__ __forceinline__ void warp_store_runs(float (&v)[32], const WarpRuns &
             for (int e = 0; e < 32; ++e) t[e] = in ? v[e] : 0.f;
             const float sum = warp_transpose_sum32(t, lane);
             part[(unit + __shfl_sync(0xffffffffu, gi32, s0)) * R + c0 + lane] = sum;
+        }
+    }
+}
+
+// The same for the 16 columns c0.. held in v.
+__device__ __forceinline__ void warp_store_runs16(float (&v)[16], const WarpRuns &w, bool valid, int gi32, int64_t unit,
+                                                  int lane, float *part, int R, int c0)
+{
+    if (w.heads == 0u) return;
+    if (w.heads == 1u) {
+        const float sum = warp_transpose_sum16(v, lane);
+        const int gi0 = __shfl_sync(0xffffffffu, gi32, 0);
+        if (lane < 16) part[(unit + gi0) * R + c0 + lane] = sum;
+    } else if (w.heads == w.vmask) {
+        if (valid) {
+            float4 *dst = reinterpret_cast<float4 *>(part + (unit + gi32) * R + c0);
+#pragma unroll
+            for (int e = 0; e < 4; ++e) dst[e] = make_float4(v[4 * e], v[4 * e + 1], v[4 * e + 2], v[4 * e + 3]);
+        }
+    } else {
+        unsigned h = w.heads;
+        while (h) {
+            const int s0 = __ffs(h) - 1;
+            h &= h - 1;
+            const int s1 = h ? __ffs(h) - 1 : 32;
+            const bool in = lane >= s0 && lane < s1;
+            float t[16];
+#pragma unroll
+            for (int e = 0; e < 16; ++e) t[e] = in ? v[e] : 0.f;
+            const float sum = warp_transpose_sum16(t, lane);
+            const int gis = __shfl_sync(0xffffffffu, gi32, s0);
+            if (lane < 16) part[(unit + gis) * R + c0 + lane] = sum;
         }
     }
 }

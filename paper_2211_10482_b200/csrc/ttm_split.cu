@@ -10,16 +10,19 @@
 // accepts: it is held to the 1e-4 tolerance of the fp32 kernels.  HBM bound (the fp32 FMA kernel of
 // the same contraction is bound by arithmetic at more than twice the time).
 //
-// Persistent blocks walk tiles of 128 fibres.  Eight converter warps read the fibres straight from
-// global memory (coalesced 16-byte loads, the next slice of 64 k-values in flight while the current
-// one is converted), split them and store hi and lo as two K-major, 128-byte-swizzled bf16 operands.
-// W is split once per block into [Wh; Wl] stacked along N.  Per 16 k-values the issuing thread runs
+// Persistent blocks walk tiles of 128 fibres.  Sixteen converter warps copy slices of 64 k-values
+// asynchronously into a landing ring (16-byte copies, every thread later reads back the chunks it
+// copied itself: no barrier), split them and store hi and lo as two K-major, 128-byte-swizzled bf16
+// operands.  (Asking for whole tiles to be brought into L2 ahead of the copies, so that DRAM would see
+// long sequential reads, was measured and made the kernel 12-20 % slower.)  W is split once per block into [Wh; Wl] stacked along N.  Per 16
+// k-values the issuing thread runs
 //     D[128 x 2R] += Bh x [Wh; Wl]^T     (N = 2R)
 //     D[128 x  R] += Bl x  Wh^T          (N = R, the first R columns of the same accumulator)
 // so the two products with Bh cost one instruction (an MMA of M = 128 takes the same time for any
 // N <= 128).  The epilogue adds the two halves of the accumulator, D[:, r] + D[:, R + r]; it is
 // double buffered in tensor memory.  Warps 0-3 epilogue (and the split of W), warp 4 MMA issue and
-// tensor-memory owner, warps 5-12 converters.
+// tensor-memory owner, warps 5-20 converters (what bounds them is the latency of the chain copy ->
+// convert -> store -> proxy fence -> barrier, so there are four of them per scheduler).
 #include "tc_common.cuh"
 #include "st_index.cuh"
 #include "mttkrp_common.cuh"
@@ -33,10 +36,12 @@ constexpr int KC = 64;                     // k-values per operand stage (128 by
 constexpr int OP_BYTES = BM * 128;         // one operand (hi or lo) of a stage: 16 KiB
 constexpr int STAGE_BYTES = 2 * OP_BYTES;  // hi + lo
 constexpr int MAX_STAGES = 4;
-constexpr int EPI_WARPS = 4, MMA_WARP = 4, CONV_WARP0 = 5, CONV_WARPS = 8;
+constexpr int EPI_WARPS = 4, MMA_WARP = 4, CONV_WARP0 = 5, CONV_WARPS = 16;
 constexpr int CONV_THREADS = 32 * CONV_WARPS;
 constexpr int THREADS = 32 * (CONV_WARP0 + CONV_WARPS);
-constexpr int LOADS = BM * (KC / 4) / CONV_THREADS;   // 16-byte loads per converter thread and stage: 8
+constexpr int LOADS = BM * (KC / 4) / CONV_THREADS;   // 16-byte copies per converter thread and stage: 4
+constexpr int ROW_STEP = CONV_THREADS / 16;           // fibres between two copies of a thread: 32
+constexpr int LAND_BYTES = BM * KC * 4;     // one stage of the landing ring of the fp32 data: 32 KiB
 constexpr int MAX_K = 2048;                // longest accumulation chain: 3 * 2048 / 16 = 384 instructions
 }  // namespace split
 
@@ -54,6 +59,12 @@ struct SplitArgs {
     int K, R, kchunks, ntiles, stages;
     uint32_t tmem_cols;
 };
+struct SplitPlan {
+    int kchunks, stages, land;
+    uint32_t tmem_cols;
+    size_t smem;
+    bool ok;
+};
 
 // two floats -> two bf16 in one word (first argument in the low half)
 __device__ __forceinline__ uint32_t bf16x2(float lo, float hi)
@@ -70,6 +81,8 @@ __device__ __forceinline__ void split2(float x0, float x1, uint32_t &hi, uint32_
     lo = bf16x2(x0 - h0, x1 - h1);
 }
 
+// LAND: stages of the landing ring (3 when shared memory has room beside W, else 2)
+template <int LAND>
 __global__ void __launch_bounds__(split::THREADS, 1) ttm_split_kernel(const SplitArgs a)
 {
     using namespace split;
@@ -115,14 +128,50 @@ __global__ void __launch_bounds__(split::THREADS, 1) ttm_split_kernel(const Spli
     const int my_tiles = (a.ntiles > (int)blockIdx.x) ? (a.ntiles - 1 - (int)blockIdx.x) / (int)gridDim.x + 1 : 0;
     const int R = a.R;
 
-    if (warp < EPI_WARPS) {
-        // ---- split W: chunk kc of 64 k-values becomes 2R rows of 128 bytes, row r = Wh[., r], row R + r =
-        // Wl[., r], K-major with the 128-byte swizzle (16-byte unit u of row n sits at unit u ^ (n & 7)).
-        // A warp takes (chunk, 16 columns r): lane = (4 columns rg, unit q of 8 k-values); it loads the
-        // float4 W[8q + e, 4rg ..] for e = 0..7 (64 contiguous bytes per k across the 4 rg lanes) and
-        // stores one 16-byte unit per column and part (the 8 lanes q of a column fill one 128-byte row).
+    // ---- converter set-up (used again in the converter branch below).  Copy u of a thread covers fibre
+    // (ct / 16 + 32 u) of the tile and the four k-values 4 * (ct % 16) of the chunk: the 16 lanes of a
+    // half-warp copy one fibre's 256 contiguous bytes and later write its 128-byte row of each operand.
+    // The fp32 data travel global -> shared by asynchronous 16-byte copies into a landing ring of LAND
+    // stages; every thread reads back exactly the chunks it copied itself, so the ring needs no barrier,
+    // only the thread's own wait on its copy groups.  LAND - 1 stages are in flight per block while one
+    // is converted.
+    const int ct = threadIdx.x - 32 * CONV_WARP0;
+    const int g = ct & 15, r_base = ct >> 4;                          // rows r_base + 32 u
+    const int64_t total = (int64_t)my_tiles * a.kchunks;
+    const uint32_t land0 = smem_u32(stage0 + (size_t)a.stages * STAGE_BYTES + 256) + (uint32_t)ct * 16u;
+    auto load = [&](int64_t it) {
+        if (it < total) {
+            const int t = (int)(it / a.kchunks), kc = (int)(it - (int64_t)t * a.kchunks);
+            const int64_t tile = blockIdx.x + (int64_t)t * gridDim.x;
+            const int k = kc * KC + g * 4;
+            const int64_t row0 = tile * BM + r_base;
+            const float *src = a.B + row0 * (int64_t)a.K + k;
+            const uint32_t dst = land0 + (uint32_t)(it % LAND) * (uint32_t)LAND_BYTES;
+#pragma unroll
+            for (int u = 0; u < LOADS; ++u) {
+                const bool in = row0 + ROW_STEP * u < a.rows && k < a.K;
+                const int sz = in ? 16 : 0;                          // src-size 0: the 16 bytes are zero-filled
+                asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst + (uint32_t)u * (CONV_THREADS * 16u)),
+                             "l"(in ? src + (int64_t)(ROW_STEP * u) * a.K : a.B), "r"(sz)
+                             : "memory");
+            }
+        }
+        asm volatile("cp.async.commit_group;" ::: "memory");           // one group per stage, empty past the end
+    };
+    // the first slices are requested before anything else, so that they travel while W is split
+    if (warp >= CONV_WARP0)
+        for (int p = 0; p < LAND; ++p) load(p);
+
+    if (warp != MMA_WARP) {
+        // ---- split W (all warps but the issuer: one cold round trip to memory each): chunk kc of 64 k-values
+        // becomes 2R rows of 128 bytes, row r = Wh[., r], row R + r = Wl[., r], K-major with the 128-byte
+        // swizzle (16-byte unit u of row n sits at unit u ^ (n & 7)).  A warp takes (chunk, 16 columns r):
+        // lane = (4 columns rg, unit q of 8 k-values); it loads the float4 W[8q + e, 4rg ..] for e = 0..7
+        // (64 contiguous bytes per k across the 4 rg lanes) and stores one 16-byte unit per column and part
+        // (the 8 lanes q of a column fill one 128-byte row).
         const int items = a.kchunks * (R / 16);
-        for (int it = warp; it < items; it += EPI_WARPS) {
+        const int wi = warp < MMA_WARP ? warp : warp - 1;
+        for (int it = wi; it < items; it += EPI_WARPS + CONV_WARPS) {
             const int kc = it / (R / 16), r0 = (it - kc * (R / 16)) * 16 + (lane >> 3) * 4;
             const int q = lane & 7, k0 = kc * KC + q * 8;
             float4 v[8];
@@ -146,57 +195,81 @@ __global__ void __launch_bounds__(split::THREADS, 1) ttm_split_kernel(const Spli
             }
         }
         fence_proxy_async();      // make the generic-proxy writes of W visible to the tensor core
-        asm volatile("bar.sync 1, %0;" ::"n"(32 * (EPI_WARPS + 1)) : "memory");
+    }
+    __syncthreads();              // W is in place
 
+    if (warp < EPI_WARPS) {
         // ---- epilogue
         const int q = warp;       // TMEM lanes 32q .. 32q + 31
         for (int t = 0; t < my_tiles; ++t) {
             const int buf = t & 1;
             const int64_t tile = blockIdx.x + (int64_t)t * gridDim.x;
-            if (!mbar_wait(&acc_full[buf], (uint32_t)((t >> 1) & 1), abort_flag, a.status, 4)) break;
-            tc_fence_after();
             const int64_t row = tile * BM + q * 32 + lane;
             const bool valid = row < a.rows;
-            const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * 2 * R);
+            // MTTKRP: the fibre's (i, j) and, for R = 32, its row of C are fetched before the accumulator is
+            // waited for -- with the memory system saturated by the fibre stream a dependent load costs
+            // microseconds, which would otherwise stall the tile after next
             int64_t gi = -1, gj = 0;
             WarpRuns runs{0u, 0u};
+            float4 cpre[8];
+            const bool pre = a.mode != SP_TTM && R == 32;
             if (a.mode != SP_TTM) {
                 if (valid) {
                     if (a.mode == SP_MTTKRP_PACKED) tri_decode(a.I, row, gi, gj);
                     else { gi = row / a.div; gj = row - gi * a.div; }
                 }
                 runs = warp_runs(valid, (int)gi, lane);
-            }
-            for (int c0 = 0; c0 < R; c0 += 32) {
-                uint32_t r1[32], r2[32];
-                tmem_ld_32x32(taddr + (uint32_t)c0, r1);
-                tmem_ld_32x32(taddr + (uint32_t)(R + c0), r2);
-                tmem_ld_wait();
-                float v[32];
+                if (pre) {
 #pragma unroll
-                for (int e = 0; e < 32; ++e) v[e] = __uint_as_float(r1[e]) + __uint_as_float(r2[e]);
+                    for (int e = 0; e < 8; ++e)
+                        cpre[e] = valid ? __ldg(reinterpret_cast<const float4 *>(a.C + gj * R) + e) : make_float4(0.f, 0.f, 0.f, 0.f);
+                }
+            }
+            if (!mbar_wait(&acc_full[buf], (uint32_t)((t >> 1) & 1), abort_flag, a.status, 4)) break;
+            tc_fence_after();
+            const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * 2 * R);
+            // 16 columns at a time keeps the register count low; cv = the fibre's four float4 of C for them
+            auto chunk = [&](int c0, const float4 &cv0, const float4 &cv1, const float4 &cv2, const float4 &cv3) {
+                float v[16];
+                {
+                    uint32_t r1[16], r2[16];
+                    tmem_ld_32x16(taddr + (uint32_t)c0, r1);
+                    tmem_ld_32x16(taddr + (uint32_t)(R + c0), r2);
+                    tmem_ld_wait();
+#pragma unroll
+                    for (int e = 0; e < 16; ++e) v[e] = __uint_as_float(r1[e]) + __uint_as_float(r2[e]);
+                }
                 if (a.mode == SP_TTM) {
                     if (valid) {
                         float4 *dst = reinterpret_cast<float4 *>(a.out + row * R + c0);
 #pragma unroll
-                        for (int e = 0; e < 8; ++e) dst[e] = make_float4(v[4 * e], v[4 * e + 1], v[4 * e + 2], v[4 * e + 3]);
+                        for (int e = 0; e < 4; ++e) dst[e] = make_float4(v[4 * e], v[4 * e + 1], v[4 * e + 2], v[4 * e + 3]);
                     }
                 } else {
-                    if (valid) {
+                    const float4 cv[4] = {cv0, cv1, cv2, cv3};
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {            // lanes without a fibre hold zeros in cv
+                        v[4 * e + 0] *= cv[e].x;
+                        v[4 * e + 1] *= cv[e].y;
+                        v[4 * e + 2] *= cv[e].z;
+                        v[4 * e + 3] *= cv[e].w;
+                    }
+                    warp_store_runs16(v, runs, valid, (int)gi, tile * (BM / 32) + q, lane, a.out, R, c0);
+                }
+            };
+            if (pre) {
+                chunk(0, cpre[0], cpre[1], cpre[2], cpre[3]);
+                chunk(16, cpre[4], cpre[5], cpre[6], cpre[7]);
+            } else {
+                const float4 z = make_float4(0.f, 0.f, 0.f, 0.f);
+                for (int c0 = 0; c0 < R; c0 += 16) {
+                    float4 cv[4] = {z, z, z, z};
+                    if (a.mode != SP_TTM && valid) {
                         const float4 *crow = reinterpret_cast<const float4 *>(a.C + gj * R + c0);
 #pragma unroll
-                        for (int e = 0; e < 8; ++e) {
-                            const float4 c = __ldg(crow + e);
-                            v[4 * e + 0] *= c.x;
-                            v[4 * e + 1] *= c.y;
-                            v[4 * e + 2] *= c.z;
-                            v[4 * e + 3] *= c.w;
-                        }
-                    } else {
-#pragma unroll
-                        for (int e = 0; e < 32; ++e) v[e] = 0.f;
+                        for (int e = 0; e < 4; ++e) cv[e] = __ldg(crow + e);
                     }
-                    warp_store_runs(v, runs, valid, (int)gi, tile * (BM / 32) + q, lane, a.out, R, c0);
+                    chunk(c0, cv[0], cv[1], cv[2], cv[3]);
                 }
             }
             tc_fence_before();
@@ -204,7 +277,6 @@ __global__ void __launch_bounds__(split::THREADS, 1) ttm_split_kernel(const Spli
             if (lane == 0) mbar_arrive(&acc_empty[buf]);
         }
     } else if (warp == MMA_WARP) {
-        asm volatile("bar.sync 1, %0;" ::"n"(32 * (EPI_WARPS + 1)) : "memory");   // W is in place
         if (elect_one()) {
             const uint32_t idesc2 = make_idesc(1, 0, 0, BM, (uint32_t)(2 * R));    // bf16 x bf16, both K-major
             const uint32_t idesc1 = make_idesc(1, 0, 0, BM, (uint32_t)R);
@@ -239,57 +311,44 @@ __global__ void __launch_bounds__(split::THREADS, 1) ttm_split_kernel(const Spli
             }
         }
     } else {
-        // ---- converters.  Load u of a thread covers fibre (ct + 256 u) / 16 of the tile and the four
-        // k-values 4 * ((ct + 256 u) % 16) of the chunk: the 16 lanes of a half-warp read one fibre's
-        // 256 contiguous bytes and write its 128-byte row of each operand.
-        const int ct = threadIdx.x - 32 * CONV_WARP0;
-        const int g = ct & 15, r_base = ct >> 4;                      // rows r_base + 16 u
-        const int64_t total = (int64_t)my_tiles * a.kchunks;
-        auto load = [&](float4 (&x)[LOADS], int64_t it) {
-            const int t = (int)(it / a.kchunks), kc = (int)(it - (int64_t)t * a.kchunks);
-            const int64_t tile = blockIdx.x + (int64_t)t * gridDim.x;
-            const int k = kc * KC + g * 4;
-            const float *src = a.B + (tile * BM + r_base) * (int64_t)a.K + k;
+        // ---- converters
+        const uint32_t op0 = smem_u32(stage0);
+        // byte offset of this thread's 8 bytes inside an operand, for its first row; row r_base + 32 u has the
+        // same swizzle phase (32 u is a multiple of 8), so the others follow at 32 * 128 bytes each
+        const uint32_t op_off = (uint32_t)r_base * 128u + (uint32_t)(((g >> 1) ^ (r_base & 7)) << 4) + (uint32_t)((g & 1) << 3);
+        for (int64_t it = 0; it < total; ++it) {
+            asm volatile("cp.async.wait_group %0;" ::"n"(LAND - 1) : "memory");   // stage `it` has landed
+            const uint32_t land = land0 + (uint32_t)(it % LAND) * (uint32_t)LAND_BYTES;
+            float4 x[LOADS];
+#pragma unroll
+            for (int u = 0; u < LOADS; ++u)
+                asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];"
+                             : "=f"(x[u].x), "=f"(x[u].y), "=f"(x[u].z), "=f"(x[u].w)
+                             : "r"(land + (uint32_t)u * (CONV_THREADS * 16u)));
+            uint32_t h[LOADS][2], l[LOADS][2];
 #pragma unroll
             for (int u = 0; u < LOADS; ++u) {
-                const int64_t row = tile * BM + r_base + 16 * u;
-                x[u] = (row < a.rows && k < a.K) ? __ldcs(reinterpret_cast<const float4 *>(src + (int64_t)(16 * u) * a.K))
-                                                 : make_float4(0.f, 0.f, 0.f, 0.f);
+                split2(x[u].x, x[u].y, h[u][0], l[u][0]);
+                split2(x[u].z, x[u].w, h[u][1], l[u][1]);
             }
-        };
-        bool ok = true;
-        auto convert = [&](const float4 (&x)[LOADS], int64_t it) {
+            // the thread's chunks of this landing slot are in registers: the slot takes stage it + LAND at once,
+            // so that LAND stages are in flight whatever the tensor core is doing
+            load(it + LAND);
             const int s = (int)(it % a.stages);
             const int64_t use = it / a.stages;
-            if (use > 0 && !mbar_wait(&op_empty[s], (uint32_t)((use - 1) & 1), abort_flag, a.status, 1)) {
-                ok = false;
-                return;
-            }
-            unsigned char *hi = stage0 + (size_t)s * STAGE_BYTES;
+            if (use > 0 && !mbar_wait(&op_empty[s], (uint32_t)((use - 1) & 1), abort_flag, a.status, 1)) break;
+            const uint32_t op = op0 + (uint32_t)s * (uint32_t)STAGE_BYTES + op_off;
 #pragma unroll
             for (int u = 0; u < LOADS; ++u) {
-                const int r = r_base + 16 * u;
-                uint32_t h0, l0, h1, l1;
-                split2(x[u].x, x[u].y, h0, l0);
-                split2(x[u].z, x[u].w, h1, l1);
-                const uint32_t off = (uint32_t)r * 128u + (uint32_t)(((g >> 1) ^ (r & 7)) << 4) + (uint32_t)((g & 1) << 3);
-                *reinterpret_cast<uint2 *>(hi + off) = make_uint2(h0, h1);
-                *reinterpret_cast<uint2 *>(hi + OP_BYTES + off) = make_uint2(l0, l1);
+                const uint32_t o = op + (uint32_t)u * (ROW_STEP * 128u);
+                asm volatile("st.shared.v2.b32 [%0], {%1, %2};" ::"r"(o), "r"(h[u][0]), "r"(h[u][1]) : "memory");
+                asm volatile("st.shared.v2.b32 [%0], {%1, %2};" ::"r"(o + (uint32_t)OP_BYTES), "r"(l[u][0]), "r"(l[u][1]) : "memory");
             }
             fence_proxy_async();      // generic-proxy stores -> visible to the tensor core
             __syncwarp();
             if (lane == 0) mbar_arrive(&op_full[s]);
-        };
-        float4 xa[LOADS], xb[LOADS];
-        if (total > 0) load(xa, 0);
-        for (int64_t it = 0; it < total && ok; it += 2) {
-            if (it + 1 < total) load(xb, it + 1);
-            convert(xa, it);
-            if (it + 1 < total && ok) {
-                if (it + 2 < total) load(xa, it + 2);
-                convert(xb, it + 1);
-            }
         }
+        asm volatile("cp.async.wait_group 0;" ::: "memory");
     }
     // MTTKRP: the kernel that adds the partial sums may be launched now (it waits for this grid to end)
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
@@ -300,13 +359,6 @@ __global__ void __launch_bounds__(split::THREADS, 1) ttm_split_kernel(const Spli
         tmem_dealloc(tmem_base, a.tmem_cols);
     }
 }
-
-struct SplitPlan {
-    int kchunks, stages;
-    uint32_t tmem_cols;
-    size_t smem;
-    bool ok;
-};
 
 static SplitPlan split_plan(int64_t K, int64_t R)
 {
@@ -321,11 +373,13 @@ static SplitPlan split_plan(int64_t K, int64_t R)
     const size_t w_bytes = (size_t)p.kchunks * 2 * R * 128;
     const size_t fixed = 1024 + w_bytes + 512;
     const size_t budget = 227 * 1024;
-    if (fixed + 2 * STAGE_BYTES > budget) return p;
-    size_t st = (budget - fixed) / STAGE_BYTES;
+    p.land = (fixed + 3 * (size_t)LAND_BYTES + 2 * STAGE_BYTES <= budget) ? 3 : 2;
+    const size_t land = (size_t)p.land * LAND_BYTES;
+    if (fixed + land + 2 * STAGE_BYTES > budget) return p;
+    size_t st = (budget - fixed - land) / STAGE_BYTES;
     if (st > MAX_STAGES) st = MAX_STAGES;
     p.stages = (int)st;
-    p.smem = fixed + st * STAGE_BYTES;
+    p.smem = fixed + land + st * STAGE_BYTES;
     p.ok = true;
     return p;
 }
@@ -348,9 +402,14 @@ static st_status split_rows_launch(const float *Bp, int64_t rows, int64_t K, con
     a.out = out; a.status = (unsigned *)ws; a.rows = rows; a.K = (int)K; a.R = (int)R;
     a.kchunks = p.kchunks; a.stages = p.stages; a.tmem_cols = p.tmem_cols;
     a.ntiles = (int)((rows + BM - 1) / BM);
-    if (!ensure_dynamic_smem(ttm_split_kernel, p.smem)) return ST_ERR_CUDA;
     const int grid = a.ntiles < di.sm_count ? a.ntiles : di.sm_count;
-    ttm_split_kernel<<<grid, THREADS, p.smem, stream>>>(a);
+    if (p.land == 3) {
+        if (!ensure_dynamic_smem(ttm_split_kernel<3>, p.smem)) return ST_ERR_CUDA;
+        ttm_split_kernel<3><<<grid, THREADS, p.smem, stream>>>(a);
+    } else {
+        if (!ensure_dynamic_smem(ttm_split_kernel<2>, p.smem)) return ST_ERR_CUDA;
+        ttm_split_kernel<2><<<grid, THREADS, p.smem, stream>>>(a);
+    }
     return launch_status();
 }
 
