@@ -137,30 +137,42 @@ __global__ void __launch_bounds__(split::THREADS, 1) ttm_split_kernel(const Spli
     // is converted.
     const int ct = threadIdx.x - 32 * CONV_WARP0;
     const int g = ct & 15, r_base = ct >> 4;                          // rows r_base + 32 u
-    const int64_t total = (int64_t)my_tiles * a.kchunks;
+    const int total = my_tiles * a.kchunks;                           // stages of this block (< 2^31: see the launch)
     const uint32_t land0 = smem_u32(stage0 + (size_t)a.stages * STAGE_BYTES + 256) + (uint32_t)ct * 16u;
-    auto load = [&](int64_t it) {
-        if (it < total) {
-            const int t = (int)(it / a.kchunks), kc = (int)(it - (int64_t)t * a.kchunks);
-            const int64_t tile = blockIdx.x + (int64_t)t * gridDim.x;
-            const int k = kc * KC + g * 4;
-            const int64_t row0 = tile * BM + r_base;
-            const float *src = a.B + row0 * (int64_t)a.K + k;
-            const uint32_t dst = land0 + (uint32_t)(it % LAND) * (uint32_t)LAND_BYTES;
+    // State of the copy stream, advanced by one stage per call: all of it in 32-bit counters and one pointer
+    // (the sixteen converter warps all run this code: divisions and 64-bit products here would cost more
+    // issue slots than the conversion itself).
+    int ld_it = 0, ld_kc = 0, ld_slot = 0;
+    const int64_t first_row = (int64_t)blockIdx.x * BM + r_base;
+    int64_t ld_rows_left = a.rows - first_row;                        // fibres from this thread's first row of the tile to the end
+    const float *ld_src = a.B + first_row * (int64_t)a.K + g * 4;       // that row, this thread's k-offset, chunk 0
+    const int64_t tile_step = (int64_t)gridDim.x * BM;                // fibres between two tiles of this block
+    auto load = [&]() {
+        if (ld_it < total) {
+            const bool k_in = ld_kc * KC + g * 4 < a.K;
+            const uint32_t dst = land0 + (uint32_t)ld_slot * (uint32_t)LAND_BYTES;
+            const float *src = ld_src + ld_kc * KC;
 #pragma unroll
             for (int u = 0; u < LOADS; ++u) {
-                const bool in = row0 + ROW_STEP * u < a.rows && k < a.K;
+                const bool in = k_in && ROW_STEP * u < ld_rows_left;
                 const int sz = in ? 16 : 0;                          // src-size 0: the 16 bytes are zero-filled
                 asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst + (uint32_t)u * (CONV_THREADS * 16u)),
                              "l"(in ? src + (int64_t)(ROW_STEP * u) * a.K : a.B), "r"(sz)
                              : "memory");
+            }
+            ++ld_it;
+            if (++ld_slot == LAND) ld_slot = 0;
+            if (++ld_kc == a.kchunks) {
+                ld_kc = 0;
+                ld_rows_left -= tile_step;
+                ld_src += tile_step * a.K;
             }
         }
         asm volatile("cp.async.commit_group;" ::: "memory");           // one group per stage, empty past the end
     };
     // the first slices are requested before anything else, so that they travel while W is split
     if (warp >= CONV_WARP0)
-        for (int p = 0; p < LAND; ++p) load(p);
+        for (int p = 0; p < LAND; ++p) load();
 
     if (warp != MMA_WARP) {
         // ---- split W (all warps but the issuer: one cold round trip to memory each): chunk kc of 64 k-values
@@ -280,16 +292,16 @@ __global__ void __launch_bounds__(split::THREADS, 1) ttm_split_kernel(const Spli
         if (elect_one()) {
             const uint32_t idesc2 = make_idesc(1, 0, 0, BM, (uint32_t)(2 * R));    // bf16 x bf16, both K-major
             const uint32_t idesc1 = make_idesc(1, 0, 0, BM, (uint32_t)R);
-            int64_t step = 0;
+            int s = 0;
+            uint32_t full_parity = 0;
             bool ok = true;
             for (int t = 0; t < my_tiles && ok; ++t) {
                 const int buf = t & 1, use = t >> 1;
                 if (use > 0 && !mbar_wait(&acc_empty[buf], (uint32_t)((use - 1) & 1), abort_flag, a.status, 2)) break;
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + (uint32_t)(buf * 2 * R);
-                for (int kc = 0; kc < a.kchunks; ++kc, ++step) {
-                    const int s = (int)(step % a.stages);
-                    if (!mbar_wait(&op_full[s], (uint32_t)((step / a.stages) & 1), abort_flag, a.status, 3)) {
+                for (int kc = 0; kc < a.kchunks; ++kc) {
+                    if (!mbar_wait(&op_full[s], full_parity, abort_flag, a.status, 3)) {
                         ok = false;
                         break;
                     }
@@ -306,6 +318,10 @@ __global__ void __launch_bounds__(split::THREADS, 1) ttm_split_kernel(const Spli
                         }
                     }
                     tc_commit(&op_empty[s]);
+                    if (++s == a.stages) {
+                        s = 0;
+                        full_parity ^= 1u;
+                    }
                 }
                 tc_commit(&acc_full[buf]);
             }
@@ -316,9 +332,13 @@ __global__ void __launch_bounds__(split::THREADS, 1) ttm_split_kernel(const Spli
         // byte offset of this thread's 8 bytes inside an operand, for its first row; row r_base + 32 u has the
         // same swizzle phase (32 u is a multiple of 8), so the others follow at 32 * 128 bytes each
         const uint32_t op_off = (uint32_t)r_base * 128u + (uint32_t)(((g >> 1) ^ (r_base & 7)) << 4) + (uint32_t)((g & 1) << 3);
-        for (int64_t it = 0; it < total; ++it) {
+        int slot = 0, s = 0;
+        uint32_t empty_parity = 0;                                    // (first pass over the operand ring: nothing to wait for)
+        bool first_pass = true;
+        for (int it = 0; it < total; ++it) {
             asm volatile("cp.async.wait_group %0;" ::"n"(LAND - 1) : "memory");   // stage `it` has landed
-            const uint32_t land = land0 + (uint32_t)(it % LAND) * (uint32_t)LAND_BYTES;
+            const uint32_t land = land0 + (uint32_t)slot * (uint32_t)LAND_BYTES;
+            if (++slot == LAND) slot = 0;
             float4 x[LOADS];
 #pragma unroll
             for (int u = 0; u < LOADS; ++u)
@@ -333,10 +353,8 @@ __global__ void __launch_bounds__(split::THREADS, 1) ttm_split_kernel(const Spli
             }
             // the thread's chunks of this landing slot are in registers: the slot takes stage it + LAND at once,
             // so that LAND stages are in flight whatever the tensor core is doing
-            load(it + LAND);
-            const int s = (int)(it % a.stages);
-            const int64_t use = it / a.stages;
-            if (use > 0 && !mbar_wait(&op_empty[s], (uint32_t)((use - 1) & 1), abort_flag, a.status, 1)) break;
+            load();
+            if (!first_pass && !mbar_wait(&op_empty[s], empty_parity, abort_flag, a.status, 1)) break;
             const uint32_t op = op0 + (uint32_t)s * (uint32_t)STAGE_BYTES + op_off;
 #pragma unroll
             for (int u = 0; u < LOADS; ++u) {
@@ -347,6 +365,11 @@ __global__ void __launch_bounds__(split::THREADS, 1) ttm_split_kernel(const Spli
             fence_proxy_async();      // generic-proxy stores -> visible to the tensor core
             __syncwarp();
             if (lane == 0) mbar_arrive(&op_full[s]);
+            if (++s == a.stages) {
+                s = 0;
+                if (first_pass) first_pass = false;
+                else empty_parity ^= 1u;
+            }
         }
         asm volatile("cp.async.wait_group 0;" ::: "memory");
     }
@@ -402,6 +425,7 @@ static st_status split_rows_launch(const float *Bp, int64_t rows, int64_t K, con
     a.out = out; a.status = (unsigned *)ws; a.rows = rows; a.K = (int)K; a.R = (int)R;
     a.kchunks = p.kchunks; a.stages = p.stages; a.tmem_cols = p.tmem_cols;
     a.ntiles = (int)((rows + BM - 1) / BM);
+    if ((int64_t)a.ntiles * p.kchunks >= (int64_t(1) << 31)) return ST_ERR_UNSUPPORTED;
     const int grid = a.ntiles < di.sm_count ? a.ntiles : di.sm_count;
     if (p.land == 3) {
         if (!ensure_dynamic_smem(ttm_split_kernel<3>, p.smem)) return ST_ERR_CUDA;

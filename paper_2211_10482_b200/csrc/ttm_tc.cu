@@ -90,11 +90,11 @@ ttm_tc_kernel(const __grid_constant__ CUtensorMap tmap, const TtmTcArgs a)
         const int nthr = THREADS - 32, t0 = threadIdx.x - 32;
         const int r4 = a.R >> 2;                                      // float4 groups per row of U
         const int total4 = a.kchunks * KC * r4;
-        constexpr int UB = 8;
+        constexpr int UB = 16;
         for (int e0 = t0; e0 < total4; e0 += UB * nthr) {
             float4 v[UB];
 #pragma unroll
-            for (int u = 0; u < UB; ++u) {                            // eight independent loads in flight
+            for (int u = 0; u < UB; ++u) {                            // sixteen independent loads in flight: W comes from cold memory
                 const int e = e0 + u * nthr;
                 const int k = e / r4;
                 v[u] = (e < total4 && k < a.K) ? __ldg(reinterpret_cast<const float4 *>(a.U) + e)
@@ -180,9 +180,29 @@ ttm_tc_kernel(const __grid_constant__ CUtensorMap tmap, const TtmTcArgs a)
             const int buf = t & 1;
             int64_t tile = blockIdx.x + (int64_t)t * gridDim.x;
             if (a.reverse) tile = a.ntiles - 1 - tile;
+            const int64_t row = tile * BM + q * 32 + lane;
+            // MTTKRP: the fibre's (i, j) and, for R = 32, its row of C are fetched before the accumulator is
+            // waited for -- with the memory system saturated by the fibre stream a dependent load costs
+            // microseconds
+            const bool valid = row < a.rows;
+            int64_t gi = -1, gj = 0;
+            WarpRuns runs{0u, 0u};
+            float4 cpre[8];
+            const bool pre = a.mode != TC_TTM && a.R == 32;
+            if (a.mode != TC_TTM) {
+                if (valid) {
+                    if (a.mode == TC_MTTKRP_PACKED) tri_decode(a.I, row, gi, gj);
+                    else { gi = row / a.div; gj = row - gi * a.div; }
+                }
+                runs = warp_runs(valid, (int)gi, lane);
+                if (pre) {
+#pragma unroll
+                    for (int e = 0; e < 8; ++e)
+                        cpre[e] = valid ? __ldg(reinterpret_cast<const float4 *>(a.C + gj * a.R) + e) : make_float4(0.f, 0.f, 0.f, 0.f);
+                }
+            }
             if (!mbar_wait(&acc_full[buf], (uint32_t)((t >> 1) & 1), abort_flag, a.status, 4)) break;
             tc_fence_after();
-            const int64_t row = tile * BM + q * 32 + lane;
             if (a.mode == TC_TTM) {
                 float *dst = a.out + row * a.R;
                 for (int c0 = 0; c0 < a.R; c0 += 32) {
@@ -201,14 +221,7 @@ ttm_tc_kernel(const __grid_constant__ CUtensorMap tmap, const TtmTcArgs a)
                 // the warp that share i and write it to partial slot (unit + i), unit = row / 32 (see
                 // mttkrp_common.cuh).  The 32 fibres of a warp are consecutive, so they usually share i:
                 // one transposing shuffle reduction and one coalesced store per 32 columns.
-                const bool valid = row < a.rows;
-                int64_t gi = -1, gj = 0;
-                if (valid) {
-                    if (a.mode == TC_MTTKRP_PACKED) tri_decode(a.I, row, gi, gj);
-                    else { gi = row / a.div; gj = row - gi * a.div; }
-                }
                 const int gi32 = (int)gi;
-                const WarpRuns runs = warp_runs(valid, gi32, lane);
                 const int64_t unit = tile * (BM / 32) + q;
                 for (int c0 = 0; c0 < a.R && runs.heads != 0u; c0 += 32) {
                     uint32_t r[32];
@@ -219,7 +232,7 @@ ttm_tc_kernel(const __grid_constant__ CUtensorMap tmap, const TtmTcArgs a)
                         const float4 *crow = reinterpret_cast<const float4 *>(a.C + gj * a.R + c0);
 #pragma unroll
                         for (int e = 0; e < 8; ++e) {
-                            const float4 c = __ldg(crow + e);
+                            const float4 c = pre ? cpre[e] : __ldg(crow + e);
                             v[4 * e + 0] = c.x * __uint_as_float(r[4 * e + 0]);
                             v[4 * e + 1] = c.y * __uint_as_float(r[4 * e + 1]);
                             v[4 * e + 2] = c.z * __uint_as_float(r[4 * e + 2]);
