@@ -126,27 +126,35 @@ ttm_tc_kernel(const __grid_constant__ CUtensorMap tmap, const TtmTcArgs a)
     if (warp == 0) {
         if (elect_one()) {
             prefetch_tmap(&tmap);
-            int64_t step = 0;
-            bool ok = true;
+            // ring position and barrier phase are carried in counters: a 64-bit division per stage would cost
+            // this single thread a good part of the time one stage takes to arrive
+            int s = 0;
+            uint32_t empty_parity = 0;
+            bool first_pass = true, ok = true;
             for (int t = 0; t < my_tiles && ok; ++t) {
                 int64_t tile = blockIdx.x + (int64_t)t * gridDim.x;
                 if (a.reverse) tile = a.ntiles - 1 - tile;
-                for (int kc = 0; kc < a.kchunks; ++kc, ++step) {
-                    const int s = (int)(step % a.stages);
-                    const int64_t use = step / a.stages;
-                    if (use > 0 && !mbar_wait(&empty[s], (uint32_t)((use - 1) & 1), abort_flag, a.status, 1)) {
+                const int y = (int)(tile * BM);
+                for (int kc = 0; kc < a.kchunks; ++kc) {
+                    if (!first_pass && !mbar_wait(&empty[s], empty_parity, abort_flag, a.status, 1)) {
                         ok = false;
                         break;
                     }
                     mbar_expect_tx(&full[s], STAGE_BYTES);
-                    tma_load_2d(stage0 + (size_t)s * STAGE_BYTES, &tmap, &full[s], kc * KC, (int)(tile * BM));
+                    tma_load_2d(stage0 + (size_t)s * STAGE_BYTES, &tmap, &full[s], kc * KC, y);
+                    if (++s == a.stages) {
+                        s = 0;
+                        if (first_pass) first_pass = false;
+                        else empty_parity ^= 1u;
+                    }
                 }
             }
         }
     } else if (warp == 1) {
         if (elect_one()) {
             const uint32_t idesc = make_idesc(2, 0, 0, BM, (uint32_t)a.R);
-            int64_t step = 0;
+            int s = 0;
+            uint32_t full_parity = 0;
             bool ok = true;
             for (int t = 0; t < my_tiles && ok; ++t) {
                 const int buf = t & 1;
@@ -154,9 +162,8 @@ ttm_tc_kernel(const __grid_constant__ CUtensorMap tmap, const TtmTcArgs a)
                 if (use > 0 && !mbar_wait(&acc_empty[buf], (uint32_t)((use - 1) & 1), abort_flag, a.status, 2)) break;
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + (uint32_t)(buf * a.R);
-                for (int kc = 0; kc < a.kchunks; ++kc, ++step) {
-                    const int s = (int)(step % a.stages);
-                    if (!mbar_wait(&full[s], (uint32_t)((step / a.stages) & 1), abort_flag, a.status, 3)) {
+                for (int kc = 0; kc < a.kchunks; ++kc) {
+                    if (!mbar_wait(&full[s], full_parity, abort_flag, a.status, 3)) {
                         ok = false;
                         break;
                     }
@@ -170,6 +177,10 @@ ttm_tc_kernel(const __grid_constant__ CUtensorMap tmap, const TtmTcArgs a)
                         mma_tf32(d_tmem, adesc, bdesc, idesc, (kc > 0 || kk > 0) ? 1u : 0u);
                     }
                     tc_commit(&empty[s]);
+                    if (++s == a.stages) {
+                        s = 0;
+                        full_parity ^= 1u;
+                    }
                 }
                 tc_commit(&acc_full[buf]);
             }
