@@ -114,10 +114,12 @@ def call_table(cfg):
     mk = dict(flops=2 * c3["R"] * nnz3 + 2 * c3["R"] * tri(c3["I"]), bytes=4 * (nnz3 + (2 * c3["I"] + c3["K"]) * c3["R"]))
     t["mttkrp_tri"] = dict(mk, bound="alu", launches=2)
     t["mttkrp_tri_tf32"] = dict(mk, bound="tensor", launches=2, tensor_scale=TF32_OVER_BF16)
+    t["mttkrp_tri_split"] = dict(mk, bound="tensor", launches=2, tensor_scale=1.0 / 3.0)   # three bf16 products per term
     rows4 = c4["nb"] * c4["bs"] ** 2
     tt = dict(flops=2 * rows4 * c4["K"] * c4["R"], bytes=4 * (rows4 * (c4["K"] + c4["R"]) + c4["K"] * c4["R"]))
     t["ttm_blockdiag"] = dict(tt, bound="alu", launches=1)
     t["ttm_blockdiag_tf32"] = dict(tt, bound="tensor", launches=1, tensor_scale=TF32_OVER_BF16)
+    t["ttm_blockdiag_split"] = dict(tt, bound="tensor", launches=1, tensor_scale=1.0 / 3.0)
     d4 = c4["nb"] * c4["bs"]
     t["unpack_blockdiag"] = dict(flops=0, bytes=4 * c4["R"] * (rows4 + d4 * d4), bound="hbm", launches=1)
     nb_, kw = cfg["band"]["d"], cfg["band"]["kl"] + cfg["band"]["ku"] + 1
@@ -135,7 +137,7 @@ def tensor_peak_tflops(entry, peaks, burst):
     one inside the long step; TF32 calls take the measured TF32 yardstick when there is one, else
     the bf16 figure times the nominal TF32 / bf16 ratio."""
     scale = entry.get("tensor_scale", 1.0)
-    if scale != 1.0 and burst and peaks.get("tf32_tflops_yardstick"):
+    if scale == TF32_OVER_BF16 and burst and peaks.get("tf32_tflops_yardstick"):
         return peaks["tf32_tflops_yardstick"]
     return peaks["bf16_tflops" if burst else "bf16_tflops_sustained"] * scale
 
@@ -223,9 +225,9 @@ def bench_config():
 # any buffer of 2 MB or more and its next read at least 400 MB stream through the 126 MB L2; only
 # the two small reconstructions of the moment outputs read what the call before them left in L2.
 STEP_CALLS = ["sym_moment2_large", "pack_tri_x_k", "unpack_tri_sym_large", "ttm_blockdiag_tf32", "pack_band",
-              "unpack_blockdiag", "mttkrp_tri", "sym_moment3", "sym_moment2", "unpack_tet_sym", "unpack_tri_sym"]
+              "unpack_blockdiag", "mttkrp_tri_split", "sym_moment3", "sym_moment2", "unpack_tet_sym", "unpack_tri_sym"]
 # Timed on their own only (variants and widened rows)
-EXTRA_CALLS = ["mttkrp_tri_tf32", "ttm_blockdiag", "sym_moment3_tf32", "sym_moment3_bf16", "sym_moment4_d32",
+EXTRA_CALLS = ["mttkrp_tri", "mttkrp_tri_tf32", "ttm_blockdiag", "ttm_blockdiag_split", "sym_moment3_tf32", "sym_moment3_bf16", "sym_moment4_d32",
                "sym_moment4_d32_bf16", "sym_moment4_d64", "sym_moment4_d64_bf16", "thp_tri_x_k", "sym_moment2_large_f32"]
 
 
@@ -271,18 +273,20 @@ class Workload:
             "band_p": torch.empty(st.st_packed_elems(self.lay_band), **f32),
             "m2l": torch.empty(tri(c5["d"]), **f32), "m2l_dense": torch.empty(c5["d"] ** 2, **f32),
         }
-        TF, BF = st.ST_FLAG_TC_TF32, st.ST_FLAG_TC_BF16
+        TF, BF, SP = st.ST_FLAG_TC_TF32, st.ST_FLAG_TC_BF16, st.ST_FLAG_TC_SPLIT
         sizes = [
             st.st_workspace_bytes(st.ST_OP_SYM_MOMENT2, c1["N"], c1["d"], st.ST_F32),
             st.st_workspace_bytes(st.ST_OP_SYM_MOMENT3, c2["N"], c2["d"]),
-            st.st_workspace_bytes(st.ST_OP_MTTKRP_TRI, c3["I"], c3["K"], c3["R"]),
+            st.st_workspace_bytes(st.ST_OP_MTTKRP_TRI, c3["I"], c3["K"], c3["R"], 0, SP),
             st.st_workspace_bytes(st.ST_OP_TTM_BLOCKDIAG, c4["nb"], c4["bs"], c4["K"], c4["R"], TF),
             st.st_workspace_bytes(st.ST_OP_SYM_MOMENT2, c5["N"], c5["d"], st.ST_BF16), 256]
         if extras:
             sizes += [st.st_workspace_bytes(st.ST_OP_SYM_MOMENT3, c2["N"], c2["d"], 0, 0, TF),
                       st.st_workspace_bytes(st.ST_OP_SYM_MOMENT3, c2["N"], c2["d"], 0, 0, BF),
                       st.st_workspace_bytes(st.ST_OP_MTTKRP_TRI, c3["I"], c3["K"], c3["R"], 0, TF),
+                      st.st_workspace_bytes(st.ST_OP_MTTKRP_TRI, c3["I"], c3["K"], c3["R"], 0, 0),
                       st.st_workspace_bytes(st.ST_OP_TTM_BLOCKDIAG, c4["nb"], c4["bs"], c4["K"], c4["R"], 0),
+                      st.st_workspace_bytes(st.ST_OP_TTM_BLOCKDIAG, c4["nb"], c4["bs"], c4["K"], c4["R"], SP),
                       st.st_workspace_bytes(st.ST_OP_SYM_MOMENT2, c5["N"], c5["d"], st.ST_F32)]
             for d4 in cfg["moment4_d"]:
                 sizes += [st.st_workspace_bytes(st.ST_OP_SYM_MOMENT4, c2["N"], d4, 0, 0, 0),
@@ -309,7 +313,8 @@ class Workload:
                                                               flags=st.ST_FLAG_TC_TF32),
             "pack_band": lambda: st.st_pack(d["band"], self.lay_band, out=o["band_p"]),
             "unpack_blockdiag": lambda: st.st_unpack(o["Ap4"].view(-1), self.lay4, out=o["A4_dense"]),
-            "mttkrp_tri": lambda: st.st_mttkrp_tri(o["Bp3"], d["C3"], d["D3"], out=o["A3"], ws=ws),
+            "mttkrp_tri_split": lambda: st.st_mttkrp_tri(o["Bp3"], d["C3"], d["D3"], out=o["A3"], ws=ws,
+                                                         flags=st.ST_FLAG_TC_SPLIT),
             "sym_moment3": lambda: st.st_sym_moment3(d["X2"], out=o["m3"], ws=ws),
             "sym_moment2": lambda: st.st_sym_moment2(d["X1"], out=o["m2"], ws=ws),
             "unpack_tet_sym": lambda: st.st_unpack(o["m3"], self.lay2, st.ST_FILL_SYMMETRIC, out=o["m3_dense"]),
@@ -329,6 +334,9 @@ class Workload:
                 self._extra["m4_%d" % d4] = torch.empty(simp4(d4), **f32)
         x = self._extra
         calls = {
+            "mttkrp_tri": lambda: st.st_mttkrp_tri(o["Bp3"], d["C3"], d["D3"], out=o["A3"], ws=ws),
+            "ttm_blockdiag_split": lambda: st.st_ttm_blockdiag(d["Bp4"], d["U4"], c4["nb"], c4["bs"], out=o["Ap4"], ws=ws,
+                                                               flags=st.ST_FLAG_TC_SPLIT),
             "mttkrp_tri_tf32": lambda: st.st_mttkrp_tri(o["Bp3"], d["C3"], d["D3"], out=o["A3"], ws=ws, flags=st.ST_FLAG_TC_TF32),
             "ttm_blockdiag": lambda: st.st_ttm_blockdiag(d["Bp4"], d["U4"], c4["nb"], c4["bs"], out=o["Ap4"], ws=ws),
             "sym_moment3_tf32": lambda: st.st_sym_moment3(d["X2"], out=x["m3_tc"], ws=ws, flags=st.ST_FLAG_TC_TF32),
@@ -407,12 +415,13 @@ def dense_controls(w, timer, torch):
     gain from structure should approach dense work / unique work."""
     st, d, o, c = w.st, w.dev, w.out, w.cfg
     c1, c2, c3, c4, c5 = (c[k] for k in ("moment2", "moment3", "mttkrp", "ttm", "moment2_large"))
-    DC, TF = st.ST_FLAG_DENSE_CONTROL, st.ST_FLAG_TC_TF32
+    DC, TF, SP = st.ST_FLAG_DENSE_CONTROL, st.ST_FLAG_TC_TF32, st.ST_FLAG_TC_SPLIT
     dev = w.device
     wsb = max(st.st_workspace_bytes(st.ST_OP_SYM_MOMENT2, c1["N"], c1["d"], st.ST_F32, 0, DC),
               st.st_workspace_bytes(st.ST_OP_SYM_MOMENT3, c2["N"], c2["d"], 0, 0, DC),
               st.st_workspace_bytes(st.ST_OP_MTTKRP_TRI, c3["I"], c3["K"], c3["R"], 0, DC),
               st.st_workspace_bytes(st.ST_OP_MTTKRP_TRI, c3["I"], c3["K"], c3["R"], 0, DC | TF),
+              st.st_workspace_bytes(st.ST_OP_MTTKRP_TRI, c3["I"], c3["K"], c3["R"], 0, DC | SP),
               st.st_workspace_bytes(st.ST_OP_SYM_MOMENT2, c5["N"], c5["d"], st.ST_BF16, 0, DC), 256)
     wsc = torch.empty(wsb, dtype=torch.uint8, device=dev)
     d4 = c4["nb"] * c4["bs"]
@@ -430,6 +439,9 @@ def dense_controls(w, timer, torch):
         "mttkrp_tri_tf32": (lambda: st.st_mttkrp_tri(o["Bp3"], d["C3"], d["D3"], out=o["A3"], ws=w.ws, flags=TF),
                             lambda: st.st_mttkrp_tri(d["B3"], d["C3"], d["D3"], out=o["A3"], ws=wsc, flags=DC | TF),
                             c3["I"] ** 2 / tri(c3["I"]), 10),
+        "mttkrp_tri_split": (lambda: st.st_mttkrp_tri(o["Bp3"], d["C3"], d["D3"], out=o["A3"], ws=w.ws, flags=SP),
+                             lambda: st.st_mttkrp_tri(d["B3"], d["C3"], d["D3"], out=o["A3"], ws=wsc, flags=DC | SP),
+                             c3["I"] ** 2 / tri(c3["I"]), 10),
         "ttm_blockdiag": (lambda: st.st_ttm_blockdiag(d["Bp4"], d["U4"], c4["nb"], c4["bs"], out=o["Ap4"], ws=w.ws),
                           lambda: st.st_ttm_blockdiag(B4_dense, d["U4"], c4["nb"], c4["bs"], out=A4_dense, ws=w.ws, flags=DC),
                           float(c4["nb"]), 3),
@@ -629,7 +641,7 @@ def run_ours(args):
         "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "f32+bf16+tf32", "data": "synthetic",
         "config": {"workload": "the five named configurations in one step, one variant each: sym_moment2 large [1048576,1024] bf16 "
-                               "tensor cores; sym_moment3 [65536,64] fp32; mttkrp_tri I=K=512 R=32 fp32; ttm_blockdiag "
+                               "tensor cores; sym_moment3 [65536,64] fp32; mttkrp_tri I=K=512 R=32 split-bf16 tensor cores (fp32 tolerance); ttm_blockdiag "
                                "64x(64x64) K=256 R=64 TF32 tensor cores; sym_moment2 [4096,64] fp32; plus the pack / unpack "
                                "calls of their operands and results (tri x K, band, block-diagonal, symmetric fills)",
                    "step_calls": names,

@@ -158,6 +158,7 @@ __global__ void __launch_bounds__(M2S_MAX_THREADS, 1) moment2_small_kernel(const
             parity ^= 1u;
         }
     }
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // the sum over the slices may be launched; it waits for this grid to end
     if (*abort_flag && tid == 0) {
         // after a time-out: give the copies still in flight a bounded time to land before the
         // shared memory is reused or released
@@ -223,6 +224,9 @@ __global__ void __launch_bounds__(256)
 moment2_small_reduce_kernel(const float *__restrict__ partials, float *__restrict__ out, int d, int nbk, int slices,
                             int dense, const M2SmallItems items)
 {
+    // launched as a programmatic dependent of the kernel that writes the partial sums: the launch overlaps
+    // that kernel's tail, and nothing is read before it has completed
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     const int o = blockIdx.x * 256 + threadIdx.x;
     const int nitems = items.n;
     if (o >= nitems * 128) return;
@@ -344,9 +348,23 @@ st_status moment2_small(const float *X, int64_t N, int64_t d, int64_t ldx, float
     moment2_small_kernel<<<p.slices, p.threads, p.smem, stream>>>(a);
     if (cudaGetLastError() != cudaSuccess) return ST_ERR_CUDA;
     const int n = p.items.n * 128;
-    moment2_small_reduce_kernel<<<(n + 255) / 256, 256, 0, stream>>>(a.partials, out, (int)d, p.nbk, p.slices, a.dense,
-                                                                     p.items);
-    return launch_status();
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)((n + 255) / 256));
+    cfg.blockDim = dim3(256);
+    cfg.dynamicSmemBytes = 0;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    const float *partials = a.partials;
+    const int di = (int)d, dense = a.dense;
+    if (cudaLaunchKernelEx(&cfg, moment2_small_reduce_kernel, partials, out, di, p.nbk, p.slices, dense, p.items) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return ST_ERR_CUDA;
+    }
+    return ST_OK;
 }
 
 }  // namespace st
