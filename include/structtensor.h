@@ -139,15 +139,16 @@ st_status st_sym_moment2(const void *X, st_dtype xdt, int64_t N, int64_t d, int6
 /* Third moment over the unique set (Section 3, M2 = f (x) vec(f (x) f) summed over
  * samples; its unique elements are i<=j<=k, Section 2 "Tensor Structures"):
  *     out[q(i,j,k)] = sum_n X[n,i] * X[n,j] * X[n,k]   for 0 <= i <= j <= k < d
- * X: fp32 [N, ldx], ldx >= d, ldx % 4 == 0.  out_packed: d(d+1)(d+2)/6 floats in ST_TET
- * order.  Supported: d % 8 == 0, 8 <= d <= 64.
+ * X: fp32 [N, ldx], ldx >= d.  out_packed: d(d+1)(d+2)/6 floats in ST_TET order.  Supported:
+ * 1 <= d <= 256 (fastest for d % 8 == 0, d <= 64, ldx % 4 == 0; beyond 64 features the tile table
+ * of the call is copied into the workspace first).
  * ST_FLAG_DENSE_CONTROL: all d*d*d products are computed and the results outside the
  * unique set discarded; the output is the same.
  * ST_FLAG_TC_TF32 / ST_FLAG_TC_BF16 (one of them, not with the dense control) select the
  * tensor-core path: with the pair product hoisted out of the k loop (Section 5.5, code
  * motion) the sum is the contraction sum_n P[n,(i,j)] X[n,k] with P = X[n,i] X[n,j]; the
  * kernel makes P on the fly as the left operand of a GEMM over the samples and never issues
- * the tiles with k < j.  Any 1 <= d <= 64 and any ldx >= d.  TF32: x and the products
+ * the tiles with k < j.  1 <= d <= 64, any ldx >= d.  TF32: x and the products
  * rounded to TF32; bf16: x_k and the fp32 products rounded to bf16; fp32 accumulation.
  * Tolerance 5e-3 of sum |terms| (bf16: for N >= 1000; 2^-7 for any N). */
 st_status st_sym_moment3(const float *X, int64_t N, int64_t d, int64_t ldx,

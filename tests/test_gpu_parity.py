@@ -277,7 +277,7 @@ def test_fixed_order_calls_give_the_same_bits_twenty_times(st):
         st._allocator.check()
 
 
-@pytest.mark.parametrize("d", [8, 16, 24, 40, 64])
+@pytest.mark.parametrize("d", [1, 2, 3, 5, 8, 16, 17, 24, 40, 57, 63, 64])
 @pytest.mark.parametrize("N", [1, 63, 64, 65, 1000])
 def test_moment3_small(st, N, d):
     X = workloads.draw((N, d), "normal", 200 + N + d)
@@ -285,6 +285,38 @@ def test_moment3_small(st, N, d):
     got = st.st_sym_moment3(dev(X))
     assert got.numel() == workloads.tet(d)
     assert oracle.rel_err(expand3(st, got, d), T, S) <= TOL_F32, (N, d)
+
+
+@pytest.mark.parametrize("N,d", [(300, 72), (700, 100), (257, 128), (130, 200), (64, 256)])
+def test_moment3_more_than_64_features(st, N, d):
+    # the tile table of the call travels through the workspace, stages are shorter, several thread blocks
+    # share a sample slice; every unique entry against the oracle
+    X = workloads.draw((N, d), "normal", 250 + N + d)
+    walk = [(i, j, k) for i in range(d) for j in range(i, d) for k in range(j, d)]
+    ii, jj, kk = (np.array(v, dtype=np.int64) for v in zip(*walk))
+    T, S = oracle.moment3_at(X, ii, jj, kk)
+    ws = guarded(st, st.st_workspace_bytes(st.ST_OP_SYM_MOMENT3, N, d), torch.uint8)
+    got = st.st_sym_moment3(dev(X), ws=ws)
+    assert st.st_check_status(ws) == st.ST_OK
+    assert got.numel() == workloads.tet(d) == len(walk)
+    assert oracle.rel_err(got.cpu().numpy(), T, S) <= TOL_F32, (N, d)
+    assert torch.equal(got, st.st_sym_moment3(dev(X), ws=ws))        # fixed-order sums
+
+
+def test_moment3_rows_with_a_pitch_that_is_not_aligned(st):
+    # X as a view of a wider matrix whose rows are not 16-byte aligned: staged with plain loads
+    N, d, ldx = 500, 21, 23
+    buf = workloads.draw((N, ldx), "normal", 260)
+    Xv = dev(buf)[:, :d]
+    got = guarded(st, workloads.tet(d))
+    ws = guarded(st, st.st_workspace_bytes(st.ST_OP_SYM_MOMENT3, N, d), torch.uint8)
+    rc = st.lib().st_sym_moment3(Xv.data_ptr(), N, d, ldx, got.data_ptr(), ws.data_ptr(), ws.numel(), 0,
+                                 torch.cuda.current_stream().cuda_stream)
+    assert rc == st.ST_OK
+    T, S = oracle.moment3(np.ascontiguousarray(buf[:, :d]))
+    assert oracle.rel_err(expand3(st, got, d), T, S) <= TOL_F32
+    ctl = st.st_sym_moment3(dev(np.ascontiguousarray(buf[:, :d])), flags=st.ST_FLAG_DENSE_CONTROL)
+    assert oracle.rel_err(expand3(st, ctl, d), T, S) <= TOL_F32
 
 
 def test_moment3_dense_control_and_all_ones(st):

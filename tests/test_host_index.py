@@ -142,9 +142,10 @@ def test_layout_sizes_and_host_side_validation():
     assert L.st_sym_moment2(256, st.ST_F32, 4, 4, 3, 512, None, 0, 0, None) == st.ST_ERR_SHAPE
     assert L.st_sym_moment2(256, st.ST_F64, 4, 4, 4, 512, None, 0, 0, None) == st.ST_ERR_DTYPE
     assert L.st_sym_moment2(256, st.ST_F32, 4, 4, 4, 512, None, 0, 0, None) == st.ST_ERR_WORKSPACE
-    assert L.st_sym_moment3(256, 4, 12, 12, 512, None, 0, 0, None) == st.ST_ERR_UNSUPPORTED
-    assert L.st_sym_moment3(256, 4, 16, 18, 512, None, 0, 0, None) == st.ST_ERR_ALIGN
+    assert L.st_sym_moment3(256, 4, 257, 257, 512, None, 0, 0, None) == st.ST_ERR_UNSUPPORTED
+    assert L.st_sym_moment3(264, 4, 16, 16, 512, None, 0, 0, None) == st.ST_ERR_ALIGN
     assert L.st_sym_moment3(256, 4, 16, 16, 512, None, 0, 0, None) == st.ST_ERR_WORKSPACE
+    assert L.st_sym_moment3(256, 4, 12, 18, 512, None, 0, 0, None) == st.ST_ERR_WORKSPACE     # any d, any pitch
     assert L.st_sym_moment3(256, 4, 72, 72, 512, None, 0, st.ST_FLAG_TC_TF32, None) == st.ST_ERR_UNSUPPORTED
     assert L.st_sym_moment3(256, 4, 13, 13, 512, None, 0, st.ST_FLAG_TC_BF16, None) == st.ST_ERR_WORKSPACE
     assert L.st_sym_moment4(256, 4, 65, 65, 512, None, 0, 0, None) == st.ST_ERR_UNSUPPORTED
@@ -154,5 +155,8 @@ def test_layout_sizes_and_host_side_validation():
     assert L.st_ttm_blockdiag(256, 2, 2, 8, 512, 24, 1024, None, 0, 0, None) == st.ST_ERR_UNSUPPORTED
     assert L.st_ttm_blockdiag(256, 2, 2, 8, 520, 32, 1024, None, 0, 0, None) == st.ST_ERR_ALIGN
     assert st.st_workspace_bytes(st.ST_OP_SYM_MOMENT3, 65536, 64) > 45760 * 4
-    assert st.st_workspace_bytes(st.ST_OP_SYM_MOMENT3, 65536, 63) == 0
+    assert st.st_workspace_bytes(st.ST_OP_SYM_MOMENT3, 65536, 63) > 41664 * 4
+    assert st.st_workspace_bytes(st.ST_OP_SYM_MOMENT3, 65536, 257) == 0
+    # beyond 64 features the tile table of the call lives in the workspace too
+    assert st.st_workspace_bytes(st.ST_OP_SYM_MOMENT3, 100, 128) > 128 * 129 * 130 // 6 * 4 + 6528 * 4
     assert st.st_workspace_bytes(st.ST_OP_SYM_MOMENT2, 4096, 64, st.ST_F32) >= 256
