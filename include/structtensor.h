@@ -159,7 +159,7 @@ st_status st_sym_moment3(const float *X, int64_t N, int64_t d, int64_t ldx,
  * samples: the last block of the degree-2 polynomial-regression covariance; its unique elements
  * are the 4-tuples with repetition i<=j<=k<=l, "about 23x" fewer than d^4):
  *     out[s(i,j,k,l)] = sum_n X[n,i] X[n,j] X[n,k] X[n,l]   for 0 <= i <= j <= k <= l < d
- * X: fp32 [N, ldx], ldx >= d, 1 <= d <= 64.  out_packed: d(d+1)(d+2)(d+3)/24 floats in the
+ * X: fp32 [N, ldx], ldx >= d, 1 <= d <= 128 (ST_FLAG_TC_BF16: d <= 89).  out_packed: d(d+1)(d+2)(d+3)/24 floats in the
  * lexicographic order of the unique set (slab i holds the tetrahedron (j,k,l) of side d-i).
  * Computed as the second moment of the pair features P[n,(i,j)] = X[n,i] X[n,j], i<=j, which
  * the call materialises in the workspace (N * roundup(d(d+1)/2, 64) elements; query the size

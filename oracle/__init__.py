@@ -22,7 +22,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 _SRC = os.path.join(_HERE, "st_oracle.c")
 _LIB = os.path.join(_HERE, "_st_oracle.so")
 
-KIND_TRI, KIND_TET, KIND_BAND, KIND_BLOCKDIAG = 0, 1, 2, 3
+KIND_TRI, KIND_TET, KIND_BAND, KIND_BLOCKDIAG, KIND_FIXED_ROW, KIND_FIXED_COL, KIND_SIMPLEX4 = 0, 1, 2, 3, 4, 5, 6
 FILL_ZERO, FILL_SYMMETRIC = 0, 1
 
 _lib = None
@@ -59,7 +59,7 @@ def _load():
         lib.oracle_pack.restype = i64
         lib.oracle_unpack.argtypes = [ci, i64, i64, i64, i64, i64, i64, i64, ci, vp, vp]
         lib.oracle_unpack.restype = i64
-        lib.oracle_locate.argtypes = [ci, i64, i64, i64, i64, i64, i64, i64, i64]
+        lib.oracle_locate.argtypes = [ci, i64, i64, i64, i64, i64, i64, i64, i64, i64]
         lib.oracle_locate.restype = i64
         _lib = lib
     return _lib
@@ -200,7 +200,7 @@ def thp(B, C):
 
 
 def _dense_rows(kind, d):
-    return d * d * d if kind == KIND_TET else d * d
+    return {KIND_TET: d ** 3, KIND_SIMPLEX4: d ** 4}.get(kind, d * d)
 
 
 def packed_rows(kind, d, kl=0, ku=0, nb=0, bs=0) -> int:
@@ -233,15 +233,16 @@ def unpack(packed, kind, d, inner=1, kl=0, ku=0, nb=0, bs=0, fill=FILL_ZERO):
     r = _load().oracle_unpack(kind, d, inner, kl, ku, nb, bs, es, fill, _ptr(packed), _ptr(out))
     if r < 0:
         raise ValueError("unsupported layout / fill")
-    shape = (d, d, d) if kind == KIND_TET else (d, d)
+    shape = {KIND_TET: (d, d, d), KIND_SIMPLEX4: (d, d, d, d)}.get(kind, (d, d))
     if inner != 1:
         shape = shape + (inner,)
     return out.reshape(shape)
 
 
-def locate(kind, d, a, b, c=0, kl=0, ku=0, nb=0, bs=0) -> int:
-    """Packed position of one index tuple, by walking T_U from the start."""
-    return int(_load().oracle_locate(kind, d, kl, ku, nb, bs, a, b, c))
+def locate(kind, d, a, b, c=0, e=0, kl=0, ku=0, nb=0, bs=0) -> int:
+    """Packed position of one index tuple, by walking T_U from the start (the fixed index of the
+    one-row / one-column kinds is passed in kl)."""
+    return int(_load().oracle_locate(kind, d, kl, ku, nb, bs, a, b, c, e))
 
 
 def rel_err(got, T, S):

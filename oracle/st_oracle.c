@@ -240,6 +240,12 @@ void oracle_ttm(const float *B, int64_t rows, int64_t K,
  *       2 band matrix                  T_U(i,j)   = i-kl<=j<=i+ku
  *       3 block-diagonal matrix = direct sum of nb blocks of bs x bs
  *                                      (Figure "operations in STUR", e1 (+) e2)
+ *       4 one row of a matrix          T_U(i,j) = (i = r)          (R_r of Figure "matrix structures";
+ *       5 one column of a matrix       T_U(i,j) = (j = c)           C_c of the same figure; Table 1's
+ *                                      "fixed i" / "fixed j" structures on the first two modes; the
+ *                                      fixed index is passed in kl)
+ *       6 order-4 tensor               T_U(i,j,k,l) = 0<=i<=j<=k<=l<d  (Section 3, the unique 4-tuples
+ *                                      of M3; dense counterpart d x d x d x d)
  * Each position carries `inner` contiguous elements of `es` bytes (a trailing
  * dense mode).  fill: 0 = zeros outside T_U, 1 = redundancy map of the
  * symmetric structure (Figure "structures in STUR": T_R(i,j,i',j') =
@@ -256,6 +262,16 @@ static void sort3(int64_t *a, int64_t *b, int64_t *c)
     if (*a > *b) { t = *a; *a = *b; *b = t; }
     if (*b > *c) { t = *b; *b = *c; *c = t; }
     if (*a > *b) { t = *a; *a = *b; *b = t; }
+}
+
+/* Kinds 4, 5, 6 are written as a walk over the WHOLE dense index space in
+ * lexicographic order with a membership test of T_U (no loop bounds derived
+ * from the structure). */
+static int in_unique_set(int kind, int64_t fixed, int64_t i, int64_t j, int64_t k, int64_t l)
+{
+    if (kind == 4) return i == fixed;
+    if (kind == 5) return j == fixed;
+    return i <= j && j <= k && k <= l;
 }
 
 int64_t oracle_pack(int kind, int64_t d, int64_t inner, int64_t kl, int64_t ku,
@@ -297,6 +313,24 @@ int64_t oracle_pack(int kind, int64_t d, int64_t inner, int64_t kl, int64_t ku,
                     if (packed) memcpy(packed + (size_t)p * w, dense + (size_t)(i * d + j) * w, w);
                     ++p;
                 }
+    } else if (kind == 4 || kind == 5) {
+        if (kl < 0 || kl >= d) return -1;
+        for (int64_t i = 0; i < d; ++i)
+            for (int64_t j = 0; j < d; ++j)
+                if (in_unique_set(kind, kl, i, j, 0, 0)) {
+                    if (packed) memcpy(packed + (size_t)p * w, dense + (size_t)(i * d + j) * w, w);
+                    ++p;
+                }
+    } else if (kind == 6) {
+        for (int64_t i = 0; i < d; ++i)
+            for (int64_t j = 0; j < d; ++j)
+                for (int64_t k = 0; k < d; ++k)
+                    for (int64_t l = 0; l < d; ++l)
+                        if (in_unique_set(kind, 0, i, j, k, l)) {
+                            if (packed) memcpy(packed + (size_t)p * w,
+                                               dense + (size_t)(((i * d + j) * d + k) * d + l) * w, w);
+                            ++p;
+                        }
     } else {
         return -1;
     }
@@ -310,7 +344,7 @@ int64_t oracle_unpack(int kind, int64_t d, int64_t inner, int64_t kl, int64_t ku
     const size_t w = (size_t)(inner * es);
     int64_t p = 0;
     if (fill != 0 && fill != 1) return -1;
-    if (fill == 1 && kind > 1) return -1;
+    if (fill == 1 && kind != 0 && kind != 1 && kind != 6) return -1;
     if (kind == 0) {
         memset(dense, 0, (size_t)(d * d) * w);
         for (int64_t i = 0; i < d; ++i)
@@ -357,6 +391,39 @@ int64_t oracle_unpack(int kind, int64_t d, int64_t inner, int64_t kl, int64_t ku
                     memcpy(dense + (size_t)(i * d + j) * w, packed + (size_t)p * w, w);
                     ++p;
                 }
+    } else if (kind == 4 || kind == 5) {
+        if (kl < 0 || kl >= d) return -1;
+        memset(dense, 0, (size_t)(d * d) * w);
+        for (int64_t i = 0; i < d; ++i)
+            for (int64_t j = 0; j < d; ++j)
+                if (in_unique_set(kind, kl, i, j, 0, 0)) {
+                    memcpy(dense + (size_t)(i * d + j) * w, packed + (size_t)p * w, w);
+                    ++p;
+                }
+    } else if (kind == 6) {
+        memset(dense, 0, (size_t)(d * d * d * d) * w);
+        for (int64_t i = 0; i < d; ++i)
+            for (int64_t j = 0; j < d; ++j)
+                for (int64_t k = 0; k < d; ++k)
+                    for (int64_t l = 0; l < d; ++l)
+                        if (in_unique_set(kind, 0, i, j, k, l)) {
+                            memcpy(dense + (size_t)(((i * d + j) * d + k) * d + l) * w, packed + (size_t)p * w, w);
+                            ++p;
+                        }
+        if (fill == 1)   /* the representative of (i,j,k,l) is its sorted index tuple */
+            for (int64_t i = 0; i < d; ++i)
+                for (int64_t j = 0; j < d; ++j)
+                    for (int64_t k = 0; k < d; ++k)
+                        for (int64_t l = 0; l < d; ++l) {
+                            int64_t v[4] = {i, j, k, l};
+                            for (int a = 1; a < 4; ++a)          /* insertion sort */
+                                for (int b = a; b > 0 && v[b - 1] > v[b]; --b) {
+                                    int64_t t = v[b]; v[b] = v[b - 1]; v[b - 1] = t;
+                                }
+                            if (v[0] == i && v[1] == j && v[2] == k && v[3] == l) continue;
+                            memcpy(dense + (size_t)(((i * d + j) * d + k) * d + l) * w,
+                                   dense + (size_t)(((v[0] * d + v[1]) * d + v[2]) * d + v[3]) * w, w);
+                        }
     } else {
         return -1;
     }
@@ -364,10 +431,10 @@ int64_t oracle_unpack(int kind, int64_t d, int64_t inner, int64_t kl, int64_t ku
 }
 
 /* Position of one index tuple in the packed order, found by walking the unique
- * set from the start (slow on purpose).  c is ignored for matrix kinds.
+ * set from the start (slow on purpose).  c (and e) are ignored for matrix kinds.
  * Returns -1 when the tuple is not in T_U. */
 int64_t oracle_locate(int kind, int64_t d, int64_t kl, int64_t ku,
-                      int64_t nb, int64_t bs, int64_t a, int64_t b, int64_t c)
+                      int64_t nb, int64_t bs, int64_t a, int64_t b, int64_t c, int64_t e)
 {
     int64_t p = 0;
     if (kind == 0) {
@@ -387,6 +454,19 @@ int64_t oracle_locate(int kind, int64_t d, int64_t kl, int64_t ku,
         for (int64_t q = 0; q < nb; ++q)
             for (int64_t i = q * bs; i < (q + 1) * bs; ++i)
                 for (int64_t j = q * bs; j < (q + 1) * bs; ++j) { if (i == a && j == b) return p; ++p; }
+    } else if (kind == 4 || kind == 5) {
+        for (int64_t i = 0; i < d; ++i)
+            for (int64_t j = 0; j < d; ++j)
+                if (in_unique_set(kind, kl, i, j, 0, 0)) { if (i == a && j == b) return p; ++p; }
+    } else if (kind == 6) {
+        for (int64_t i = 0; i < d; ++i)
+            for (int64_t j = 0; j < d; ++j)
+                for (int64_t k = 0; k < d; ++k)
+                    for (int64_t l = 0; l < d; ++l)
+                        if (in_unique_set(kind, 0, i, j, k, l)) {
+                            if (i == a && j == b && k == c && l == e) return p;
+                            ++p;
+                        }
     }
     return -1;
 }

@@ -24,7 +24,7 @@ size_t moment2_workspace(int64_t N, int64_t d, int xdt, unsigned flags);
 
 namespace m4 {
 
-constexpr int MAX_D = 64;
+constexpr int MAX_D = 128;          // fp32 path; the bf16 path ends where the pair features exceed the tensor-core kernel's 4096 columns (d <= 89)
 constexpr int EXP_ROWS = 32;        // sample rows per pass of a block
 constexpr int EXP_THREADS = 192;
 

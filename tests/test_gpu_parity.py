@@ -486,6 +486,44 @@ def test_moment4_sampled_entries_and_multiplicity_identity(st, flag_name, N, d, 
     assert abs(lhs - rhs) <= tol * float(np.sum(np.abs(Xd).sum(axis=1) ** 4))
 
 
+@pytest.mark.parametrize("flag_name,N,d", [("f32", 40, 72), ("bf16", 1200, 72), ("f32", 24, 128)])
+def test_moment4_more_than_64_features(st, flag_name, N, d):
+    flags = st.ST_FLAG_TC_BF16 if flag_name == "bf16" else 0
+    X = workloads.draw((N, d), "normal", 800 + N + d)
+    got = st.st_sym_moment4(dev(X), flags=flags).cpu().numpy()
+    assert st.st_check_status() == st.ST_OK
+    n = math.comb(d + 3, 4)
+    assert got.size == n
+    # sampled entries, their positions found by the closed form of the running count (checked against the
+    # walk for d <= 64 by the host tests) ...
+    rng = np.random.default_rng(11)
+    tup = np.sort(rng.integers(0, d, (6000, 4)), axis=1)
+    tup = np.concatenate([tup, [[0, 0, 0, 0], [d - 1] * 4, [0, 0, 0, d - 1], [0, d - 1, d - 1, d - 1], [63, 64, 64, 65]]])
+    def pos(t):     # number of unique 4-tuples that precede t in lexicographic order, by counting
+        i, j, k, l = (int(v) for v in t)
+        c = sum(math.comb(d - a + 2, 3) for a in range(i))                      # first index smaller
+        c += sum(math.comb(d - b + 1, 2) for b in range(i, j))                  # second index smaller
+        c += sum(d - e for e in range(j, k))                                    # third index smaller
+        return c + (l - k)
+    p = np.array([pos(t) for t in tup])
+    T, S = oracle.moment4_at(X, tup[:, 0], tup[:, 1], tup[:, 2], tup[:, 3])
+    assert oracle.rel_err(got[p], T, S) <= (5e-3 if flags else TOL_F32), (flag_name, N, d)
+    # ... and the multiplicity identity over the whole output: sum_n (sum_i x_i)^4
+    Xd = X.astype(np.float64)
+    idx = np.array(list(itertools.combinations_with_replacement(range(d), 4)), dtype=np.int32) if d <= 72 else None
+    if idx is not None:
+        assert len(idx) == n
+        same = [(idx[:, a] == idx[:, a + 1]) for a in range(3)]
+        # multiplicity 24 / prod(run lengths!)
+        mult = np.full(n, 24.0)
+        run = np.ones(n)
+        for a in range(3):
+            run = np.where(same[a], run + 1, 1.0)
+            mult /= np.where(same[a], run, 1.0)
+        lhs, rhs = float(np.dot(mult, got.astype(np.float64))), float(np.sum(Xd.sum(axis=1) ** 4))
+        assert abs(lhs - rhs) <= (5e-3 if flags else TOL_F32) * float(np.sum(np.abs(Xd).sum(axis=1) ** 4))
+
+
 def test_moment4_all_ones_pitch_and_errors(st):
     ones = torch.ones((321, 20), dtype=torch.float32, device="cuda")
     assert torch.all(st.st_sym_moment4(ones) == 321.0)
@@ -501,7 +539,7 @@ def test_moment4_all_ones_pitch_and_errors(st):
     ii, jj, kk, ll = (np.array(v) for v in zip(*simplex4_tuples(d)))
     assert oracle.rel_err(out.cpu().numpy(), T[ii, jj, kk, ll], S[ii, jj, kk, ll]) <= TOL_F32
     assert L.st_sym_moment4(None, N, d, 20, out.data_ptr(), ws.data_ptr(), ws.numel(), 0, s) == st.ST_ERR_NULL
-    assert L.st_sym_moment4(wide.data_ptr(), N, 65, 65, out.data_ptr(), ws.data_ptr(), ws.numel(), 0, s) == st.ST_ERR_UNSUPPORTED
+    assert L.st_sym_moment4(wide.data_ptr(), N, 129, 129, out.data_ptr(), ws.data_ptr(), ws.numel(), 0, s) == st.ST_ERR_UNSUPPORTED
     assert L.st_sym_moment4(wide.data_ptr(), N, d, 20, out.data_ptr(), ws.data_ptr(), 1024, 0, s) == st.ST_ERR_WORKSPACE
     assert L.st_sym_moment4(wide.data_ptr(), N, d, 8, out.data_ptr(), ws.data_ptr(), ws.numel(), 0, s) == st.ST_ERR_SHAPE
     assert L.st_sym_moment4(wide.data_ptr(), N, d, 20, out.data_ptr(), ws.data_ptr(), ws.numel(), 1, s) == st.ST_ERR_UNSUPPORTED

@@ -148,7 +148,7 @@ def test_layout_sizes_and_host_side_validation():
     assert L.st_sym_moment3(256, 4, 12, 18, 512, None, 0, 0, None) == st.ST_ERR_WORKSPACE     # any d, any pitch
     assert L.st_sym_moment3(256, 4, 72, 72, 512, None, 0, st.ST_FLAG_TC_TF32, None) == st.ST_ERR_UNSUPPORTED
     assert L.st_sym_moment3(256, 4, 13, 13, 512, None, 0, st.ST_FLAG_TC_BF16, None) == st.ST_ERR_WORKSPACE
-    assert L.st_sym_moment4(256, 4, 65, 65, 512, None, 0, 0, None) == st.ST_ERR_UNSUPPORTED
+    assert L.st_sym_moment4(256, 4, 129, 129, 512, None, 0, 0, None) == st.ST_ERR_UNSUPPORTED
     assert L.st_sym_moment4(256, 4, 8, 8, 512, None, 0, 0, None) == st.ST_ERR_WORKSPACE
     assert L.st_mttkrp_tri(256, 4, 8, 512, 768, 12, 1024, None, 0, 0, None) == st.ST_ERR_UNSUPPORTED
     assert L.st_mttkrp_tri(256, 4, 8, 512, 768, 0, 1024, None, 0, 0, None) == st.ST_ERR_SHAPE

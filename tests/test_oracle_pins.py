@@ -327,22 +327,34 @@ def in_unique(kind, idx, d, kl=0, ku=0, bs=1):
         return idx[0] <= idx[1]
     if kind == oracle.KIND_TET:
         return idx[0] <= idx[1] <= idx[2]
+    if kind == oracle.KIND_SIMPLEX4:
+        return idx[0] <= idx[1] <= idx[2] <= idx[3]
     if kind == oracle.KIND_BAND:
         return idx[0] - kl <= idx[1] <= idx[0] + ku
+    if kind == oracle.KIND_FIXED_ROW:       # R_r of Figure "matrix structures": the fixed index travels in kl
+        return idx[0] == kl
+    if kind == oracle.KIND_FIXED_COL:       # C_c
+        return idx[1] == kl
     return idx[0] // bs == idx[1] // bs
+
+
+def order_of(kind):
+    return {oracle.KIND_TET: 3, oracle.KIND_SIMPLEX4: 4}.get(kind, 2)
 
 
 LAYOUTS = [
     (oracle.KIND_TRI, 7, {}), (oracle.KIND_TET, 5, {}),
     (oracle.KIND_BAND, 8, dict(kl=2, ku=1)), (oracle.KIND_BAND, 4, dict(kl=5, ku=0)),
     (oracle.KIND_BLOCKDIAG, 6, dict(nb=3, bs=2)),
+    (oracle.KIND_FIXED_ROW, 5, dict(kl=3)), (oracle.KIND_FIXED_COL, 6, dict(kl=0)), (oracle.KIND_FIXED_COL, 4, dict(kl=3)),
+    (oracle.KIND_SIMPLEX4, 4, {}),
 ]
 
 
 @pytest.mark.parametrize("kind,d,kw", LAYOUTS)
 @pytest.mark.parametrize("inner", [1, 3])
 def test_pack_is_lexicographic_walk_of_unique_set(kind, d, kw, inner):
-    order = 3 if kind == oracle.KIND_TET else 2
+    order = order_of(kind)
     shape = (d,) * order + (inner,)
     dense = np.arange(np.prod(shape), dtype=np.int32).reshape(shape) + 1
     packed = oracle.pack(dense, kind, d, inner=inner, **kw).reshape(-1, inner)
@@ -353,15 +365,15 @@ def test_pack_is_lexicographic_walk_of_unique_set(kind, d, kw, inner):
                 expect.append(dense[i, j] if 0 <= j < d else np.zeros(inner, np.int32))
     else:
         for idx in itertools.product(range(d), repeat=order):
-            if in_unique(kind, idx, d, bs=kw.get("bs", 1)):
+            if in_unique(kind, idx, d, kl=kw.get("kl", 0), bs=kw.get("bs", 1)):
                 expect.append(dense[idx])
     assert np.array_equal(packed, np.array(expect))
     # locate() agrees with the position found above
     pos = 0
     if kind != oracle.KIND_BAND:
         for idx in itertools.product(range(d), repeat=order):
-            a = tuple(idx) + (0,) * (3 - order)
-            if in_unique(kind, idx, d, bs=kw.get("bs", 1)):
+            a = tuple(idx) + (0,) * (4 - order)
+            if in_unique(kind, idx, d, kl=kw.get("kl", 0), bs=kw.get("bs", 1)):
                 assert oracle.locate(kind, d, *a, **kw) == pos
                 pos += 1
             else:
@@ -370,7 +382,7 @@ def test_pack_is_lexicographic_walk_of_unique_set(kind, d, kw, inner):
 
 @pytest.mark.parametrize("kind,d,kw", LAYOUTS)
 def test_round_trips_and_properties(kind, d, kw):
-    order = 3 if kind == oracle.KIND_TET else 2
+    order = order_of(kind)
     inner = 2
     rows = oracle.packed_rows(kind, d, **kw)
     P = workloads.draw((rows, inner), "normal", 99)
@@ -420,6 +432,51 @@ def test_symmetric_reconstruction_property5():
                 assert R3[i, j, k] == T3[i, j, k]
     with pytest.raises(ValueError):
         oracle.unpack(np.zeros(12, np.float32), oracle.KIND_BLOCKDIAG, 6, nb=3, bs=2, fill=oracle.FILL_SYMMETRIC)
+
+
+def test_four_simplex_counts_redundancy_map_and_slice_structures():
+    """The unique 4-tuples of M3 (Section 3): 35 of them at 4 features (Section 2: 65 = 10 + 20 + 35), about
+    23x fewer than d^4; the redundancy map sends every index tuple to its sorted representative; the
+    one-row / one-column structures hold d positions."""
+    g = golden()
+    n4 = g["pr2_distinct"] - oracle.packed_rows(oracle.KIND_TRI, 4) - oracle.packed_rows(oracle.KIND_TET, 4)
+    assert oracle.packed_rows(oracle.KIND_SIMPLEX4, 4) == n4 == 35
+    for d in range(1, 9):
+        assert oracle.packed_rows(oracle.KIND_SIMPLEX4, d) == math.comb(d + 3, 4)
+    assert 20 < 64 ** 4 / oracle.packed_rows(oracle.KIND_SIMPLEX4, 64) < 24
+    d = 4
+    rows = oracle.packed_rows(oracle.KIND_SIMPLEX4, d)
+    ids = np.arange(1, rows + 1, dtype=np.int32)
+    dense = oracle.unpack(ids, oracle.KIND_SIMPLEX4, d, fill=oracle.FILL_SYMMETRIC)
+    assert dense.shape == (d, d, d, d)
+    covered = 0
+    for idx in itertools.product(range(d), repeat=4):
+        rep = tuple(sorted(idx))
+        assert dense[idx] == ids[oracle.locate(oracle.KIND_SIMPLEX4, d, *rep)]
+        covered += 1
+    assert covered == d ** 4
+    # Property 5 on a real fourth moment: the symmetric fill restores the dense tensor
+    X = rnd((7, d), 31)
+    T4, _ = oracle.moment4(X)
+    P4 = oracle.pack(T4, oracle.KIND_SIMPLEX4, d)
+    R4 = oracle.unpack(P4, oracle.KIND_SIMPLEX4, d, fill=oracle.FILL_SYMMETRIC)
+    np.testing.assert_allclose(R4, T4, rtol=1e-13, atol=1e-13)
+    for perm in itertools.permutations(range(4)):
+        assert np.array_equal(R4, R4.transpose(perm))
+    # one row / one column of a matrix
+    for kind, fixed in ((oracle.KIND_FIXED_ROW, 2), (oracle.KIND_FIXED_COL, 4)):
+        assert oracle.packed_rows(kind, 6, kl=fixed) == 6
+        assert oracle.packed_rows(kind, 6, kl=6) == -1
+        M = rnd((6, 6), 32)
+        P = oracle.pack(M, kind, 6, kl=fixed)
+        assert np.array_equal(P, M[fixed, :] if kind == oracle.KIND_FIXED_ROW else M[:, fixed])
+        back = oracle.unpack(P, kind, 6, kl=fixed)
+        keep = np.zeros((6, 6), bool)
+        if kind == oracle.KIND_FIXED_ROW:
+            keep[fixed, :] = True
+        else:
+            keep[:, fixed] = True
+        assert np.array_equal(back, np.where(keep, M, 0.0))
 
 
 def test_unique_and_redundant_sets_partition_the_index_space():
