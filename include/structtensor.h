@@ -34,7 +34,12 @@
  *                 by st_pack and ignored by st_unpack.
  *   ST_BLOCKDIAG  direct sum of nblocks square blocks of size bs (Figure
  *                 "operations in STUR", e1 (+) e2): row (b*bs+i')*bs+j'.
- *   The dense counterpart is [d,d,inner] (ST_TET: [d,d,d,inner]).
+ *   ST_FIXED_ROW  T_U(i,j) = (i = r), ST_FIXED_COL T_U(i,j) = (j = c): the row / column structures R_r,
+ *                 C_c of Figure "matrix structures", i.e. Table 1's "fixed i" / "fixed j" on the first
+ *                 two modes; the fixed index is passed in `kl`; d rows (row j, resp. row i).
+ *   ST_SIMPLEX4   T_U(i,j,k,l) = 0<=i<=j<=k<=l<d (the unique 4-tuples of M3, Section 3): slab i holds
+ *                 the tetrahedron (j,k,l) of side d-i; d(d+1)(d+2)(d+3)/24 rows.
+ *   The dense counterpart is [d,d,inner] (ST_TET: [d,d,d,inner], ST_SIMPLEX4: [d,d,d,d,inner]).
  */
 #ifndef STRUCTTENSOR_H
 #define STRUCTTENSOR_H
@@ -62,7 +67,8 @@ typedef enum {
 } st_status;
 
 typedef enum { ST_F32 = 0, ST_BF16 = 1, ST_F64 = 2 } st_dtype;
-typedef enum { ST_TRI_UPPER = 0, ST_TET = 1, ST_BAND = 2, ST_BLOCKDIAG = 3 } st_kind;
+typedef enum { ST_TRI_UPPER = 0, ST_TET = 1, ST_BAND = 2, ST_BLOCKDIAG = 3, ST_FIXED_ROW = 4, ST_FIXED_COL = 5,
+               ST_SIMPLEX4 = 6 } st_kind;
 typedef enum { ST_FILL_ZERO = 0, ST_FILL_SYMMETRIC = 1 } st_fill;
 typedef enum { ST_OP_SYM_MOMENT2 = 0, ST_OP_SYM_MOMENT3 = 1, ST_OP_MTTKRP_TRI = 2,
                ST_OP_TTM_BLOCKDIAG = 3, ST_OP_SYM_MOMENT4 = 4, ST_OP_MTTKRP_SLICE = 5 } st_op;
@@ -84,7 +90,7 @@ typedef struct {
     int32_t reserved;  /* must be 0 */
     int64_t d;         /* structured extent: the matrix is d x d, ST_TET is d x d x d */
     int64_t inner;     /* trailing dense extent carried by every position (>= 1) */
-    int64_t kl, ku;    /* ST_BAND: sub- and super-diagonals kept (>= 0) */
+    int64_t kl, ku;    /* ST_BAND: sub- and super-diagonals kept (>= 0); ST_FIXED_ROW / ST_FIXED_COL: kl = the fixed index */
     int64_t nblocks;   /* ST_BLOCKDIAG: number of blocks; d must equal nblocks*bs */
     int64_t bs;        /* ST_BLOCKDIAG: block size */
 } st_layout;
@@ -93,7 +99,7 @@ typedef struct {
  * invalid layout.  Host only. */
 int64_t st_packed_elems(const st_layout *layout);
 
-/* Number of elements of the dense counterpart (d*d*inner or d*d*d*inner), or -1. */
+/* Number of elements of the dense counterpart (d*d*inner, d*d*d*inner or d*d*d*d*inner), or -1. */
 int64_t st_dense_elems(const st_layout *layout);
 
 /* T_C = T * T_U, stored contiguously (Section 4, "Compressed Tensor"; Section 6,
@@ -109,7 +115,8 @@ st_status st_pack(const st_layout *layout, st_dtype dtype, const void *dense, vo
  * (ST_FILL_ZERO: sparsity structure, T_R empty) or through the redundancy map of the
  * symmetric structure (ST_FILL_SYMMETRIC; ST_TRI_UPPER: T(i,j) = T_C(j,i) for j<i,
  * Figure "structures in STUR"; ST_TET: T(i,j,k) = T_C(sorted (i,j,k))).
- * ST_FILL_SYMMETRIC with ST_BAND / ST_BLOCKDIAG returns ST_ERR_UNSUPPORTED. */
+ * ST_SIMPLEX4 likewise: the sorted 4-tuple, so that the fourth moment is reconstructed once, at
+ * the end of a chain).  ST_FILL_SYMMETRIC with any other kind returns ST_ERR_UNSUPPORTED. */
 st_status st_unpack(const st_layout *layout, st_dtype dtype, const void *packed, void *dense,
                     st_fill fill, void *stream);
 

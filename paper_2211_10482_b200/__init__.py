@@ -24,7 +24,7 @@ ST_STATIC_SCRATCH_BYTES = 16 << 20
 # st_dtype
 ST_F32, ST_BF16, ST_F64 = 0, 1, 2
 # st_kind
-ST_TRI_UPPER, ST_TET, ST_BAND, ST_BLOCKDIAG = 0, 1, 2, 3
+ST_TRI_UPPER, ST_TET, ST_BAND, ST_BLOCKDIAG, ST_FIXED_ROW, ST_FIXED_COL, ST_SIMPLEX4 = 0, 1, 2, 3, 4, 5, 6
 # st_fill
 ST_FILL_ZERO, ST_FILL_SYMMETRIC = 0, 1
 # st_op

@@ -43,6 +43,16 @@ __device__ __forceinline__ int64_t dense_row_of_packed(const LayoutArgs &a, int6
         const int64_t i = p / a.width;
         const int64_t j = i + (p - i * a.width) - a.kl;
         return (j >= 0 && j < a.d) ? i * a.d + j : -1;
+    } else if (KIND == ST_FIXED_ROW) {
+        return a.kl * a.d + p;
+    } else if (KIND == ST_FIXED_COL) {
+        return p * a.d + a.kl;
+    } else if (KIND == ST_SIMPLEX4) {
+        int64_t i = 0;                                   // slab i: the largest i with simp4_slab_start(d, i) <= p
+        while (i + 1 < a.d && simp4_slab_start(a.d, i + 1) <= p) ++i;
+        int64_t j, k, l;
+        tet_decode(a.d - i, p - simp4_slab_start(a.d, i), j, k, l);
+        return (((i * a.d) + (i + j)) * a.d + (i + k)) * a.d + (i + l);
     } else {
         const int64_t bb = a.bs * a.bs;
         const int64_t b = p / bb;
@@ -80,6 +90,26 @@ __device__ __forceinline__ int64_t packed_row_of_dense(const LayoutArgs &a, int6
         const int64_t i = r / a.d, j = r - i * a.d;
         const int64_t s = j - i + a.kl;
         return (s >= 0 && s < a.width) ? i * a.width + s : -1;
+    } else if (KIND == ST_FIXED_ROW) {
+        const int64_t i = r / a.d;
+        return i == a.kl ? r - i * a.d : -1;
+    } else if (KIND == ST_FIXED_COL) {
+        const int64_t i = r / a.d;
+        return r - i * a.d == a.kl ? i : -1;
+    } else if (KIND == ST_SIMPLEX4) {
+        int64_t v[4];
+        int64_t q = r;
+        v[3] = q % a.d; q /= a.d;
+        v[2] = q % a.d; q /= a.d;
+        v[1] = q % a.d; v[0] = q / a.d;
+        if (!(v[0] <= v[1] && v[1] <= v[2] && v[2] <= v[3])) {
+            if (a.fill != ST_FILL_SYMMETRIC) return -1;
+            // representative = sorted index tuple (sorting network for four keys)
+#define ST_CSWAP(x, y) { if (v[x] > v[y]) { const int64_t t = v[x]; v[x] = v[y]; v[y] = t; } }
+            ST_CSWAP(0, 1) ST_CSWAP(2, 3) ST_CSWAP(0, 2) ST_CSWAP(1, 3) ST_CSWAP(1, 2)
+#undef ST_CSWAP
+        }
+        return simp4_encode(a.d, v[0], v[1], v[2], v[3]);
     } else {
         const int64_t i = r / a.d, j = r - i * a.d;
         const int64_t b = i / a.bs;
@@ -176,6 +206,17 @@ __device__ __forceinline__ void slice_run(const LayoutArgs &a, int64_t s, int64_
         hi = s + a.ku + 1; if (hi > a.d) hi = a.d;
         if (hi < lo) hi = lo;
         prow = s * a.width + (lo - (s - a.kl));
+    } else if (KIND == ST_FIXED_ROW) {
+        if (s == a.kl) { lo = 0; hi = a.d; } else { lo = hi = 0; }
+        prow = 0;
+    } else if (KIND == ST_FIXED_COL) {
+        lo = a.kl; hi = a.kl + 1; prow = s;
+    } else if (KIND == ST_SIMPLEX4) {
+        // slice s = (i, j, k): its unique entries are l = k .. d-1 when i <= j <= k
+        const int64_t ij = s / a.d, k = s - ij * a.d;
+        const int64_t i = ij / a.d, j = ij - i * a.d;
+        if (i <= j && j <= k) { lo = k; hi = a.d; prow = simp4_encode(a.d, i, j, k, k); }
+        else { lo = hi = 0; prow = 0; }
     } else {
         const int64_t b = s / a.bs;
         lo = b * a.bs; hi = lo + a.bs; prow = s * a.bs;
@@ -192,7 +233,7 @@ slice_copy_kernel(const U *__restrict__ src, U *__restrict__ dst, LayoutArgs a, 
     const int lane = (int)(threadIdx.x & (g - 1));
     const int64_t gid = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> group_shift;
     const int64_t ngroups = ((int64_t)gridDim.x * blockDim.x) >> group_shift;
-    const int64_t nslices = (KIND == ST_TET) ? a.d * a.d : a.d;
+    const int64_t nslices = (KIND == ST_TET) ? a.d * a.d : (KIND == ST_SIMPLEX4) ? a.d * a.d * a.d : a.d;
     const int64_t su = a.d * a.chunks;                        // units per dense slice
     for (int64_t item = gid; item < nslices * parts; item += ngroups) {
         const int64_t s = item / parts;
@@ -266,6 +307,9 @@ static bool layout_ok(const st_layout *L)
     switch (L->kind) {
     case ST_TRI_UPPER: return true;
     case ST_TET: return L->d <= (int64_t(1) << 20);
+    case ST_SIMPLEX4: return L->d <= 32768;
+    case ST_FIXED_ROW:
+    case ST_FIXED_COL: return L->kl >= 0 && L->kl < L->d;
     case ST_BAND: return L->kl >= 0 && L->ku >= 0 && L->kl < (int64_t(1) << 31) && L->ku < (int64_t(1) << 31);
     case ST_BLOCKDIAG: return L->nblocks > 0 && L->bs > 0 && L->nblocks * L->bs == L->d;
     default: return false;
@@ -277,6 +321,9 @@ static int64_t packed_rows_of(const st_layout *L)
     switch (L->kind) {
     case ST_TRI_UPPER: return tri_rows(L->d);
     case ST_TET: return tet_rows(L->d);
+    case ST_SIMPLEX4: return simp4_rows(L->d);
+    case ST_FIXED_ROW:
+    case ST_FIXED_COL: return L->d;
     case ST_BAND: return L->d * (L->kl + L->ku + 1);
     default: return L->nblocks * L->bs * L->bs;
     }
@@ -284,6 +331,7 @@ static int64_t packed_rows_of(const st_layout *L)
 
 static int64_t dense_rows_of(const st_layout *L)
 {
+    if (L->kind == ST_SIMPLEX4) return L->d * L->d * L->d * L->d;
     return L->kind == ST_TET ? L->d * L->d * L->d : L->d * L->d;
 }
 
@@ -322,13 +370,14 @@ static st_status launch_copy(const void *src, void *dst, const LayoutArgs &a, cu
     int64_t run_rows = a.d;
     if (KIND == ST_BAND) run_rows = a.width < a.d ? a.width : a.d;
     if (KIND == ST_BLOCKDIAG) run_rows = a.bs;
+    if (KIND == ST_FIXED_COL) run_rows = 1;
     const int64_t su = (PACK ? run_rows : a.d) * a.chunks;
     int parts = (int)((su + 8191) / 8192);
     if (parts < 1) parts = 1;
     const int64_t pu = (su + parts - 1) / parts;
     int shift = 0;
     while ((1 << shift) < 256 && (int64_t(8) << shift) < pu) ++shift;
-    const int64_t nslices = (KIND == ST_TET) ? a.d * a.d : a.d;
+    const int64_t nslices = (KIND == ST_TET) ? a.d * a.d : (KIND == ST_SIMPLEX4) ? a.d * a.d * a.d : a.d;
     const int64_t threads = (nslices * parts) << shift;
     const int64_t want = (threads + 255) / 256;
     const int grid = (int)(want < cap ? (want < 1 ? 1 : want) : cap);
@@ -343,6 +392,9 @@ static st_status dispatch_kind(const void *src, void *dst, const LayoutArgs &a, 
     case ST_TRI_UPPER: return launch_copy<ST_TRI_UPPER, U, PACK>(src, dst, a, s, mul);
     case ST_TET: return launch_copy<ST_TET, U, PACK>(src, dst, a, s, mul);
     case ST_BAND: return launch_copy<ST_BAND, U, PACK>(src, dst, a, s, mul);
+    case ST_FIXED_ROW: return launch_copy<ST_FIXED_ROW, U, PACK>(src, dst, a, s, mul);
+    case ST_FIXED_COL: return launch_copy<ST_FIXED_COL, U, PACK>(src, dst, a, s, mul);
+    case ST_SIMPLEX4: return launch_copy<ST_SIMPLEX4, U, PACK>(src, dst, a, s, mul);
     default: return launch_copy<ST_BLOCKDIAG, U, PACK>(src, dst, a, s, mul);
     }
 }
@@ -356,7 +408,8 @@ static st_status copy_entry(const st_layout *L, st_dtype dtype, const void *src,
     const int es = dtype_bytes(dtype);
     if (es == 0) return ST_ERR_DTYPE;
     if (fill != ST_FILL_ZERO && fill != ST_FILL_SYMMETRIC) return ST_ERR_UNSUPPORTED;
-    if (fill == ST_FILL_SYMMETRIC && (L->kind == ST_BAND || L->kind == ST_BLOCKDIAG)) return ST_ERR_UNSUPPORTED;
+    if (fill == ST_FILL_SYMMETRIC && L->kind != ST_TRI_UPPER && L->kind != ST_TET && L->kind != ST_SIMPLEX4)
+        return ST_ERR_UNSUPPORTED;
     if (!aligned16(src) || !aligned16(dst)) return ST_ERR_ALIGN;
     LayoutArgs a;
     a.kind = L->kind;

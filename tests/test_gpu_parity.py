@@ -87,6 +87,10 @@ def layouts(st):
             st.Layout(st.ST_BAND, 33, kl=0, ku=0), st.Layout(st.ST_BAND, 70, kl=1, ku=5)]
     out += [st.Layout(st.ST_BLOCKDIAG, 12, nblocks=3, bs=4), st.Layout(st.ST_BLOCKDIAG, 7, nblocks=7, bs=1),
             st.Layout(st.ST_BLOCKDIAG, 64, nblocks=1, bs=64), st.Layout(st.ST_BLOCKDIAG, 96, nblocks=3, bs=32)]
+    # one row / one column of a matrix (the fixed index travels in kl), and the packed 4-simplex
+    out += [st.Layout(st.ST_FIXED_ROW, 1, kl=0), st.Layout(st.ST_FIXED_ROW, 9, kl=4), st.Layout(st.ST_FIXED_ROW, 70, kl=69),
+            st.Layout(st.ST_FIXED_COL, 1, kl=0), st.Layout(st.ST_FIXED_COL, 9, kl=0), st.Layout(st.ST_FIXED_COL, 70, kl=33)]
+    out += [st.Layout(st.ST_SIMPLEX4, d) for d in (1, 2, 3, 5, 9, 17)]
     return out
 
 
@@ -115,7 +119,7 @@ def test_pack_unpack_bit_exact(st, inner, dtype):
         got_p = st.st_pack(dense_t, lay)
         assert got_p.dtype == tdt
         assert np.array_equal(got_p.cpu().numpy().view(u), want_p), (lay, "pack")
-        fills = [st.ST_FILL_ZERO] + ([st.ST_FILL_SYMMETRIC] if lay.kind in (st.ST_TRI_UPPER, st.ST_TET) else [])
+        fills = [st.ST_FILL_ZERO] + ([st.ST_FILL_SYMMETRIC] if lay.kind in (st.ST_TRI_UPPER, st.ST_TET, st.ST_SIMPLEX4) else [])
         for fill in fills:
             want_d = oracle.unpack(want_p, lay.kind, lay.d, inner=inner, fill=fill, **okw(lay)).reshape(-1)
             got_d = st.st_unpack(got_p, lay, fill=fill)
@@ -524,6 +528,21 @@ def test_moment4_more_than_64_features(st, flag_name, N, d):
         assert abs(lhs - rhs) <= (5e-3 if flags else TOL_F32) * float(np.sum(np.abs(Xd).sum(axis=1) ** 4))
 
 
+def test_moment4_is_reconstructed_once_at_the_end_of_a_chain(st):
+    # fourth moments of two batches are added in packed space (one structure: the sum keeps it) and the dense
+    # d^4 tensor is rebuilt once through the redundancy map of the 4-simplex (Section 5.5; Section 6, Property 5)
+    d = 9
+    Xa, Xb = workloads.draw((400, d), "normal", 1401), workloads.draw((250, d), "normal", 1402)
+    m4 = st.st_packed_axpby(1.0, st.st_sym_moment4(dev(Xa)), 1.0, st.st_sym_moment4(dev(Xb)))
+    lay = st.Layout(st.ST_SIMPLEX4, d)
+    full = st.st_unpack(m4, lay, fill=st.ST_FILL_SYMMETRIC).cpu().numpy().reshape(d, d, d, d)
+    T, S = oracle.moment4(np.concatenate([Xa, Xb]))
+    assert oracle.rel_err(full, T, S) <= TOL_F32
+    for perm in ((1, 0, 2, 3), (3, 2, 1, 0), (0, 2, 3, 1)):
+        assert np.array_equal(full, full.transpose(perm))
+    assert torch.equal(st.st_pack(dev(full), lay), m4)
+
+
 def test_moment4_all_ones_pitch_and_errors(st):
     ones = torch.ones((321, 20), dtype=torch.float32, device="cuda")
     assert torch.all(st.st_sym_moment4(ones) == 321.0)
@@ -842,6 +861,8 @@ def test_mttkrp_tf32_config(st, mttkrp_config_oracle):
 def _table1_layouts(st, K):
     return [st.Layout(st.ST_TRI_UPPER, 13, inner=K),                      # upper half cube (i <= j)
             st.Layout(st.ST_BLOCKDIAG, 37, inner=K, nblocks=37, bs=1),     # diagonal plane (i = j)
+            st.Layout(st.ST_FIXED_ROW, 19, inner=K, kl=7),                 # Table 1 "fixed i"
+            st.Layout(st.ST_FIXED_COL, 45, inner=K, kl=44),                # Table 1 "fixed j"
             st.Layout(st.ST_BAND, 21, inner=K, kl=2, ku=1),
             st.Layout(st.ST_BLOCKDIAG, 24, inner=K, nblocks=3, bs=8),
             st.Layout(st.ST_TET, 7, inner=K)]
@@ -849,7 +870,8 @@ def _table1_layouts(st, K):
 
 def _okind(st, lay):
     return {st.ST_TRI_UPPER: oracle.KIND_TRI, st.ST_TET: oracle.KIND_TET, st.ST_BAND: oracle.KIND_BAND,
-            st.ST_BLOCKDIAG: oracle.KIND_BLOCKDIAG}[lay.kind]
+            st.ST_BLOCKDIAG: oracle.KIND_BLOCKDIAG, st.ST_FIXED_ROW: oracle.KIND_FIXED_ROW,
+            st.ST_FIXED_COL: oracle.KIND_FIXED_COL, st.ST_SIMPLEX4: oracle.KIND_SIMPLEX4}[lay.kind]
 
 
 @pytest.mark.parametrize("flag_name,K,R", [("f32", 36, 32), ("f32", 64, 8), ("tf32", 64, 32), ("tf32", 36, 48),
