@@ -216,6 +216,29 @@ def test_moment2_f32_small(st, N, d):
         assert oracle.rel_err(got, T, S) <= TOL_F32, (N, d, flags)
 
 
+@pytest.mark.parametrize("N,d", [(1, 128), (15, 128), (16, 132), (17, 256), (300, 200), (2049, 384), (5000, 516), (40000, 128)])
+def test_moment2_f32_many_features(st, N, d):
+    # d >= 128 with aligned rows: 128 x 128 tiles, ragged last tiles, sample splits with a ragged tail
+    X = workloads.draw((N, d), "normal", 150 + N + d)
+    T, S = oracle.moment2(X)
+    for flags in (0, st.ST_FLAG_DENSE_CONTROL):
+        got = expand2(st, st.st_sym_moment2(dev(X), flags=flags), d)
+        assert oracle.rel_err(got, T, S) <= TOL_F32, (N, d, flags)
+    assert torch.equal(st.st_sym_moment2(dev(X)), st.st_sym_moment2(dev(X)))
+    # the same through a pitch: X as a view of a wider matrix
+    if N == 300:
+        wide = dev(workloads.draw((N, d + 8), "normal", 151))
+        Xv = wide[:, :d]
+        out = guarded(st, d * (d + 1) // 2)
+        nbytes = st.st_workspace_bytes(st.ST_OP_SYM_MOMENT2, N, d, st.ST_F32)
+        ws = guarded(st, nbytes, torch.uint8)
+        rc = st.lib().st_sym_moment2(Xv.data_ptr(), st.ST_F32, N, d, d + 8, out.data_ptr(), ws.data_ptr(), nbytes, 0,
+                                     torch.cuda.current_stream().cuda_stream)
+        assert rc == st.ST_OK
+        Tw, Sw = oracle.moment2(np.ascontiguousarray(wide.cpu().numpy()[:, :d]))
+        assert oracle.rel_err(expand2(st, out, d), Tw, Sw) <= TOL_F32
+
+
 def test_moment2_f32_strided_rows_and_all_ones(st):
     N, d, ldx = 300, 20, 28
     buf = workloads.draw((N, ldx), "normal", 5)
