@@ -1,20 +1,24 @@
 // st_ttm_blockdiag and st_mttkrp_tri, fp32 FMA path (Table 1: TTM, MTTKRP).
 //
 // In the packed layouts both kernels contract the trailing dense mode k of a tall matrix of
-// fibres with a small dense factor W[K,R] that stays in shared memory:
+// fibres with a small dense factor W[K,R]:
 //     Y[m, r] = sum_k Bp[m, k] * W[k, r]
 //   TTM     m runs over the fibres of the diagonal blocks only; Y is the packed output
 //           (the zero blocks of the direct sum are never touched: A_U(i,j,r) = B_U(i,j,.)).
 //   MTTKRP  m = p(i,j) runs over i<=j only; W = D; then A[i,r] += C[j,r] * Y[m,r], the
 //           product with C hoisted out of the k loop (Section 5.5, loop-invariant code motion).
 //
-// A thread block owns tiles of consecutive fibres (256 for R=64 and R<=16, 512 for R=32); 256
-// threads each keep TM x 8 sums in registers (TM = 8 for R >= 32).  Fibres are streamed through
-// a cp.async pipeline in slices of 32 k-values; work items (tile, k-split) are walked in one flattened loop so the
-// pipeline never drains between tiles.  MTTKRP splits k over work items when that evens out
-// the load (its output is a sum over k anyway); the sum over j is taken in a fixed order: every
-// warp writes the sums of its runs of fibres with equal i to partial slots and a second kernel
-// adds the slots of every row of A (mttkrp_common.cuh).
+// A warp owns a unit of consecutive fibres (32 for R = 64, 64 otherwise) and each of its threads keeps
+// 8 x 8 sums (fewer rows for R < 32) in registers.  That shape is set by what limits an fp32 FMA kernel that is
+// fed from shared memory on this GPU: an SM can issue 128 FMAs but deliver only 32 words from shared memory to its
+// registers per cycle, broadcasts included (an inner-loop probe ran at 0.87 of the FMA peak on registers alone,
+// 0.73 with an 8 x 8 tile, 0.67 with 8 x 4), so a thread must not read more than 16 words per 64 FMAs.
+// The units are dealt to the thread blocks in equal contiguous ranges; a block walks its range 16 units at
+// a time (in a last, partial step the warps without a unit skip the arithmetic).  Fibres stream through a cp.async
+// pipeline in stages of 16 k-values, each stage together with its 16 rows of W, so neither K nor R is limited by
+// the shared memory.  The sum over j of MTTKRP is taken in a fixed order: every warp adds the fibres of its unit
+// that share a row of A (i-slots in the thread, then a shuffle butterfly) and writes the sum to the partial slot
+// (unit + row); a second kernel adds the slots of every row of A (mttkrp_common.cuh).
 #include "st_common.cuh"
 #include "st_index.cuh"
 #include "mttkrp_common.cuh"
@@ -38,9 +42,8 @@ static inline unsigned *ws_status(void *ws, size_t ws_bytes)
     return (ws && ws_bytes >= kWsHeaderBytes && aligned256(ws)) ? (unsigned *)ws : nullptr;
 }
 
-constexpr int RG_THREADS = 256;
-constexpr int RG_KC = 32;         // k-values per stage
-constexpr int RG_LD = RG_KC + 4;  // padded row stride (floats) of a stage
+constexpr int RG_THREADS = 512;
+constexpr int RG_KC = 16;         // k-values per stage: one fibre contributes 64 bytes = four 16-byte chunks
 
 enum { RG_TTM = 0, RG_MTTKRP_PACKED = 1, RG_MTTKRP_DENSE = 2 };
 
@@ -59,57 +62,76 @@ struct RgArgs {
     int64_t rows;
     int K, R, I;         // I: rows of A reachable from `out`
     int64_t div;         // RG_MTTKRP_DENSE: fibre `row` belongs to (i, j) = (row / div, row % div)
-    int tiles, ksplit, kchunks_per_split, kchunks;
+    int kchunks;
+    int64_t units, units_per_block;   // a unit = the consecutive fibres of one warp; block b owns units b*upb .. (b+1)*upb-1
     unsigned *status;    // workspace header, or NULL
 };
 
-// TM rows x 8 columns per thread, CT column threads (R = 8*CT), RG_ROWS = 256/CT*TM fibres per tile.
+// R = 8 CT columns.  A warp owns WR = TM * (32 / CT) consecutive fibres: lane (fib, tc) holds, for each of its TM
+// "i-slots", fibre i * US + fib and the eight columns 4tc .. 4tc+3, R/2 + 4tc .. R/2 + 4tc+3.  What a thread reads
+// from shared memory per FMA decides the speed of this kernel (an SM returns 32 words per cycle to its registers and
+// can issue 128 FMAs): TM + 8 words per 8 TM FMAs.  A stage holds 16 k-values of every fibre of the tile without
+// padding; the four 16-byte chunks of a fibre are permuted by (fibre >> 1) so that the fibres of one load
+// instruction (consecutive `fib`) fall into different banks.
 template <int TM, int CT, int RG_STAGES, int MODE>
 __global__ void __launch_bounds__(RG_THREADS, 1) rowgemm_kernel(const RgArgs a)
 {
-    constexpr int RG_ROWS = RG_THREADS / CT * TM;
-    extern __shared__ __align__(16) float smem[];
-    float *Ws = smem;                                   // [kchunks*RG_KC][R], rows >= K are zero
-    float *Bs = Ws + (size_t)a.kchunks * RG_KC * a.R;   // RG_STAGES x [RG_ROWS][RG_LD]
     constexpr int R_ = CT * 8;
-    constexpr int RT = RG_THREADS / CT;                 // row threads; thread rows = tr + a*RT
-    const int tid = threadIdx.x;
-    const int tc = tid % CT, tr = tid / CT;
+    constexpr int US = 32 / CT;                         // fibres of one i-slot in a warp
+    constexpr int WR = TM * US;                         // consecutive fibres of a warp
+    constexpr int RG_ROWS = (RG_THREADS / 32) * WR;
+    constexpr int SWMASK = US >= 8 ? 3 : 1;             // chunk c of fibre f sits at chunk c ^ ((f >> 1) & SWMASK)
+    extern __shared__ __align__(16) float smem[];
+    constexpr int STAGE = RG_ROWS * RG_KC + RG_KC * R_; // floats of a stage: fibres [RG_ROWS][RG_KC], then W [RG_KC][R]
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int tc = lane % CT, fib = lane / CT;
 
     if (a.status && blockIdx.x == 0 && tid == 0) {      // no bounded waits in this kernel: the status is "ok"
         a.status[kWsStatusWord] = 0;
         a.status[kWsDetailWord] = 0;
     }
-    for (int e = tid; e < a.kchunks * RG_KC * a.R / 4; e += RG_THREADS)
-        reinterpret_cast<float4 *>(Ws)[e] =
-            (e < a.K * a.R / 4) ? reinterpret_cast<const float4 *>(a.W)[e] : make_float4(0.f, 0.f, 0.f, 0.f);
+    // The block owns a contiguous range of units and walks it in tiles of 16 (one unit per warp); in the last
+    // tile the warps without a unit skip the arithmetic, so a partial tile costs what its units cost.  The
+    // (tile, k-chunk) steps form one sequence; the loader runs RG_STAGES - 1 steps ahead of the arithmetic.
+    const int64_t u0 = (int64_t)blockIdx.x * a.units_per_block;
+    int64_t u1 = u0 + a.units_per_block;
+    if (u1 > a.units) u1 = a.units;
+    int64_t row_end = u1 * WR;
+    if (row_end > a.rows) row_end = a.rows;
+    const int my_items = u1 > u0 ? (int)((u1 - u0 + RG_THREADS / 32 - 1) / (RG_THREADS / 32)) : 0;
+    int ld_it = 0, ld_kcl = 0, ld_slot = 0;
 
-    const int items = a.tiles * a.ksplit;
-    // flattened (item, k-chunk) sequence of this block
-    const int my_items = (items > (int)blockIdx.x) ? (items - 1 - (int)blockIdx.x) / (int)gridDim.x + 1 : 0;
-    const int64_t total_steps = (int64_t)my_items * a.kchunks_per_split;
-
-    auto issue = [&](int64_t step) {
-        if (step < total_steps) {
-            const int it = (int)(step / a.kchunks_per_split);
-            const int kc_local = (int)(step - (int64_t)it * a.kchunks_per_split);
-            const int item = blockIdx.x + it * gridDim.x;
-            const int tile = item / a.ksplit, ks = item - tile * a.ksplit;
-            const int kc = ks * a.kchunks_per_split + kc_local;
-            float *dst = Bs + (int)(step % RG_STAGES) * (RG_ROWS * RG_LD);
-            const int64_t row0 = (int64_t)tile * RG_ROWS;
-            for (int c = tid; c < RG_ROWS * (RG_KC / 4); c += RG_THREADS) {
-                const int r = c >> 3, q = c & 7;
-                const int64_t row = row0 + r;
-                const int k = kc * RG_KC + q * 4;
-                const bool ok = row < a.rows && k < a.K && kc < a.kchunks;
-                rg_cp_async16(dst + r * RG_LD + q * 4, a.B + (ok ? row * a.K + k : 0), ok);
+    auto issue = [&]() {
+        if (ld_it < my_items) {
+            const int kc = ld_kcl;
+            const int q = tid & 3, r0 = tid >> 2;
+            const int k = kc * RG_KC + q * 4;
+            const bool kok = k < a.K;
+            int64_t row = (u0 + (int64_t)ld_it * (RG_THREADS / 32)) * WR + r0;
+            const float *src = a.B + row * a.K + k;
+            // rows advance by 128 per pass, so (row >> 1) & SWMASK stays what it is for r0
+            float *stage = smem + ld_slot * STAGE;
+            float *dst = stage + r0 * RG_KC + ((q ^ ((r0 >> 1) & SWMASK)) << 2);
+#pragma unroll
+            for (int u = 0; u < RG_ROWS / (RG_THREADS / 4); ++u) {
+                const bool ok = kok && row < row_end;
+                rg_cp_async16(dst, ok ? src : a.B, ok);
+                row += RG_THREADS / 4;
+                src += (int64_t)(RG_THREADS / 4) * a.K;
+                dst += (RG_THREADS / 4) * RG_KC;
             }
+            // the 16 rows of W that go with this k-chunk (from L2 after the first tile); rows >= K are zero
+            if (tid < RG_KC * R_ / 4) {
+                const bool wok = kc * RG_KC + tid / (R_ / 4) < a.K;
+                rg_cp_async16(stage + RG_ROWS * RG_KC + tid * 4, wok ? a.W + (size_t)kc * RG_KC * R_ + tid * 4 : a.W, wok);
+            }
+            if (++ld_kcl == a.kchunks) { ld_kcl = 0; ++ld_it; }
+            if (++ld_slot == RG_STAGES) ld_slot = 0;
         }
         asm volatile("cp.async.commit_group;\n" ::);
     };
 
-    for (int s = 0; s < RG_STAGES - 1; ++s) issue(s);
+    for (int s = 0; s < RG_STAGES - 1; ++s) issue();
 
     float acc[TM][8];
 #pragma unroll
@@ -117,29 +139,30 @@ __global__ void __launch_bounds__(RG_THREADS, 1) rowgemm_kernel(const RgArgs a)
 #pragma unroll
         for (int j = 0; j < 8; ++j) acc[i][j] = 0.f;
 
-    for (int64_t step = 0; step < total_steps; ++step) {
-        asm volatile("cp.async.wait_group %0;\n" ::"n"(RG_STAGES - 2));
-        __syncthreads();                       // stage `step` landed; stage step-1 is free again
-        issue(step + RG_STAGES - 1);
-        const int it = (int)(step / a.kchunks_per_split);
-        const int kc_local = (int)(step - (int64_t)it * a.kchunks_per_split);
-        const int item = blockIdx.x + it * gridDim.x;
-        const int tile = item / a.ksplit, ks = item - tile * a.ksplit;
-        const int kc = ks * a.kchunks_per_split + kc_local;
-        const float *bs = Bs + (int)(step % RG_STAGES) * (RG_ROWS * RG_LD);
-        const float *ws = Ws + (size_t)kc * RG_KC * R_ + tc * 8;
-        if (kc < a.kchunks) {
-#pragma unroll 2
-            for (int k4 = 0; k4 < RG_KC; k4 += 4) {
+    const int sw = (fib >> 1) & SWMASK;
+    int slot = 0;
+    for (int it = 0; it < my_items; ++it) {
+        const int64_t unit = u0 + (int64_t)it * (RG_THREADS / 32) + warp;
+        const bool active = unit < u1;
+        for (int kc = 0; kc < a.kchunks; ++kc) {
+            asm volatile("cp.async.wait_group %0;\n" ::"n"(RG_STAGES - 2));
+            __syncthreads();                       // this step's stage landed; the stage of the step before is free again
+            issue();
+            const float *bs = smem + slot * STAGE + (warp * WR + fib) * RG_KC;
+            const float *ws = smem + slot * STAGE + RG_ROWS * RG_KC + tc * 4;
+            if (++slot == RG_STAGES) slot = 0;
+            if (!active) continue;
+#pragma unroll
+            for (int c = 0; c < RG_KC / 4; ++c) {
                 float4 b[TM];
 #pragma unroll
                 for (int i = 0; i < TM; ++i)
-                    b[i] = *reinterpret_cast<const float4 *>(bs + (tr + i * RT) * RG_LD + k4);
+                    b[i] = *reinterpret_cast<const float4 *>(bs + i * (US * RG_KC) + ((c ^ sw) << 2));
 #pragma unroll
                 for (int kk = 0; kk < 4; ++kk) {
                     // k beyond K: the fibre slice was zero-filled and the rows of Ws are zero
-                    const float4 w0 = *reinterpret_cast<const float4 *>(ws + (k4 + kk) * R_);
-                    const float4 w1 = *reinterpret_cast<const float4 *>(ws + (k4 + kk) * R_ + 4);
+                    const float4 w0 = *reinterpret_cast<const float4 *>(ws + (4 * c + kk) * R_);
+                    const float4 w1 = *reinterpret_cast<const float4 *>(ws + (4 * c + kk) * R_ + R_ / 2);
                     const float wv[8] = {w0.x, w0.y, w0.z, w0.w, w1.x, w1.y, w1.z, w1.w};
 #pragma unroll
                     for (int i = 0; i < TM; ++i) {
@@ -150,93 +173,73 @@ __global__ void __launch_bounds__(RG_THREADS, 1) rowgemm_kernel(const RgArgs a)
                 }
             }
         }
-        if (kc_local == a.kchunks_per_split - 1) {
-            // ---- epilogue of this work item
-            const int64_t row0 = (int64_t)tile * RG_ROWS;
-            if (MODE == RG_TTM) {
+        // ---- epilogue of this work item
+        const int64_t wbase = unit * WR;                             // first fibre of this warp
+        if (!active) continue;
+        if (MODE == RG_TTM) {
 #pragma unroll
-                for (int i = 0; i < TM; ++i) {
-                    const int64_t row = row0 + tr + i * RT;
-                    if (row < a.rows) {
-                        float4 *o = reinterpret_cast<float4 *>(a.out + row * R_ + tc * 8);
-                        o[0] = make_float4(acc[i][0], acc[i][1], acc[i][2], acc[i][3]);
-                        o[1] = make_float4(acc[i][4], acc[i][5], acc[i][6], acc[i][7]);
-                    }
-                }
-            } else {
-                // A warp holds, for each i-slot, US = 32/CT consecutive fibres (8 columns per lane): one unit.
-                // Every run of fibres of the unit that share the row of A is summed with a shuffle butterfly
-                // (masked when the unit holds several runs) and written to partial slot (unit + row of A).
-                constexpr int US = 32 / CT;
-                const int lane = tid & 31;
-                const int fib = lane / CT;                 // fibre of this lane within the unit
-#pragma unroll
-                for (int i = 0; i < TM; ++i) {
-                    const int64_t row = row0 + tr + i * RT;
-                    const bool valid = row < a.rows;
-                    int64_t gi = -1, gj = 0;
-                    if (valid) {
-                        if (MODE == RG_MTTKRP_PACKED) tri_decode(a.I, row, gi, gj);
-                        else { gi = row / a.div; gj = row - gi * a.div; }
-                    }
-                    float v[8];
-                    if (valid) {
-                        const float4 c0 = *reinterpret_cast<const float4 *>(a.C + gj * R_ + tc * 8);
-                        const float4 c1 = *reinterpret_cast<const float4 *>(a.C + gj * R_ + tc * 8 + 4);
-                        const float cv[8] = {c0.x, c0.y, c0.z, c0.w, c1.x, c1.y, c1.z, c1.w};
-#pragma unroll
-                        for (int j = 0; j < 8; ++j) v[j] = cv[j] * acc[i][j];
-                    } else {
-#pragma unroll
-                        for (int j = 0; j < 8; ++j) v[j] = 0.f;
-                    }
-                    const int gi32 = (int)gi;
-                    const int prev = __shfl_up_sync(0xffffffffu, gi32, CT);
-                    // one bit per fibre (taken from the lanes with tc == 0)
-                    const unsigned heads = __ballot_sync(0xffffffffu, valid && tc == 0 && (fib == 0 || prev != gi32));
-                    const unsigned vmask = __ballot_sync(0xffffffffu, valid && tc == 0);
-                    if (heads == 0u) continue;             // no fibre of this unit exists
-                    const int64_t unit = (row - fib) / US; // the unit's first row is a multiple of US
-                    const int64_t unit0 = __shfl_sync(0xffffffffu, (long long)unit, 0);
-                    auto store = [&](int64_t slot, const float (&w)[8]) {
-                        float4 *dst = reinterpret_cast<float4 *>(a.out + (slot * a.ksplit + ks) * R_ + tc * 8);
-                        dst[0] = make_float4(w[0], w[1], w[2], w[3]);
-                        dst[1] = make_float4(w[4], w[5], w[6], w[7]);
-                    };
-                    const int gi0 = __shfl_sync(0xffffffffu, gi32, 0);
-                    if (heads == 1u) {
-#pragma unroll
-                        for (int off = CT; off < 32; off <<= 1)
-#pragma unroll
-                            for (int j = 0; j < 8; ++j) v[j] += __shfl_xor_sync(0xffffffffu, v[j], off);
-                        if (lane < CT) store(unit0 + gi0, v);
-                    } else if (heads == vmask) {
-                        if (valid) store(unit0 + gi, v);
-                    } else {
-                        unsigned h = heads;
-                        while (h) {
-                            const int l0 = __ffs(h) - 1;
-                            h &= h - 1;
-                            const int l1 = h ? __ffs(h) - 1 : 32;
-                            const bool in = lane >= l0 && lane < l1;
-                            float w[8];
-#pragma unroll
-                            for (int j = 0; j < 8; ++j) w[j] = in ? v[j] : 0.f;
-#pragma unroll
-                            for (int off = CT; off < 32; off <<= 1)
-#pragma unroll
-                                for (int j = 0; j < 8; ++j) w[j] += __shfl_xor_sync(0xffffffffu, w[j], off);
-                            const int gis = __shfl_sync(0xffffffffu, gi32, l0);
-                            if (lane < CT) store(unit0 + gis, w);
-                        }
-                    }
+            for (int i = 0; i < TM; ++i) {
+                const int64_t row = wbase + i * US + fib;
+                if (row < a.rows) {
+                    float *o = a.out + row * R_ + 4 * tc;
+                    *reinterpret_cast<float4 *>(o) = make_float4(acc[i][0], acc[i][1], acc[i][2], acc[i][3]);
+                    *reinterpret_cast<float4 *>(o + R_ / 2) = make_float4(acc[i][4], acc[i][5], acc[i][6], acc[i][7]);
                 }
             }
+        } else {
+            // The warp's WR fibres are one unit.  Every run of fibres of the unit that share the row g of A is summed
+            // in a fixed order (i-slots in the thread, then a shuffle butterfly over the fibres of a slot) and written
+            // to partial slot (unit + g); rows are sorted by g, so the runs are g0 .. g1.
+            int64_t wlast = wbase + WR - 1;
+            if (wlast >= a.rows) wlast = a.rows - 1;
+            int64_t g0, j0, g1, j1;
+            if (MODE == RG_MTTKRP_PACKED) {
+                tri_decode(a.I, wbase, g0, j0);
+                tri_decode(a.I, wlast, g1, j1);
+            } else {
+                g0 = wbase / a.div; j0 = wbase - g0 * a.div;
+                g1 = wlast / a.div; j1 = wlast - g1 * a.div;
+            }
+            (void)j1;
+            int gi[TM];
 #pragma unroll
-            for (int i = 0; i < TM; ++i)
+            for (int i = 0; i < TM; ++i) {
+                const int64_t row = wbase + i * US + fib;
+                int64_t g = -1, j = 0;
+                if (row < a.rows) {
+                    if (g0 == g1) { g = g0; j = j0 + (row - wbase); }
+                    else if (MODE == RG_MTTKRP_PACKED) tri_decode(a.I, row, g, j);
+                    else { g = row / a.div; j = row - g * a.div; }
+                    const float4 c0 = *reinterpret_cast<const float4 *>(a.C + j * R_ + 4 * tc);
+                    const float4 c1 = *reinterpret_cast<const float4 *>(a.C + j * R_ + R_ / 2 + 4 * tc);
+                    acc[i][0] *= c0.x; acc[i][1] *= c0.y; acc[i][2] *= c0.z; acc[i][3] *= c0.w;
+                    acc[i][4] *= c1.x; acc[i][5] *= c1.y; acc[i][6] *= c1.z; acc[i][7] *= c1.w;
+                }
+                gi[i] = (int)g;
+            }
+            for (int g = (int)g0; g <= (int)g1; ++g) {
+                float w[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-                for (int j = 0; j < 8; ++j) acc[i][j] = 0.f;
+                for (int i = 0; i < TM; ++i)
+                    if (gi[i] == g) {
+#pragma unroll
+                        for (int c = 0; c < 8; ++c) w[c] += acc[i][c];
+                    }
+#pragma unroll
+                for (int off = CT; off < 32; off <<= 1)
+#pragma unroll
+                    for (int c = 0; c < 8; ++c) w[c] += __shfl_xor_sync(0xffffffffu, w[c], off);
+                if (lane < CT) {
+                    float *o = a.out + (unit + g) * R_ + 4 * tc;
+                    *reinterpret_cast<float4 *>(o) = make_float4(w[0], w[1], w[2], w[3]);
+                    *reinterpret_cast<float4 *>(o + R_ / 2) = make_float4(w[4], w[5], w[6], w[7]);
+                }
+            }
         }
+#pragma unroll
+        for (int i = 0; i < TM; ++i)
+#pragma unroll
+            for (int j = 0; j < 8; ++j) acc[i][j] = 0.f;
     }
     asm volatile("cp.async.wait_group 0;\n" ::);
     if (MODE != RG_TTM) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // the row sums may be launched
@@ -302,49 +305,44 @@ st_status mttkrp_rowsum_launch(const float *part, float *A_full, int64_t I_full,
     return ST_OK;
 }
 
-// tile shape by R: {TM, stages}; rows per tile = 256 / (R/8) * TM
+// tile shape by R: {TM, stages}; a warp owns TM * 32 / (R/8) consecutive fibres, a tile is the block's 16 warps
 static void rowgemm_shape(int64_t R, int &tm, int &stages)
 {
-    if (R == 64) { tm = 8; stages = 3; }
-    else if (R == 32) { tm = 8; stages = 2; }
-    else { tm = (int)R / 8; stages = 3; }
+    if (R == 64) { tm = 8; stages = 6; }          // 512 fibres per tile, 36 KiB per stage
+    else if (R == 32) { tm = 8; stages = 3; }     // 1024 fibres per tile from here on, 66 KiB per stage
+    else { tm = (int)R / 4; stages = 3; }
+}
+static int64_t rowgemm_warp_rows(int64_t R)
+{
+    int tm, stages;
+    rowgemm_shape(R, tm, stages);
+    return (int64_t)tm * (32 / (R / 8));
 }
 
 static size_t rowgemm_smem(int64_t K, int64_t R)
 {
     int tm, stages;
     rowgemm_shape(R, tm, stages);
-    const size_t rows = (size_t)RG_THREADS / (R / 8) * tm;
-    const size_t kpad = (size_t)((K + RG_KC - 1) / RG_KC) * RG_KC;
-    return (kpad * R + (size_t)stages * rows * RG_LD) * sizeof(float);
+    const size_t rows = (size_t)(RG_THREADS / 32) * rowgemm_warp_rows(R);
+    (void)K;
+    return (size_t)stages * (rows * RG_KC + (size_t)RG_KC * R) * sizeof(float);
 }
 
 struct RgPlan {
-    int tiles, ksplit, kchunks, unit_rows;
+    int kchunks, unit_rows, grid;
+    int64_t units, units_per_block;
 };
 
-// Tiles and, for MTTKRP, the k-split that wastes the fewest SM slots in the last wave.
-static RgPlan rowgemm_plan(int64_t rows, int64_t K, int64_t R, bool mttkrp)
+// Units of consecutive fibres (one per warp and tile step) dealt to the blocks in equal contiguous ranges.
+static RgPlan rowgemm_plan(int64_t rows, int64_t K, int64_t R)
 {
     RgPlan p;
-    int tm, stages;
-    rowgemm_shape(R, tm, stages);
-    const int64_t tile_rows = (int64_t)RG_THREADS / (R / 8) * tm;
-    p.tiles = (int)((rows + tile_rows - 1) / tile_rows);
+    p.unit_rows = (int)rowgemm_warp_rows(R);
     p.kchunks = (int)((K + RG_KC - 1) / RG_KC);
-    p.unit_rows = (int)(32 / (R / 8));
-    p.ksplit = 1;
-    if (mttkrp) {
-        const int sms = sm_count_or_default();
-        double best = -1.0;
-        for (int ks = 1; ks <= 4; ks *= 2) {
-            if (p.kchunks % ks) continue;
-            const int64_t items = (int64_t)p.tiles * ks;
-            const int64_t waves = (items + sms - 1) / sms;
-            const double eff = (double)items / (double)(waves * sms);
-            if (eff > best + 0.02) { best = eff; p.ksplit = ks; }
-        }
-    }
+    p.units = (rows + p.unit_rows - 1) / p.unit_rows;
+    const int sms = sm_count_or_default();
+    p.units_per_block = (p.units + sms - 1) / sms;
+    p.grid = (int)((p.units + p.units_per_block - 1) / p.units_per_block);
     return p;
 }
 
@@ -356,23 +354,21 @@ static st_status rowgemm_launch(const RgArgs &a0, cudaStream_t stream)
     if (!di.ok) return ST_ERR_CUDA;
     const size_t smem = rowgemm_smem(a.K, a.R);
     if (smem > (size_t)di.max_smem_optin) return ST_ERR_UNSUPPORTED;
-    const RgPlan p = rowgemm_plan(a.rows, a.K, a.R, MODE != RG_TTM);
+    const RgPlan p = rowgemm_plan(a.rows, a.K, a.R);
     a.kchunks = p.kchunks;
-    a.tiles = p.tiles;
-    a.ksplit = p.ksplit;
-    a.kchunks_per_split = a.kchunks / a.ksplit;
-    const int64_t items = (int64_t)a.tiles * a.ksplit;
-    const int grid = (int)(items < di.sm_count ? items : di.sm_count);
+    a.units = p.units;
+    a.units_per_block = p.units_per_block;
+    const int grid = p.grid;
     auto run = [&](auto kernel) -> st_status {
         if (!ensure_dynamic_smem(kernel, smem)) return ST_ERR_CUDA;
         kernel<<<grid, RG_THREADS, smem, stream>>>(a);
         return launch_status();
     };
     switch (a.R) {
-    case 8: return run(rowgemm_kernel<1, 1, 3, MODE>);
-    case 16: return run(rowgemm_kernel<2, 2, 3, MODE>);
-    case 32: return run(rowgemm_kernel<8, 4, 2, MODE>);
-    case 64: return run(rowgemm_kernel<8, 8, 3, MODE>);
+    case 8: return run(rowgemm_kernel<2, 1, 3, MODE>);
+    case 16: return run(rowgemm_kernel<4, 2, 3, MODE>);
+    case 32: return run(rowgemm_kernel<8, 4, 3, MODE>);
+    case 64: return run(rowgemm_kernel<8, 8, 6, MODE>);
     default: return ST_ERR_UNSUPPORTED;
     }
 }
@@ -387,8 +383,8 @@ size_t mttkrp_workspace(int64_t rows, int64_t I, int64_t K, int64_t R, unsigned 
     if (flags & ST_FLAG_TC_TF32) return mttkrp_tf32_tc_workspace(rows, I, K, R);
     if (flags & ST_FLAG_TC_SPLIT) return mttkrp_split_workspace(rows, I, K, R);
     if (!rowgemm_r_ok(R)) return 0;
-    const RgPlan p = rowgemm_plan(rows, K, R, true);
-    return kWsHeaderBytes + (size_t)mttkrp_slots(rows, p.unit_rows, I, p.ksplit) * R * sizeof(float);
+    const RgPlan p = rowgemm_plan(rows, K, R);
+    return kWsHeaderBytes + (size_t)mttkrp_slots(rows, p.unit_rows, I, 1) * R * sizeof(float);
 }
 
 // Both passes of MTTKRP; `m` says how a row maps to (i, j), the fibres reach rows i_off .. of A_full.
@@ -404,7 +400,7 @@ static st_status mttkrp_run(const float *Bp, const MttkrpRows &m, int64_t K, con
     const size_t need = mttkrp_workspace(m.rows, m.I, K, R, flags);
     if (!ws || ws_bytes < need) return ST_ERR_WORKSPACE;
     if (!aligned256(ws)) return ST_ERR_ALIGN;
-    const RgPlan p = rowgemm_plan(m.rows, K, R, true);
+    const RgPlan p = rowgemm_plan(m.rows, K, R);
     RgArgs a{};
     a.B = Bp; a.W = D; a.C = C; a.out = (float *)((unsigned char *)ws + kWsHeaderBytes);
     a.K = (int)K; a.R = (int)R; a.I = m.I; a.rows = m.rows; a.div = m.div;
@@ -412,7 +408,7 @@ static st_status mttkrp_run(const float *Bp, const MttkrpRows &m, int64_t K, con
     const st_status rc = m.mode == MK_PACKED ? rowgemm_launch<RG_MTTKRP_PACKED>(a, stream)
                                              : rowgemm_launch<RG_MTTKRP_DENSE>(a, stream);
     if (rc != ST_OK) return rc;
-    return mttkrp_rowsum_launch(a.out, A_full, I_full, i_off, m, (int)R, p.unit_rows, p.ksplit, stream);
+    return mttkrp_rowsum_launch(a.out, A_full, I_full, i_off, m, (int)R, p.unit_rows, 1, stream);
 }
 
 }  // namespace st

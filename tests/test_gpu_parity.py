@@ -590,7 +590,11 @@ def test_moment4_all_ones_pitch_and_errors(st):
 # ------------------------------------------------------------------------------ MTTKRP / TTM
 
 @pytest.mark.parametrize("I,K,R", [(1, 4, 8), (2, 8, 16), (5, 36, 32), (16, 64, 64), (40, 100, 32), (70, 32, 8),
-                                   (33, 68, 64)])
+                                   (33, 68, 64),
+                                   # fibres far longer than any shared-memory stage; a k tail inside a stage
+                                   (12, 2052, 32), (9, 1300, 16),
+                                   # every block busy, several units per block, more than one step of 16 units in a block
+                                   (150, 20, 64), (200, 16, 8), (390, 16, 64)])
 def test_mttkrp_small(st, I, K, R):
     Bp, C, D = workloads.mttkrp_inputs(I, K, R)
     Bd = oracle.unpack(Bp.reshape(-1), oracle.KIND_TRI, I, inner=K)
@@ -626,7 +630,9 @@ def test_mttkrp_config(st, mttkrp_config_oracle):
 
 
 @pytest.mark.parametrize("nb,bs,K,R", [(1, 1, 4, 8), (3, 2, 8, 16), (2, 5, 36, 32), (4, 8, 64, 64), (7, 1, 32, 64),
-                                       (2, 17, 100, 8)])
+                                       (2, 17, 100, 8),
+                                       # long fibres with a k tail; more than one step of 16 units in a block
+                                       (2, 6, 2052, 64), (1, 40, 24, 32), (5, 124, 8, 64)])
 def test_ttm_small(st, nb, bs, K, R):
     Bp, U = workloads.ttm_inputs(nb, bs, K, R)
     d = nb * bs
