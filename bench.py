@@ -359,28 +359,36 @@ class Workload:
 
 
 class Isolated:
-    """Times one call on its own: the L2 is flushed (a 256 MB buffer is overwritten) before every
-    repetition, and the flush keeps the GPU busy while the host queues the call, so that the two
-    events bracket GPU time only."""
+    """Times one call on its own: the L2 is flushed before every repetition, and the flush keeps the GPU
+    busy while the host queues the call, so that the two events bracket GPU time only.  The flush
+    overwrites a 256 MB buffer and then (clean=True) reads another 256 MB: after the write alone about
+    100 MB of the flush buffer sit in the L2 as dirty lines, and their write-back to HBM would run inside
+    the timed region, on top of the traffic of the call (10 us and more on the streaming calls)."""
 
     def __init__(self, torch, device):
         self.torch = torch
         self.flush = torch.empty(256 << 20, dtype=torch.uint8, device=device)
+        self.sweep = torch.zeros(64 << 20, dtype=torch.float32, device=device)
 
-    def __call__(self, fn, reps=20, warm=3):
+    def __call__(self, fn, reps=20, warm=3, clean=True):
         torch = self.torch
         for _ in range(warm):
             fn()
         torch.cuda.synchronize()
-        ts = []
+        # all repetitions are queued before the one synchronisation, so that the GPU never idles (and never
+        # leaves its boost clock) between a flush and the call it precedes
+        pairs = []
         for _ in range(reps):
             self.flush.zero_()
+            if clean:
+                self.sweep.sum()
             e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
             e0.record()
             fn()
             e1.record()
-            torch.cuda.synchronize()
-            ts.append(e0.elapsed_time(e1) * 1e3)
+            pairs.append((e0, e1))
+        torch.cuda.synchronize()
+        ts = [e0.elapsed_time(e1) * 1e3 for e0, e1 in pairs]
         return float(np.median(ts)), float(min(ts))
 
 
@@ -580,6 +588,7 @@ def run_ours(args):
     # ---- every call on its own, L2 flushed
     timer = Isolated(torch, device)
     isolated = {}
+    dirty = {}          # the same with the write-only flush: dirty lines of the flush buffer left in the L2
     if extras:
         peaks["tf32_tflops_yardstick"] = round(tf32_yardstick(torch, device), 1)
         every = dict(step_calls)
@@ -595,6 +604,7 @@ def run_ours(args):
                 continue
             big = table[n]["bytes"] > (1 << 30) or n.startswith("sym_moment2_large")
             isolated[n] = timer(every[n], reps=(10 if big else 20), warm=3)
+            dirty[n] = timer(every[n], reps=(5 if big else 10), warm=1, clean=False)
         if st.st_check_status(w.ws) != st.ST_OK:
             raise RuntimeError("a kernel reported a device-side error during the isolated timings")
 
@@ -610,6 +620,8 @@ def run_ours(args):
             ent.update({"us": round(us, 2), "us_min": round(us_min, 2), "gflops": round(table[n]["flops"] / us / 1e3, 1),
                         "gbs": round(table[n]["bytes"] / us / 1e3, 1), "roofline_us": round(rl, 2), "roofline_of": bound,
                         "frac": round(rl / us, 4)})
+            if n in dirty:
+                ent["us_dirty_l2"] = round(dirty[n][0], 2)
         else:
             rl, bound = roofline_us(table[n], peaks, burst=False)
             us = ent["in_step_us"]
@@ -632,7 +644,7 @@ def run_ours(args):
     roof["frac"] = roof["achieved"] / roof["peak"]
     roof["traffic"] = ncu_traffic().get(dominant)
     roof["kernel"] = dominant
-    roof["timing"] = ("isolated launch, L2 flushed, median of %d" % 10) if burst else "inside the step"
+    roof["timing"] = ("isolated launch, L2 flushed (256 MB written, then 256 MB read), median of %d" % 10) if burst else "inside the step"
     roof["peak_source"] = ("derived from unit counts and clocks" if bound == "alu" else
                            peaks["source"] + ((" (burst)" if burst else " (sustained)") if bound == "tensor" else ""))
 
@@ -648,7 +660,9 @@ def run_ours(args):
                    "l2": "inputs larger than L2: between the write of any buffer of 2 MB or more and its next read at least "
                          "400 MB stream through the 126 MB L2; the two small symmetric reconstructions read the moment "
                          "outputs (<= 183 KB) that the call before them left in L2.  The per-call fractions come from "
-                         "isolated launches with the L2 flushed before each repetition (kernels[*].us), not from the step",
+                         "isolated launches with the L2 flushed before each repetition (kernels[*].us: 256 MB written, then "
+                         "256 MB of another buffer read so that no dirty line of the flush is written back inside the timed "
+                         "region; kernels[*].us_dirty_l2 is the same call after the write alone), not from the step",
                    "replicas": "independent replicas, no collective" if world > 1 else "single GPU"},
         "roofline": roof,
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": w.h2d_bytes, "d2h_bytes_per_step": w.d2h_bytes,
