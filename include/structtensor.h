@@ -76,7 +76,7 @@ typedef enum { ST_OP_SYM_MOMENT2 = 0, ST_OP_SYM_MOMENT3 = 1, ST_OP_MTTKRP_TRI = 
 /* flags (bit mask) */
 #define ST_FLAG_DENSE_CONTROL 1u /* run the same kernel over the dense, unstructured iteration
                                     space (a control for measurements; see each call) */
-#define ST_FLAG_TC_TF32       2u /* st_ttm_blockdiag, st_mttkrp_tri, st_sym_moment3: tensor cores, operands read as TF32 */
+#define ST_FLAG_TC_TF32       2u /* st_ttm_blockdiag, st_mttkrp_tri, st_sym_moment3, st_sym_moment2 (fp32 input): tensor cores, operands read as TF32 */
 #define ST_FLAG_TC_BF16       4u /* st_sym_moment3, st_sym_moment4: tensor cores, operands rounded to bf16 */
 #define ST_FLAG_TC_SPLIT      8u /* st_ttm_blockdiag, st_ttm_packed, st_mttkrp_tri, st_mttkrp_slice: tensor cores with
                                     both operands split into two bf16 parts and three of the four partial products
@@ -137,6 +137,10 @@ size_t st_workspace_bytes(st_op op, int64_t a, int64_t b, int64_t c, int64_t e, 
  * X: [N, ldx] with ldx >= d, dtype ST_F32 (fp32 FMA path, any d) or ST_BF16 (tensor-core
  * path: bf16 products, fp32 accumulation; needs d % 8 == 0, ldx % 8 == 0).
  * out_packed: d(d+1)/2 floats in ST_TRI_UPPER order.
+ * ST_FLAG_TC_TF32 (ST_F32 input only): the tensor cores read the fp32 words of X as TF32 (the 13 low
+ * mantissa bits are ignored: both factors of every product are truncated, so sums of positive products come out
+ * low by about 1e-3 relative), fp32 accumulation; 5e-3 tolerance; needs d % 4 == 0, ldx % 4 == 0, d <= 4096;
+ * about 15 times faster than the fp32 FMA path at d = 1024.
  * ST_FLAG_DENSE_CONTROL: all d*d products are computed (lower-triangle tiles too) and
  * the lower results discarded; the output is the same. */
 st_status st_sym_moment2(const void *X, st_dtype xdt, int64_t N, int64_t d, int64_t ldx,

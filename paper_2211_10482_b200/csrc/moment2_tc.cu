@@ -248,18 +248,31 @@ moment2_tc_reduce_kernel(const float *__restrict__ partials, float *__restrict__
 // the one-block kernel (whose tensor pipe idled ~30% of the time waiting for operands).  Four
 // stages of 64 samples are the measured optimum: with 6 or 7 stages the blocks of a sample range
 // drift apart, share less of X in L2 and the kernel gets 5-12% slower; with 3 it starves.
+//
+// The same kernel reads an fp32 X as TF32 (template argument): the tensor core takes the upper 19 bits of every
+// fp32 word, so the boxes are 32 columns (128 bytes) wide, a stage holds 32 samples and an MMA spans 8 of them;
+// the bytes per stage, the MMAs per stage and everything after the accumulator are the same.  An MN-major
+// operand of 32-bit elements has one legal shared-memory form, the 128-byte swizzle of 32-byte units, which
+// the copies write (tensor-map swizzle "128B, atom 32B") and the descriptors name.
 namespace m2tc2 {
 constexpr int BM = 256, BN = 256;               // tile of the pair
 constexpr int HALF = 128;                       // rows / B columns staged per block
-constexpr int KROWS = 64, BOXC = m2tc::BOXC, BOX_BYTES = BOXC * KROWS * 2;
-constexpr int NBOX = HALF / BOXC;               // 2 boxes per operand per block
-constexpr int STAGE_BYTES = 2 * NBOX * BOX_BYTES;   // 32 KiB
+constexpr int STAGE_BYTES = 32768;              // HALF columns of A and of B over the sample rows of one stage
 constexpr int STAGES = 4;
 constexpr int THREADS = 192;
 constexpr int MAX_TILES = 160;
 constexpr uint32_t TMEM_COLS = 512;
-constexpr int FLUSH_CHUNKS = 4096 / KROWS;        // 4096 samples (256 MMAs) per accumulator phase
 constexpr size_t SMEM_BYTES = (size_t)STAGES * STAGE_BYTES + 1024 + 256;
+template <bool TF32> struct Shape {
+    static constexpr int ELEM = TF32 ? 4 : 2;
+    static constexpr int KROWS = TF32 ? 32 : 64;            // sample rows per stage
+    static constexpr int KMMA = TF32 ? 8 : 16;              // sample rows per MMA
+    static constexpr int BOXC = 128 / ELEM;                 // columns per TMA box (128 bytes)
+    static constexpr int BOX_BYTES = 128 * KROWS;
+    static constexpr int NBOX = HALF / BOXC;                // boxes per operand per block
+    static constexpr int FLUSH_CHUNKS = 4096 / KROWS;       // 4096 samples (256 or 512 MMAs) per accumulator phase
+    static_assert(2 * NBOX * BOX_BYTES == STAGE_BYTES, "stage size");
+};
 
 struct TileTable {
     int ntiles, nsplit;
@@ -268,12 +281,15 @@ struct TileTable {
 };
 }  // namespace m2tc2
 
+template <bool TF32>
 __global__ void __launch_bounds__(m2tc2::THREADS, 1)
 moment2_tc_pair_kernel(const __grid_constant__ CUtensorMap tmap, float *__restrict__ partials, unsigned *status,
                        int chunks_total, const __grid_constant__ m2tc2::TileTable tab)
 {
     using namespace m2tc2;
     using namespace tc;
+    using S = Shape<TF32>;
+    constexpr int KROWS = S::KROWS, BOXC = S::BOXC, BOX_BYTES = S::BOX_BYTES, NBOX = S::NBOX, FLUSH_CHUNKS = S::FLUSH_CHUNKS;
     extern __shared__ unsigned char smem_raw[];
     unsigned char *smem = (unsigned char *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     uint64_t *bars = (uint64_t *)(smem + (size_t)STAGES * STAGE_BYTES);
@@ -344,11 +360,12 @@ moment2_tc_pair_kernel(const __grid_constant__ CUtensorMap tmap, float *__restri
     } else if (warp == 1) {
         // ---------------- MMA issuer (leader only)
         if (rank == 0 && elect_one()) {
-            constexpr uint32_t idesc = make_idesc(1, 1, 1, BM, BN);
+            constexpr uint32_t idesc = make_idesc(TF32 ? 2 : 1, 1, 1, BM, BN);
             const uint32_t a_off = diag ? 0u : (uint32_t)(NBOX * BOX_BYTES);
             const uint32_t sb0 = smem_u32(smem);
-            const uint64_t adesc_base = make_smem_desc(sb0 + a_off, BOX_BYTES, 1024);
-            const uint64_t bdesc_base = make_smem_desc(sb0, BOX_BYTES, 1024);
+            // bf16: groups of 8 sample rows, 16-byte swizzle units; fp32 read as TF32: groups of 4, 32-byte units
+            const uint64_t adesc_base = make_smem_desc(sb0 + a_off, BOX_BYTES, TF32 ? 512 : 1024, TF32 ? 1 : 2);
+            const uint64_t bdesc_base = make_smem_desc(sb0, BOX_BYTES, TF32 ? 512 : 1024, TF32 ? 1 : 2);
             bool ok = true;
             int c = 0;
             for (int ph = 0; ph < nphases && ok; ++ph) {
@@ -368,8 +385,11 @@ moment2_tc_pair_kernel(const __grid_constant__ CUtensorMap tmap, float *__restri
                     const uint64_t ad = adesc_base + (uint64_t)(s * (STAGE_BYTES >> 4));
                     const uint64_t bd = bdesc_base + (uint64_t)(s * (STAGE_BYTES >> 4));
 #pragma unroll
-                    for (int k = 0; k < KROWS / 16; ++k) {
-                        mma_bf16_pair(d_tmem, ad + (uint64_t)(k * 128), bd + (uint64_t)(k * 128), idesc, accumulate);
+                    for (int k = 0; k < KROWS / S::KMMA; ++k) {
+                        // one MMA spans KMMA sample rows of 128 bytes: 2048 bytes (bf16) or 1024 bytes (TF32) further on
+                        constexpr int STEP = S::KMMA * 128 / 16;
+                        if (TF32) mma_tf32_pair(d_tmem, ad + (uint64_t)(k * STEP), bd + (uint64_t)(k * STEP), idesc, accumulate);
+                        else mma_bf16_pair(d_tmem, ad + (uint64_t)(k * STEP), bd + (uint64_t)(k * STEP), idesc, accumulate);
                         accumulate = 1;
                     }
                     tc_commit_pair(&empty[s]);
@@ -454,9 +474,10 @@ struct M2Tc2Plan {
     bool ok;
 };
 
-static M2Tc2Plan m2tc2_plan(int64_t N, int64_t d, unsigned flags)
+static M2Tc2Plan m2tc2_plan(int64_t N, int64_t d, unsigned flags, bool tf32 = false)
 {
     using namespace m2tc2;
+    const int KROWS = tf32 ? Shape<true>::KROWS : Shape<false>::KROWS;
     M2Tc2Plan p;
     p.ok = false;
     const bool dense = (flags & ST_FLAG_DENSE_CONTROL) != 0;
@@ -543,6 +564,60 @@ static M2TcPlan m2tc_plan(int64_t N, int64_t d, unsigned flags)
     return p;
 }
 
+// Launches the pair kernel and the sum of its partial tiles.
+template <bool TF32>
+static st_status m2_pair_launch(const M2Tc2Plan &q, const void *X, int64_t N, int64_t d, int64_t ldx, float *out, void *ws,
+                                cudaStream_t stream)
+{
+    using S = m2tc2::Shape<TF32>;
+    CUtensorMap tm2;
+    if (!tc::make_tmap_2d(&tm2, TF32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, X, (uint64_t)N,
+                          (uint64_t)d, (uint64_t)ldx * S::ELEM, S::BOXC, S::KROWS,
+                          TF32 ? CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B : CU_TENSOR_MAP_SWIZZLE_128B))
+        return ST_ERR_CUDA;
+    float *part2 = (float *)((unsigned char *)ws + kWsHeaderBytes);
+    if (!ensure_dynamic_smem(moment2_tc_pair_kernel<TF32>, m2tc2::SMEM_BYTES)) return ST_ERR_CUDA;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(2 * q.tab.ntiles * q.tab.nsplit);
+    cfg.blockDim = dim3(m2tc2::THREADS);
+    cfg.dynamicSmemBytes = m2tc2::SMEM_BYTES;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    if (cudaLaunchKernelEx(&cfg, moment2_tc_pair_kernel<TF32>, tm2, part2, (unsigned *)ws, q.chunks_total, q.tab) !=
+        cudaSuccess) {
+        (void)cudaGetLastError();
+        return ST_ERR_CUDA;
+    }
+    moment2_tc_pair_reduce_kernel<<<dim3(q.tab.ntiles, 64), 256, 0, stream>>>(part2, out, (int)d, q.tab);
+    return launch_status();
+}
+
+// fp32 input read as TF32 by the pair kernel (any d that is a multiple of 4: tiles beyond d are zero-filled by the copies)
+size_t moment2_tf32_tc_workspace(int64_t N, int64_t d, unsigned flags)
+{
+    if (N <= 0 || d <= 0 || d % 4 != 0 || d > 4096 || N > (int64_t(1) << 31) - 64) return 0;
+    const M2Tc2Plan q = m2tc2_plan(N, d, flags, true);
+    return q.ok ? kWsHeaderBytes + q.partial_bytes : 0;
+}
+
+st_status moment2_tf32_tc(const void *X, int64_t N, int64_t d, int64_t ldx, float *out, void *ws, size_t ws_bytes,
+                          unsigned flags, cudaStream_t stream)
+{
+    if (d % 4 != 0 || ldx % 4 != 0) return ST_ERR_ALIGN;
+    if (d > 4096 || N > (int64_t(1) << 31) - 64) return ST_ERR_UNSUPPORTED;
+    const M2Tc2Plan q = m2tc2_plan(N, d, flags, true);
+    if (!q.ok) return ST_ERR_UNSUPPORTED;
+    if (!ws || ws_bytes < kWsHeaderBytes + q.partial_bytes) return ST_ERR_WORKSPACE;
+    if (!aligned256(ws)) return ST_ERR_ALIGN;
+    return m2_pair_launch<true>(q, X, N, d, ldx, out, ws, stream);
+}
+
 size_t moment2_bf16_tc_workspace(int64_t N, int64_t d, unsigned flags)
 {
     if (N <= 0 || d <= 0 || d % 8 != 0 || d > 4096 || N > (int64_t(1) << 31) - 64) return 0;
@@ -565,31 +640,7 @@ st_status moment2_bf16_tc(const void *X, int64_t N, int64_t d, int64_t ldx, floa
         if (!q.ok) return ST_ERR_UNSUPPORTED;
         if (!ws || ws_bytes < kWsHeaderBytes + q.partial_bytes) return ST_ERR_WORKSPACE;
         if (!aligned256(ws)) return ST_ERR_ALIGN;
-        CUtensorMap tm2;
-        if (!tc::make_tmap_2d(&tm2, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, X, (uint64_t)N, (uint64_t)d, (uint64_t)ldx * 2,
-                              m2tc2::BOXC, m2tc2::KROWS))
-            return ST_ERR_CUDA;
-        float *part2 = (float *)((unsigned char *)ws + kWsHeaderBytes);
-        if (!ensure_dynamic_smem(moment2_tc_pair_kernel, m2tc2::SMEM_BYTES)) return ST_ERR_CUDA;
-        cudaLaunchConfig_t cfg = {};
-        cfg.gridDim = dim3(2 * q.tab.ntiles * q.tab.nsplit);
-        cfg.blockDim = dim3(m2tc2::THREADS);
-        cfg.dynamicSmemBytes = m2tc2::SMEM_BYTES;
-        cfg.stream = stream;
-        cudaLaunchAttribute attr[1];
-        attr[0].id = cudaLaunchAttributeClusterDimension;
-        attr[0].val.clusterDim.x = 2;
-        attr[0].val.clusterDim.y = 1;
-        attr[0].val.clusterDim.z = 1;
-        cfg.attrs = attr;
-        cfg.numAttrs = 1;
-        if (cudaLaunchKernelEx(&cfg, moment2_tc_pair_kernel, tm2, part2, (unsigned *)ws, q.chunks_total, q.tab) !=
-            cudaSuccess) {
-            (void)cudaGetLastError();
-            return ST_ERR_CUDA;
-        }
-        moment2_tc_pair_reduce_kernel<<<dim3(q.tab.ntiles, 64), 256, 0, stream>>>(part2, out, (int)d, q.tab);
-        return launch_status();
+        return m2_pair_launch<false>(q, X, N, d, ldx, out, ws, stream);
     }
     const M2TcPlan p = m2tc_plan(N, d, flags);
     if (!p.ok) return ST_ERR_UNSUPPORTED;

@@ -108,14 +108,18 @@ __device__ __forceinline__ void tc_commit(uint64_t *bar)
 // Shared-memory matrix descriptor.  Fields (bits): start address >> 4 [0,14), leading byte
 // offset >> 4 [16,30), stride byte offset >> 4 [32,46), descriptor version 1 [46,48),
 // swizzle mode [61,64) (2 = 128-byte swizzle).
-__device__ __forceinline__ uint64_t make_smem_desc(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes)
+// layout: 2 = 128-byte swizzle of 16-byte units; 1 = 128-byte swizzle of 32-byte units, the one form an MN-major
+// operand of 32-bit elements may have (the TMA mode "128B, atom 32B" writes it: rows of 128 bytes whose 32-byte
+// chunk c sits at chunk c ^ (row & 3); the pattern repeats every four rows, so the next group of K starts 512
+// bytes further on).
+__device__ __forceinline__ uint64_t make_smem_desc(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes, uint32_t layout = 2)
 {
     uint64_t d = 0;
     d |= (uint64_t)((saddr >> 4) & 0x3FFF);
     d |= (uint64_t)((lbo_bytes >> 4) & 0x3FFF) << 16;
     d |= (uint64_t)((sbo_bytes >> 4) & 0x3FFF) << 32;
     d |= (uint64_t)1 << 46;
-    d |= (uint64_t)2 << 61;
+    d |= (uint64_t)layout << 61;
     return d;
 }
 
@@ -207,7 +211,8 @@ inline EncodeTiledFn encode_tiled_fn()
 // Row-major [rows, cols] matrix with a row pitch of `pitch_bytes`; box of box_cols x box_rows,
 // 128-byte swizzle, out-of-range elements read as zero.
 inline bool make_tmap_2d(CUtensorMap *m, CUtensorMapDataType dt, const void *base, uint64_t rows, uint64_t cols,
-                         uint64_t pitch_bytes, uint32_t box_cols, uint32_t box_rows)
+                         uint64_t pitch_bytes, uint32_t box_cols, uint32_t box_rows,
+                         CUtensorMapSwizzle swizzle = CU_TENSOR_MAP_SWIZZLE_128B)
 {
     EncodeTiledFn fn = encode_tiled_fn();
     if (!fn) return false;
@@ -216,7 +221,7 @@ inline bool make_tmap_2d(CUtensorMap *m, CUtensorMapDataType dt, const void *bas
     cuuint32_t box[2] = {box_cols, box_rows};
     cuuint32_t estr[2] = {1, 1};
     return fn(m, dt, 2, const_cast<void *>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-              CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              swizzle, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
@@ -279,6 +284,15 @@ __device__ __forceinline__ void mma_bf16_pair(uint32_t d_tmem, uint64_t adesc, u
         "{\n\t.reg .pred p;\n\t"
         "setp.ne.b32 p, %4, 0;\n\t"
         "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+__device__ __forceinline__ void mma_tf32_pair(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::2.kind::tf32 [%0], %1, %2, %3, p;\n\t}"
         ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
         : "memory");
 }

@@ -701,6 +701,47 @@ def test_moment2_bf16_tensor_core_small(st, N, d):
     assert st.st_check_status() == st.ST_OK
 
 
+@pytest.mark.parametrize("N,d", [(1, 4), (31, 8), (100, 36), (33, 128), (1000, 256), (4097, 260), (9000, 520),
+                                 (20000, 1024), (3000, 1028)])
+def test_moment2_tf32_tensor_core_on_fp32_input(st, N, d):
+    """fp32 X read as TF32 by the tensor core (ST_FLAG_TC_TF32): 5e-3 against the oracle on X itself, and 1e-4
+    against the oracle on X with the 13 low mantissa bits cleared, which is what the tensor core multiplies."""
+    X = workloads.draw((N, d), "normal", 900 + N + d)
+    ws = torch.empty(st.st_workspace_bytes(st.ST_OP_SYM_MOMENT2, N, d, st.ST_F32, 0, st.ST_FLAG_TC_TF32),
+                     dtype=torch.uint8, device="cuda")
+    got = expand2(st, st.st_sym_moment2(dev(X), ws=ws, flags=st.ST_FLAG_TC_TF32), d)
+    assert st.st_check_status(ws) == st.ST_OK
+    T, S = oracle.moment2(X)
+    assert oracle.rel_err(got, T, S) <= TOL_TC, (N, d)
+    Xt = (X.view(np.uint32) & np.uint32(0xFFFFE000)).view(np.float32)
+    Tt, St = oracle.moment2(Xt)
+    assert oracle.rel_err(got, Tt, St) <= TOL_F32, (N, d)
+    ctl = expand2(st, st.st_sym_moment2(dev(X), ws=ws, flags=st.ST_FLAG_TC_TF32 | st.ST_FLAG_DENSE_CONTROL), d)
+    assert oracle.rel_err(ctl, Tt, St) <= TOL_F32
+    # a row pitch wider than d
+    Xw = torch.zeros((N, d + 12), device="cuda")
+    Xw[:, :d] = dev(X)
+    out2 = torch.empty(d * (d + 1) // 2, device="cuda")
+    assert st.lib().st_sym_moment2(Xw.data_ptr(), st.ST_F32, N, d, d + 12, out2.data_ptr(), ws.data_ptr(), ws.numel(),
+                                   st.ST_FLAG_TC_TF32, None) == st.ST_OK
+    assert st.st_check_status(ws) == st.ST_OK
+    assert np.array_equal(expand2(st, out2, d), got)
+
+
+def test_moment2_tf32_rejects_what_it_cannot_run(st):
+    L = st.lib()
+    X = torch.zeros((64, 66), device="cuda")
+    out = torch.zeros(66 * 67 // 2, device="cuda")
+    ws = torch.zeros(1 << 22, dtype=torch.uint8, device="cuda")
+    # d not a multiple of 4
+    assert L.st_sym_moment2(X.data_ptr(), st.ST_F32, 64, 66, 66, out.data_ptr(), ws.data_ptr(), ws.numel(),
+                            st.ST_FLAG_TC_TF32, None) == st.ST_ERR_ALIGN
+    # the flag goes with fp32 input only
+    Xb = torch.zeros((64, 64), dtype=torch.bfloat16, device="cuda")
+    assert L.st_sym_moment2(Xb.data_ptr(), st.ST_BF16, 64, 64, 64, out.data_ptr(), ws.data_ptr(), ws.numel(),
+                            st.ST_FLAG_TC_TF32, None) == st.ST_ERR_UNSUPPORTED
+
+
 def test_moment2_bf16_all_ones(st):
     ones = torch.ones((3001, 256), dtype=torch.bfloat16, device="cuda")
     assert torch.all(st.st_sym_moment2(ones) == 3001.0)
