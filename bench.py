@@ -130,6 +130,9 @@ def call_table(cfg):
     t["sym_moment2_large_f32"] = dict(m2l, bytes=4 * c5["N"] * c5["d"] + 4 * tri(c5["d"]), bound="alu", launches=2)
     t["sym_moment2_large_f32_tf32"] = dict(m2l, bytes=4 * c5["N"] * c5["d"] + 4 * tri(c5["d"]), bound="tensor", launches=2,
                                            tensor_scale=TF32_OVER_BF16)
+    # three bf16 partial products per term; the split pass reads X and writes as many bytes, the GEMM passes read them again
+    t["sym_moment2_large_f32_split"] = dict(m2l, bytes=4 * c5["N"] * c5["d"] + 4 * tri(c5["d"]), bound="tensor", launches=3,
+                                            tensor_scale=1.0 / 3.0)
     t["unpack_tri_sym_large"] = dict(flops=0, bytes=4 * (tri(c5["d"]) + c5["d"] ** 2), bound="hbm", launches=1)
     return t
 
@@ -231,7 +234,7 @@ STEP_CALLS = ["sym_moment2_large", "pack_tri_x_k", "unpack_tri_sym_large", "ttm_
 # Timed on their own only (variants and widened rows)
 EXTRA_CALLS = ["mttkrp_tri", "mttkrp_tri_tf32", "ttm_blockdiag", "ttm_blockdiag_split", "sym_moment3_tf32", "sym_moment3_bf16", "sym_moment4_d32",
                "sym_moment4_d32_bf16", "sym_moment4_d64", "sym_moment4_d64_bf16", "thp_tri_x_k", "sym_moment2_large_f32",
-               "sym_moment2_large_f32_tf32"]
+               "sym_moment2_large_f32_tf32", "sym_moment2_large_f32_split"]
 
 
 class Workload:
@@ -599,20 +602,20 @@ def run_ours(args):
         c5 = cfg["moment2_large"]
         X5f = None
         for n in names + EXTRA_CALLS:
-            if n == "sym_moment2_large_f32_tf32":
+            if n in ("sym_moment2_large_f32_tf32", "sym_moment2_large_f32_split"):
                 continue                             # timed together with the fp32 FMA path below
             if n == "sym_moment2_large_f32":       # the fp32 copy of the large input lives only for these two measurements
                 X5f = w.dev["X5"].float()
                 m2f = torch.empty_like(w.out["m2l"])
                 isolated[n] = timer(lambda: st.st_sym_moment2(X5f, out=m2f, ws=w.ws), reps=3, warm=1)
-                if "sym_moment2_large_f32_tf32" in EXTRA_CALLS:
-                    wst = torch.empty(st.st_workspace_bytes(st.ST_OP_SYM_MOMENT2, X5f.shape[0], X5f.shape[1], st.ST_F32, 0,
-                                                            st.ST_FLAG_TC_TF32), dtype=torch.uint8, device=device)
-                    tf = lambda: st.st_sym_moment2(X5f, out=m2f, ws=wst, flags=st.ST_FLAG_TC_TF32)
-                    isolated["sym_moment2_large_f32_tf32"] = timer(tf, reps=10, warm=2)
-                    dirty["sym_moment2_large_f32_tf32"] = timer(tf, reps=5, warm=1, clean=False)
+                for name, flag in (("sym_moment2_large_f32_tf32", st.ST_FLAG_TC_TF32), ("sym_moment2_large_f32_split", st.ST_FLAG_TC_SPLIT)):
+                    wst = torch.empty(st.st_workspace_bytes(st.ST_OP_SYM_MOMENT2, X5f.shape[0], X5f.shape[1], st.ST_F32, 0, flag),
+                                      dtype=torch.uint8, device=device)
+                    tf = lambda: st.st_sym_moment2(X5f, out=m2f, ws=wst, flags=flag)
+                    isolated[name] = timer(tf, reps=10, warm=2)
+                    dirty[name] = timer(tf, reps=5, warm=1, clean=False)
                     if st.st_check_status(wst) != st.ST_OK:
-                        raise RuntimeError("the TF32 second moment reported a device-side error")
+                        raise RuntimeError("the tensor-core second moment on fp32 input reported a device-side error")
                     del wst
                 del X5f, m2f
                 continue

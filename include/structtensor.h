@@ -78,7 +78,8 @@ typedef enum { ST_OP_SYM_MOMENT2 = 0, ST_OP_SYM_MOMENT3 = 1, ST_OP_MTTKRP_TRI = 
                                     space (a control for measurements; see each call) */
 #define ST_FLAG_TC_TF32       2u /* st_ttm_blockdiag, st_mttkrp_tri, st_sym_moment3, st_sym_moment2 (fp32 input): tensor cores, operands read as TF32 */
 #define ST_FLAG_TC_BF16       4u /* st_sym_moment3, st_sym_moment4: tensor cores, operands rounded to bf16 */
-#define ST_FLAG_TC_SPLIT      8u /* st_ttm_blockdiag, st_ttm_packed, st_mttkrp_tri, st_mttkrp_slice: tensor cores with
+#define ST_FLAG_TC_SPLIT      8u /* st_ttm_blockdiag, st_ttm_packed, st_mttkrp_tri, st_mttkrp_slice (and st_sym_moment2 on fp32 input,
+                                    see there): tensor cores with
                                     both operands split into two bf16 parts and three of the four partial products
                                     kept: meets the 1e-4 tolerance of the fp32 path, at the speed of the HBM stream
                                     (needs K % 4 == 0, R % 32 == 0, R <= 128, and the split factor, 4*K*R bytes rounded up to
@@ -141,6 +142,10 @@ size_t st_workspace_bytes(st_op op, int64_t a, int64_t b, int64_t c, int64_t e, 
  * mantissa bits are ignored: both factors of every product are truncated, so sums of positive products come out
  * low by about 1e-3 relative), fp32 accumulation; 5e-3 tolerance; needs d % 4 == 0, ldx % 4 == 0, d <= 4096;
  * about 15 times faster than the fp32 FMA path at d = 1024.
+ * ST_FLAG_TC_SPLIT (ST_F32 input only): every x is split into hi = bf16(x) and lo = bf16(x - hi) by a first pass
+ * (the workspace holds both parts: 4 bytes per element of X), then hi^T hi + hi^T lo + lo^T hi on the tensor
+ * cores with fp32 accumulation: the tolerance of the fp32 path (1e-4) about five times faster; d % 8 == 0,
+ * ldx % 4 == 0, d <= 4096, N <= 2^29.
  * ST_FLAG_DENSE_CONTROL: all d*d products are computed (lower-triangle tiles too) and
  * the lower results discarded; the output is the same. */
 st_status st_sym_moment2(const void *X, st_dtype xdt, int64_t N, int64_t d, int64_t ldx,

@@ -24,6 +24,9 @@ size_t moment2_bf16_tc_workspace(int64_t N, int64_t d, unsigned flags);
 st_status moment2_tf32_tc(const void *X, int64_t N, int64_t d, int64_t ldx, float *out, void *ws,
                           size_t ws_bytes, unsigned flags, cudaStream_t stream);
 size_t moment2_tf32_tc_workspace(int64_t N, int64_t d, unsigned flags);
+st_status moment2_split_tc(const float *X, int64_t N, int64_t d, int64_t ldx, float *out, void *ws, size_t ws_bytes,
+                           unsigned flags, cudaStream_t stream);
+size_t moment2_split_tc_workspace(int64_t N, int64_t d, unsigned flags);
 bool moment2_small_applies(int64_t N, int64_t d);
 size_t moment2_small_workspace(int64_t N, int64_t d, unsigned flags);
 st_status moment2_small(const float *X, int64_t N, int64_t d, int64_t ldx, float *out, void *ws, size_t ws_bytes,
@@ -421,8 +424,11 @@ static st_status moment2_f32(const float *X, int64_t N, int64_t d, int64_t ldx, 
 size_t moment2_workspace(int64_t N, int64_t d, int xdt, unsigned flags)
 {
     if (N <= 0 || d <= 0) return 0;
-    if (xdt == ST_BF16) return (flags & ST_FLAG_TC_TF32) ? 0 : moment2_bf16_tc_workspace(N, d, flags);
+    const unsigned tc = flags & (ST_FLAG_TC_TF32 | ST_FLAG_TC_SPLIT);
+    if (tc == (ST_FLAG_TC_TF32 | ST_FLAG_TC_SPLIT)) return 0;
+    if (xdt == ST_BF16) return tc ? 0 : moment2_bf16_tc_workspace(N, d, flags);
     if (xdt == ST_F32 && (flags & ST_FLAG_TC_TF32)) return moment2_tf32_tc_workspace(N, d, flags & ~ST_FLAG_TC_TF32);
+    if (xdt == ST_F32 && (flags & ST_FLAG_TC_SPLIT)) return moment2_split_tc_workspace(N, d, flags & ~ST_FLAG_TC_SPLIT);
     if (xdt != ST_F32 || d > 32768) return 0;
     const M2Plan p = moment2_plan(N, d, flags);
     size_t need = kWsHeaderBytes + p.ticket_bytes + p.partial_bytes;
@@ -445,12 +451,16 @@ extern "C" st_status st_sym_moment2(const void *X, st_dtype xdt, int64_t N, int6
     if (!X || !out_packed) return ST_ERR_NULL;
     if (N <= 0 || d <= 0 || ldx < d) return ST_ERR_SHAPE;
     if (xdt != ST_F32 && xdt != ST_BF16) return ST_ERR_DTYPE;
-    if (flags & ~(ST_FLAG_DENSE_CONTROL | ST_FLAG_TC_TF32)) return ST_ERR_UNSUPPORTED;
-    if ((flags & ST_FLAG_TC_TF32) && xdt != ST_F32) return ST_ERR_UNSUPPORTED;
+    if (flags & ~(ST_FLAG_DENSE_CONTROL | ST_FLAG_TC_TF32 | ST_FLAG_TC_SPLIT)) return ST_ERR_UNSUPPORTED;
+    if ((flags & (ST_FLAG_TC_TF32 | ST_FLAG_TC_SPLIT)) && xdt != ST_F32) return ST_ERR_UNSUPPORTED;
+    if ((flags & ST_FLAG_TC_TF32) && (flags & ST_FLAG_TC_SPLIT)) return ST_ERR_UNSUPPORTED;
     if (!st::aligned16(X) || !st::aligned16(out_packed)) return ST_ERR_ALIGN;
     if (xdt == ST_BF16)
         return st::moment2_bf16_tc(X, N, d, ldx, out_packed, ws, ws_bytes, flags, (cudaStream_t)stream);
     if (flags & ST_FLAG_TC_TF32)
         return st::moment2_tf32_tc(X, N, d, ldx, out_packed, ws, ws_bytes, flags & ~ST_FLAG_TC_TF32, (cudaStream_t)stream);
+    if (flags & ST_FLAG_TC_SPLIT)
+        return st::moment2_split_tc((const float *)X, N, d, ldx, out_packed, ws, ws_bytes, flags & ~ST_FLAG_TC_SPLIT,
+                                    (cudaStream_t)stream);
     return st::moment2_f32((const float *)X, N, d, ldx, out_packed, ws, ws_bytes, flags, (cudaStream_t)stream);
 }

@@ -27,6 +27,7 @@
 // warps 2..5 = epilogue (TMEM -> registers -> global), one per 32-lane quarter of TMEM.
 #include "tc_common.cuh"
 #include "st_index.cuh"
+#include <cuda_bf16.h>
 
 namespace st {
 
@@ -284,8 +285,11 @@ struct TileTable {
 template <bool TF32>
 __global__ void __launch_bounds__(m2tc2::THREADS, 1)
 moment2_tc_pair_kernel(const __grid_constant__ CUtensorMap tmap, float *__restrict__ partials, unsigned *status,
-                       int chunks_total, const __grid_constant__ m2tc2::TileTable tab)
+                       int chunks_total, const __grid_constant__ m2tc2::TileTable tab, int seg_chunks, int lo_row0)
 {
+    // seg_chunks > 0: the rows of the tensor are [hi part of X; lo part of X] (lo_row0 = first row of the lo part)
+    // and the sample loop runs over three segments of seg_chunks stages: A and B from hi, A from hi and B from lo,
+    // A from lo and B from hi -- the sum is hi^T hi + hi^T lo + lo^T hi, symmetric, so the tiles stay the upper ones.
     using namespace m2tc2;
     using namespace tc;
     using S = Shape<TF32>;
@@ -302,7 +306,7 @@ moment2_tc_pair_kernel(const __grid_constant__ CUtensorMap tmap, float *__restri
     const int cluster = blockIdx.x >> 1;
     const int tile = cluster / tab.nsplit, split = cluster - tile * tab.nsplit;
     const int tm = tab.tm[tile], tn = tab.tn[tile];
-    const bool diag = (tm == tn);                       // A columns == B columns in every block
+    const bool diag = (tm == tn) && seg_chunks == 0;    // A columns == B columns (and rows) in every block: one load serves both
     const int chunks_per_split = (chunks_total + tab.nsplit - 1) / tab.nsplit;
     const int c_begin = split * chunks_per_split;
     int c_end = c_begin + chunks_per_split;
@@ -349,12 +353,18 @@ moment2_tc_pair_kernel(const __grid_constant__ CUtensorMap tmap, float *__restri
                 unsigned char *st_base = smem + (size_t)s * STAGE_BYTES;
                 if (rank == 0) mbar_expect_tx(&full[s], 2 * own_tx);
                 const uint32_t bar = map_to_cta(smem_u32(&full[s]), 0);
-                const int row = (c_begin + c) * KROWS;
+                int row_a = (c_begin + c) * KROWS, row_b = row_a;
+                if (seg_chunks > 0) {
+                    const int gc = c_begin + c, seg = gc / seg_chunks;
+                    row_a = row_b = (gc - seg * seg_chunks) * KROWS;
+                    if (seg == 1) row_b += lo_row0;
+                    if (seg == 2) row_a += lo_row0;
+                }
                 for (int b = 0; b < NBOX; ++b)          // B half (and A on diagonal tiles)
-                    tma_load_2d_pair(st_base + b * BOX_BYTES, &tmap, bar, tn * BN + (int)rank * HALF + b * BOXC, row);
+                    tma_load_2d_pair(st_base + b * BOX_BYTES, &tmap, bar, tn * BN + (int)rank * HALF + b * BOXC, row_b);
                 if (!diag)
                     for (int b = 0; b < NBOX; ++b)      // A rows of this block
-                        tma_load_2d_pair(st_base + (NBOX + b) * BOX_BYTES, &tmap, bar, tm * BM + (int)rank * HALF + b * BOXC, row);
+                        tma_load_2d_pair(st_base + (NBOX + b) * BOX_BYTES, &tmap, bar, tm * BM + (int)rank * HALF + b * BOXC, row_a);
             }
         }
     } else if (warp == 1) {
@@ -474,7 +484,7 @@ struct M2Tc2Plan {
     bool ok;
 };
 
-static M2Tc2Plan m2tc2_plan(int64_t N, int64_t d, unsigned flags, bool tf32 = false)
+static M2Tc2Plan m2tc2_plan(int64_t N, int64_t d, unsigned flags, bool tf32 = false, int segments = 1)
 {
     using namespace m2tc2;
     const int KROWS = tf32 ? Shape<true>::KROWS : Shape<false>::KROWS;
@@ -493,7 +503,7 @@ static M2Tc2Plan m2tc2_plan(int64_t N, int64_t d, unsigned flags, bool tf32 = fa
         }
     for (int i = n; i < MAX_TILES; ++i) p.tab.tm[i] = p.tab.tn[i] = 0;
     p.tab.ntiles = n;
-    const int64_t chunks = (N + KROWS - 1) / KROWS;
+    const int64_t chunks = segments * ((N + KROWS - 1) / KROWS);
     if (chunks > (int64_t(1) << 30)) return p;
     p.chunks_total = (int)chunks;
     int64_t per = (sm_count_or_default() / 2) / n;   // clusters per tile: equal, so that sample ranges run in step
@@ -567,7 +577,7 @@ static M2TcPlan m2tc_plan(int64_t N, int64_t d, unsigned flags)
 // Launches the pair kernel and the sum of its partial tiles.
 template <bool TF32>
 static st_status m2_pair_launch(const M2Tc2Plan &q, const void *X, int64_t N, int64_t d, int64_t ldx, float *out, void *ws,
-                                cudaStream_t stream)
+                                cudaStream_t stream, size_t part_off = kWsHeaderBytes, int seg_chunks = 0, int lo_row0 = 0)
 {
     using S = m2tc2::Shape<TF32>;
     CUtensorMap tm2;
@@ -575,7 +585,7 @@ static st_status m2_pair_launch(const M2Tc2Plan &q, const void *X, int64_t N, in
                           (uint64_t)d, (uint64_t)ldx * S::ELEM, S::BOXC, S::KROWS,
                           TF32 ? CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B : CU_TENSOR_MAP_SWIZZLE_128B))
         return ST_ERR_CUDA;
-    float *part2 = (float *)((unsigned char *)ws + kWsHeaderBytes);
+    float *part2 = (float *)((unsigned char *)ws + part_off);
     if (!ensure_dynamic_smem(moment2_tc_pair_kernel<TF32>, m2tc2::SMEM_BYTES)) return ST_ERR_CUDA;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(2 * q.tab.ntiles * q.tab.nsplit);
@@ -589,8 +599,8 @@ static st_status m2_pair_launch(const M2Tc2Plan &q, const void *X, int64_t N, in
     attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    if (cudaLaunchKernelEx(&cfg, moment2_tc_pair_kernel<TF32>, tm2, part2, (unsigned *)ws, q.chunks_total, q.tab) !=
-        cudaSuccess) {
+    if (cudaLaunchKernelEx(&cfg, moment2_tc_pair_kernel<TF32>, tm2, part2, (unsigned *)ws, q.chunks_total, q.tab, seg_chunks,
+                           lo_row0) != cudaSuccess) {
         (void)cudaGetLastError();
         return ST_ERR_CUDA;
     }
@@ -616,6 +626,77 @@ st_status moment2_tf32_tc(const void *X, int64_t N, int64_t d, int64_t ldx, floa
     if (!ws || ws_bytes < kWsHeaderBytes + q.partial_bytes) return ST_ERR_WORKSPACE;
     if (!aligned256(ws)) return ST_ERR_ALIGN;
     return m2_pair_launch<true>(q, X, N, d, ldx, out, ws, stream);
+}
+
+// ---------------------------------------------------------------------------------------------
+// fp32 input at the fp32 tolerance on the tensor cores (ST_FLAG_TC_SPLIT): every x is written once as
+// hi = bf16(x) and lo = bf16(x - hi) (x - hi - lo is below 2^-16 |x|), and the pair kernel adds
+// hi^T hi + hi^T lo + lo^T hi over three passes of the samples (lo^T lo is below 2^-16 of the result).
+// The split pass reads X once and writes the same number of bytes; the three passes then run at the bf16 rate.
+__global__ void __launch_bounds__(256)
+moment2_split_rows_kernel(const float *__restrict__ X, int64_t N, int64_t Np, int d, int64_t ldx, __nv_bfloat16 *__restrict__ Z)
+{
+    // Z: [2 Np, d]; rows 0 .. Np-1 hi, rows Np .. 2Np-1 lo; rows N .. Np-1 of either part are zero
+    const int64_t quads = (int64_t)Np * (d / 4);
+    for (int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; e < quads; e += (int64_t)gridDim.x * blockDim.x) {
+        const int64_t n = e / (d / 4);
+        const int c = (int)(e - n * (d / 4)) * 4;
+        float4 x = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (n < N) x = __ldcs(reinterpret_cast<const float4 *>(X + n * ldx + c));
+        const __nv_bfloat162 h0 = __floats2bfloat162_rn(x.x, x.y), h1 = __floats2bfloat162_rn(x.z, x.w);
+        const float2 f0 = __bfloat1622float2(h0), f1 = __bfloat1622float2(h1);
+        const __nv_bfloat162 l0 = __floats2bfloat162_rn(x.x - f0.x, x.y - f0.y), l1 = __floats2bfloat162_rn(x.z - f1.x, x.w - f1.y);
+        *reinterpret_cast<uint2 *>(Z + n * d + c) =
+            make_uint2(*reinterpret_cast<const uint32_t *>(&h0), *reinterpret_cast<const uint32_t *>(&h1));
+        *reinterpret_cast<uint2 *>(Z + (Np + n) * d + c) =
+            make_uint2(*reinterpret_cast<const uint32_t *>(&l0), *reinterpret_cast<const uint32_t *>(&l1));
+    }
+}
+
+struct M2SplitPlan {
+    M2Tc2Plan q;
+    int64_t Np;
+    size_t z_off, part_off, total;
+    bool ok;
+};
+
+static M2SplitPlan m2_split_plan(int64_t N, int64_t d, unsigned flags)
+{
+    M2SplitPlan p{};
+    p.ok = false;
+    if (N <= 0 || d <= 0 || d % 8 != 0 || d > 4096 || N > (int64_t(1) << 29)) return p;
+    const int KROWS = m2tc2::Shape<false>::KROWS;
+    p.Np = (N + KROWS - 1) / KROWS * KROWS;
+    p.q = m2tc2_plan(N, d, flags, false, 3);
+    if (!p.q.ok) return p;
+    p.z_off = kWsHeaderBytes;
+    p.part_off = round_up(p.z_off + (size_t)2 * p.Np * d * sizeof(__nv_bfloat16), 256);
+    p.total = p.part_off + p.q.partial_bytes;
+    p.ok = true;
+    return p;
+}
+
+size_t moment2_split_tc_workspace(int64_t N, int64_t d, unsigned flags)
+{
+    const M2SplitPlan p = m2_split_plan(N, d, flags);
+    return p.ok ? p.total : 0;
+}
+
+st_status moment2_split_tc(const float *X, int64_t N, int64_t d, int64_t ldx, float *out, void *ws, size_t ws_bytes,
+                           unsigned flags, cudaStream_t stream)
+{
+    if (d % 8 != 0 || ldx % 4 != 0) return ST_ERR_ALIGN;
+    const M2SplitPlan p = m2_split_plan(N, d, flags);
+    if (!p.ok) return ST_ERR_UNSUPPORTED;
+    if (!ws || ws_bytes < p.total) return ST_ERR_WORKSPACE;
+    if (!aligned256(ws)) return ST_ERR_ALIGN;
+    __nv_bfloat16 *Z = (__nv_bfloat16 *)((unsigned char *)ws + p.z_off);
+    const int64_t quads = p.Np * (d / 4);
+    const int64_t want = (quads + 255) / 256;
+    const int64_t cap = (int64_t)sm_count_or_default() * 16;
+    moment2_split_rows_kernel<<<(unsigned)(want < cap ? want : cap), 256, 0, stream>>>(X, N, p.Np, (int)d, ldx, Z);
+    if (cudaGetLastError() != cudaSuccess) return ST_ERR_CUDA;
+    return m2_pair_launch<false>(p.q, Z, 2 * p.Np, d, d, out, ws, stream, p.part_off, p.q.chunks_total / 3, (int)p.Np);
 }
 
 size_t moment2_bf16_tc_workspace(int64_t N, int64_t d, unsigned flags)

@@ -728,6 +728,39 @@ def test_moment2_tf32_tensor_core_on_fp32_input(st, N, d):
     assert np.array_equal(expand2(st, out2, d), got)
 
 
+@pytest.mark.parametrize("N,d", [(1, 8), (63, 16), (100, 40), (65, 128), (1000, 256), (4097, 264), (9000, 520),
+                                 (20000, 1024), (3000, 1032)])
+def test_moment2_split_tensor_core_on_fp32_input(st, N, d):
+    """fp32 X as hi + lo bf16 parts, three partial products on the tensor cores (ST_FLAG_TC_SPLIT): the fp32 tolerance."""
+    X = workloads.draw((N, d), "normal", 950 + N + d)
+    ws = torch.empty(st.st_workspace_bytes(st.ST_OP_SYM_MOMENT2, N, d, st.ST_F32, 0, st.ST_FLAG_TC_SPLIT),
+                     dtype=torch.uint8, device="cuda")
+    got = expand2(st, st.st_sym_moment2(dev(X), ws=ws, flags=st.ST_FLAG_TC_SPLIT), d)
+    assert st.st_check_status(ws) == st.ST_OK
+    T, S = oracle.moment2(X)
+    assert oracle.rel_err(got, T, S) <= TOL_F32, (N, d)
+    ctl = expand2(st, st.st_sym_moment2(dev(X), ws=ws, flags=st.ST_FLAG_TC_SPLIT | st.ST_FLAG_DENSE_CONTROL), d)
+    assert oracle.rel_err(ctl, T, S) <= TOL_F32
+    # a row pitch wider than d, and the same result twice
+    Xw = torch.zeros((N, d + 12), device="cuda")
+    Xw[:, :d] = dev(X)
+    out2 = torch.empty(d * (d + 1) // 2, device="cuda")
+    assert st.lib().st_sym_moment2(Xw.data_ptr(), st.ST_F32, N, d, d + 12, out2.data_ptr(), ws.data_ptr(), ws.numel(),
+                                   st.ST_FLAG_TC_SPLIT, None) == st.ST_OK
+    assert st.st_check_status(ws) == st.ST_OK
+    assert np.array_equal(expand2(st, out2, d), got)
+
+
+def test_moment2_split_sums_of_squares_do_not_drift(st):
+    """All-positive sums over many samples: the accumulation chain is cut often enough that the diagonal stays
+    inside the fp32 tolerance (a tensor-core accumulator rounds towards zero)."""
+    N, d = 200000, 64
+    X = np.abs(workloads.draw((N, d), "normal", 77)) + 0.5
+    got = expand2(st, st.st_sym_moment2(dev(X), flags=st.ST_FLAG_TC_SPLIT), d)
+    T, S = oracle.moment2(X)
+    assert oracle.rel_err(got, T, S) <= TOL_F32
+
+
 def test_moment2_tf32_rejects_what_it_cannot_run(st):
     L = st.lib()
     X = torch.zeros((64, 66), device="cuda")
