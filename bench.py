@@ -104,7 +104,7 @@ def call_table(cfg):
     t["sym_moment3_bf16"] = dict(m3, bound="tensor", launches=2, tensor_scale=1.0)
     for d4 in cfg["moment4_d"]:
         m4 = dict(flops=2 * c2["N"] * simp4(d4) + c2["N"] * tri(d4), bytes=4 * (c2["N"] * d4 + simp4(d4)))
-        t["sym_moment4_d%d" % d4] = dict(m4, bound="alu", launches=4)
+        t["sym_moment4_d%d" % d4] = dict(m4, bound="tensor", launches=4, tensor_scale=1.0 / 3.0)   # split pair features, three products
         t["sym_moment4_d%d_bf16" % d4] = dict(m4, bound="tensor", launches=4, tensor_scale=1.0)
     t["unpack_tet_sym"] = dict(flops=0, bytes=4 * (tet(c2["d"]) + c2["d"] ** 3), bound="hbm", launches=1)
     nnz3 = tri(c3["I"]) * c3["K"]

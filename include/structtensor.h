@@ -179,9 +179,11 @@ st_status st_sym_moment3(const float *X, int64_t N, int64_t d, int64_t ldx,
  * lexicographic order of the unique set (slab i holds the tetrahedron (j,k,l) of side d-i).
  * Computed as the second moment of the pair features P[n,(i,j)] = X[n,i] X[n,j], i<=j, which
  * the call materialises in the workspace (N * roundup(d(d+1)/2, 64) elements; query the size
- * with ST_OP_SYM_MOMENT4), followed by a gather of the entries with j <= k.  fp32 arithmetic by
- * default (1e-4 tolerance); ST_FLAG_TC_BF16 stores P in bf16 and runs the tensor-core triangular
- * tile GEMM (5e-3 tolerance for N >= 1000). */
+ * with ST_OP_SYM_MOMENT4), followed by a gather of the entries with j <= k.  Default: the 1e-4 tolerance of
+ * the fp32 paths -- for d <= 89 every fp32 pair product is stored as hi + lo bf16 parts and the tensor-core
+ * triangular tile GEMM adds three partial products (hi hi + hi lo + lo hi) with fp32 accumulation; for larger d
+ * an fp32 P and fp32 FMA arithmetic.  ST_FLAG_TC_BF16 stores P rounded to bf16 and runs one pass of the same
+ * GEMM (5e-3 tolerance for N >= 1000). */
 st_status st_sym_moment4(const float *X, int64_t N, int64_t d, int64_t ldx,
                          float *out_packed, void *ws, size_t ws_bytes, unsigned flags,
                          void *stream);

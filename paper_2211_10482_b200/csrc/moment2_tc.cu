@@ -676,6 +676,26 @@ static M2SplitPlan m2_split_plan(int64_t N, int64_t d, unsigned flags)
     return p;
 }
 
+// The three-segment product for a caller that has written the parts itself (the fourth moment makes its pair
+// features straight into this form): Z = [hi rows; lo rows], each part N rounded up to 64 rows with zero rows
+// at the end, d columns, bf16.
+int64_t moment2_split_part_rows(int64_t N) { return (N + 63) / 64 * 64; }
+
+size_t moment2_split_parts_workspace(int64_t N, int64_t d)
+{
+    const M2SplitPlan p = m2_split_plan(N, d, 0);
+    return p.ok ? kWsHeaderBytes + p.q.partial_bytes : 0;
+}
+
+st_status moment2_split_tc_parts(const void *Z, int64_t N, int64_t d, float *out, void *ws, size_t ws_bytes, cudaStream_t stream)
+{
+    const M2SplitPlan p = m2_split_plan(N, d, 0);
+    if (!p.ok) return ST_ERR_UNSUPPORTED;
+    if (!ws || ws_bytes < kWsHeaderBytes + p.q.partial_bytes) return ST_ERR_WORKSPACE;
+    if (!aligned256(ws) || !aligned16(Z)) return ST_ERR_ALIGN;
+    return m2_pair_launch<false>(p.q, Z, 2 * p.Np, d, d, out, ws, stream, kWsHeaderBytes, p.q.chunks_total / 3, (int)p.Np);
+}
+
 size_t moment2_split_tc_workspace(int64_t N, int64_t d, unsigned flags)
 {
     const M2SplitPlan p = m2_split_plan(N, d, flags);

@@ -7,8 +7,10 @@
 //     out[s(i,j,k,l)] = sum_n P[n,(i,j)] P[n,(k,l)],
 // and (i,j,k,l) is a unique 4-tuple exactly when j <= k.  Three steps, all on the GPU:
 //   1. pair_expand_kernel    P [N, dP], dP = d(d+1)/2 rounded up to 64 (zero columns), fp32 or bf16
-//   2. st_sym_moment2 on P   the packed upper triangle of P^T P (fp32 kernels, or the bf16
-//                            tensor-core triangular tile GEMM with ST_FLAG_TC_BF16)
+//   2. st_sym_moment2 on P   the packed upper triangle of P^T P: the tensor-core triangular tile GEMM, on P rounded
+//                            to bf16 (ST_FLAG_TC_BF16, 5e-3) or, for the fp32 tolerance, on P written as hi + lo
+//                            bf16 parts and multiplied in three partial products (d <= 89: the pair features
+//                            fit the kernel's 4096 columns); beyond that the fp32 FMA kernel on an fp32 P
 //   3. simplex_gather_kernel rows (i,j,k,*) of the 4-simplex are runs of row (i,j), columns
 //                            (k,k)..(k,d-1) of that triangle: contiguous on both sides
 // Step 2 works on the symmetric pair-by-pair matrix, whose unique set (pairs p <= q) is about
@@ -21,6 +23,9 @@
 namespace st {
 
 size_t moment2_workspace(int64_t N, int64_t d, int xdt, unsigned flags);
+int64_t moment2_split_part_rows(int64_t N);
+size_t moment2_split_parts_workspace(int64_t N, int64_t d);
+st_status moment2_split_tc_parts(const void *Z, int64_t N, int64_t d, float *out, void *ws, size_t ws_bytes, cudaStream_t stream);
 
 namespace m4 {
 
@@ -29,9 +34,9 @@ constexpr int EXP_ROWS = 32;        // sample rows per pass of a block
 constexpr int EXP_THREADS = 192;
 
 struct Plan {
-    int64_t dP, p_bytes, m2_elems, m2_ws;
+    int64_t dP, p_bytes, m2_elems, m2_ws, Np;
     size_t off_p, off_m2, off_ws, total;
-    bool bf16, ok;
+    bool bf16, split, ok;
 };
 
 static Plan plan(int64_t N, int64_t d, unsigned flags)
@@ -41,9 +46,18 @@ static Plan plan(int64_t N, int64_t d, unsigned flags)
     if (N <= 0 || d < 1 || d > MAX_D) return p;
     p.bf16 = (flags & ST_FLAG_TC_BF16) != 0;
     p.dP = (tri_rows(d) + 63) / 64 * 64;
-    p.p_bytes = N * p.dP * (p.bf16 ? 2 : 4);
     p.m2_elems = tri_rows(p.dP);
-    p.m2_ws = (int64_t)moment2_workspace(N, p.dP, p.bf16 ? ST_BF16 : ST_F32, 0);
+    // fp32 result: the pair features are written as hi + lo bf16 parts and multiplied on the tensor cores in three
+    // partial products (the fp32 tolerance) wherever that kernel reaches; else fp32 features and the fp32 FMA kernel
+    p.Np = moment2_split_part_rows(N);
+    p.m2_ws = p.bf16 ? 0 : (int64_t)moment2_split_parts_workspace(N, p.dP);
+    p.split = !p.bf16 && p.m2_ws != 0;
+    if (p.split) {
+        p.p_bytes = 2 * p.Np * p.dP * 2;
+    } else {
+        p.p_bytes = N * p.dP * (p.bf16 ? 2 : 4);
+        p.m2_ws = (int64_t)moment2_workspace(N, p.dP, p.bf16 ? ST_BF16 : ST_F32, 0);
+    }
     if (p.m2_ws == 0) return p;
     p.off_p = kWsHeaderBytes;
     p.off_m2 = round_up(p.off_p + (size_t)p.p_bytes, 256);
@@ -67,9 +81,12 @@ __device__ __forceinline__ void store4(__nv_bfloat16 *dst, float a, float b, flo
 // columns.  A block stages EXP_ROWS rows of X per pass (one extra column holds zero); a thread owns
 // four adjacent columns of P, decodes their index pairs once and writes them for every staged
 // row with one 8- or 16-byte store.  HBM bound: the write of P.
-template <typename OutT>
+// SPLIT: every product p is written twice, hi = bf16(p) in row n and lo = bf16(p - hi) in row Np + n; the rows
+// N .. Np-1 of either part are zero.
+template <typename OutT, bool SPLIT>
 __global__ void __launch_bounds__(EXP_THREADS)
-pair_expand_kernel(const float *__restrict__ X, int64_t N, int d, int64_t ldx, OutT *__restrict__ P, int dP, int npairs)
+pair_expand_kernel(const float *__restrict__ X, int64_t N, int d, int64_t ldx, OutT *__restrict__ P, int dP, int npairs,
+                   int64_t Np)
 {
     extern __shared__ __align__(16) float xs[];                       // [EXP_ROWS][d + 1], column d is zero
     const int pitch = d + 1;
@@ -87,20 +104,28 @@ pair_expand_kernel(const float *__restrict__ X, int64_t N, int d, int64_t ldx, O
         }
     }
     const bool inside = p < dP;
-    for (int64_t row0 = (int64_t)blockIdx.y * EXP_ROWS; row0 < N; row0 += (int64_t)gridDim.y * EXP_ROWS) {
-        const int nrows = N - row0 < EXP_ROWS ? (int)(N - row0) : EXP_ROWS;
+    const int64_t rows_total = SPLIT ? Np : N;
+    for (int64_t row0 = (int64_t)blockIdx.y * EXP_ROWS; row0 < rows_total; row0 += (int64_t)gridDim.y * EXP_ROWS) {
+        const int nrows = rows_total - row0 < EXP_ROWS ? (int)(rows_total - row0) : EXP_ROWS;
         __syncthreads();
         for (int e = threadIdx.x; e < nrows * pitch; e += EXP_THREADS) {
             const int r = e / pitch, c = e - r * pitch;
-            xs[e] = c < d ? X[(row0 + r) * ldx + c] : 0.f;
+            xs[e] = (c < d && (!SPLIT || row0 + r < N)) ? X[(row0 + r) * ldx + c] : 0.f;
         }
         __syncthreads();
         if (!inside) continue;
         OutT *dst = P + row0 * dP + p;
         const float *x = xs;
 #pragma unroll 4
-        for (int r = 0; r < nrows; ++r, dst += dP, x += pitch)
-            store4(dst, x[ci[0]] * x[cj[0]], x[ci[1]] * x[cj[1]], x[ci[2]] * x[cj[2]], x[ci[3]] * x[cj[3]]);
+        for (int r = 0; r < nrows; ++r, dst += dP, x += pitch) {
+            const float v0 = x[ci[0]] * x[cj[0]], v1 = x[ci[1]] * x[cj[1]], v2 = x[ci[2]] * x[cj[2]], v3 = x[ci[3]] * x[cj[3]];
+            store4(dst, v0, v1, v2, v3);
+            if (SPLIT) {
+                const float h0 = __bfloat162float(__float2bfloat16_rn(v0)), h1 = __bfloat162float(__float2bfloat16_rn(v1)),
+                            h2 = __bfloat162float(__float2bfloat16_rn(v2)), h3 = __bfloat162float(__float2bfloat16_rn(v3));
+                store4(dst + Np * dP, v0 - h0, v1 - h1, v2 - h2, v3 - h3);
+            }
+        }
     }
 }
 
@@ -153,18 +178,22 @@ extern "C" st_status st_sym_moment4(const float *X, int64_t N, int64_t d, int64_
     const int npairs = (int)tri_rows(d);
     const size_t smem = (size_t)EXP_ROWS * (d + 1) * sizeof(float);
     const unsigned col_groups = (unsigned)((p.dP + 4 * EXP_THREADS - 1) / (4 * EXP_THREADS));
-    const int64_t passes = (N + EXP_ROWS - 1) / EXP_ROWS;
+    const int64_t passes = ((p.split ? p.Np : N) + EXP_ROWS - 1) / EXP_ROWS;
     const int64_t cap = ((int64_t)sm_count_or_default() * 8 + col_groups - 1) / col_groups;
     const dim3 grid(col_groups, (unsigned)(passes < cap ? passes : cap));
-    if (p.bf16)
-        pair_expand_kernel<__nv_bfloat16><<<grid, EXP_THREADS, smem, stream>>>(X, N, (int)d, ldx, (__nv_bfloat16 *)(w + p.off_p),
-                                                                                (int)p.dP, npairs);
+    if (p.split)
+        pair_expand_kernel<__nv_bfloat16, true><<<grid, EXP_THREADS, smem, stream>>>(
+            X, N, (int)d, ldx, (__nv_bfloat16 *)(w + p.off_p), (int)p.dP, npairs, p.Np);
+    else if (p.bf16)
+        pair_expand_kernel<__nv_bfloat16, false><<<grid, EXP_THREADS, smem, stream>>>(
+            X, N, (int)d, ldx, (__nv_bfloat16 *)(w + p.off_p), (int)p.dP, npairs, p.Np);
     else
-        pair_expand_kernel<float><<<grid, EXP_THREADS, smem, stream>>>(X, N, (int)d, ldx, (float *)(w + p.off_p), (int)p.dP,
-                                                                        npairs);
+        pair_expand_kernel<float, false><<<grid, EXP_THREADS, smem, stream>>>(X, N, (int)d, ldx, (float *)(w + p.off_p),
+                                                                               (int)p.dP, npairs, p.Np);
     if (cudaGetLastError() != cudaSuccess) return ST_ERR_CUDA;
-    const st_status rc = st_sym_moment2(w + p.off_p, p.bf16 ? ST_BF16 : ST_F32, N, p.dP, p.dP, M2, w + p.off_ws,
-                                        (size_t)p.m2_ws, 0, stream_);
+    const st_status rc = p.split ? moment2_split_tc_parts(w + p.off_p, N, p.dP, M2, w + p.off_ws, (size_t)p.m2_ws, stream)
+                                 : st_sym_moment2(w + p.off_p, p.bf16 ? ST_BF16 : ST_F32, N, p.dP, p.dP, M2, w + p.off_ws,
+                                                  (size_t)p.m2_ws, 0, stream_);
     if (rc != ST_OK) return rc;
     simplex_gather_kernel<<<(unsigned)tet_rows(d), 64, 0, stream>>>(M2, out_packed, (int)d, p.dP, (unsigned *)w,
                                                                     (const unsigned *)(w + p.off_ws));
