@@ -11,8 +11,8 @@
 //                            to bf16 (ST_FLAG_TC_BF16, 5e-3) or, for the fp32 tolerance, on P written as hi + lo
 //                            bf16 parts and multiplied in three partial products (d <= 89: the pair features
 //                            fit the kernel's 4096 columns); beyond that the fp32 FMA kernel on an fp32 P
-//   3. simplex_gather_kernel rows (i,j,k,*) of the 4-simplex are runs of row (i,j), columns
-//                            (k,k)..(k,d-1) of that triangle: contiguous on both sides
+//   3. simplex_gather_kernel all entries (i,j,*,*) of the 4-simplex are one run of row (i,j) of that triangle,
+//                            from column (j,j) on: contiguous on both sides
 // Step 2 works on the symmetric pair-by-pair matrix, whose unique set (pairs p <= q) is about
 // three times larger than the set of unique 4-tuples: the entries with j > k are computed and
 // not gathered.
@@ -108,9 +108,10 @@ pair_expand_kernel(const float *__restrict__ X, int64_t N, int d, int64_t ldx, O
     for (int64_t row0 = (int64_t)blockIdx.y * EXP_ROWS; row0 < rows_total; row0 += (int64_t)gridDim.y * EXP_ROWS) {
         const int nrows = rows_total - row0 < EXP_ROWS ? (int)(rows_total - row0) : EXP_ROWS;
         __syncthreads();
-        for (int e = threadIdx.x; e < nrows * pitch; e += EXP_THREADS) {
-            const int r = e / pitch, c = e - r * pitch;
-            xs[e] = (c < d && (!SPLIT || row0 + r < N)) ? X[(row0 + r) * ldx + c] : 0.f;
+        for (int r = threadIdx.x >> 5; r < nrows; r += EXP_THREADS / 32) {
+            const float *xr = X + (row0 + r) * ldx;
+            const bool row_in = !SPLIT || row0 + r < N;
+            for (int c = threadIdx.x & 31; c < pitch; c += 32) xs[r * pitch + c] = (c < d && row_in) ? xr[c] : 0.f;
         }
         __syncthreads();
         if (!inside) continue;
@@ -129,9 +130,10 @@ pair_expand_kernel(const float *__restrict__ X, int64_t N, int d, int64_t ldx, O
     }
 }
 
-// One block per row (i,j,k) of the 4-simplex: out[s(i,j,k,l)], l = k..d-1, is the run of row (i,j),
-// columns (k,k)..(k,d-1) of the packed pair-by-pair triangle.
-__global__ void __launch_bounds__(64)
+// One block per unique pair (i,j): the entries (i,j,k,l), j <= k <= l, follow each other in the 4-simplex in the
+// order of the pairs (k,l), and in row (i,j) of the packed pair-by-pair triangle they are the columns from pair
+// (j,j) to the last one: one contiguous run on both sides, of d-j + ... + 1 elements.
+__global__ void __launch_bounds__(128)
 simplex_gather_kernel(const float *__restrict__ M2, float *__restrict__ out, int d, int64_t dP, unsigned *status,
                       const unsigned *inner_status)
 {
@@ -140,12 +142,14 @@ simplex_gather_kernel(const float *__restrict__ M2, float *__restrict__ out, int
         status[kWsStatusWord] = inner_status[kWsStatusWord];
         status[kWsDetailWord] = inner_status[kWsDetailWord];
     }
-    int64_t i, j, k;
-    tet_decode(d, blockIdx.x, i, j, k);
-    const int64_t p = tri_encode(d, i, j), q = tri_encode(d, k, k);       // p <= q because j <= k
-    const float *src = M2 + tri_encode(dP, p, q);
-    float *dst = out + simp4_encode(d, i, j, k, k);
-    for (int o = threadIdx.x; o < d - k; o += 64) dst[o] = src[o];
+    const int64_t p = blockIdx.x;
+    int64_t i, j;
+    tri_decode(d, p, i, j);
+    const int64_t q0 = tri_encode(d, j, j);                               // p <= q0 because i <= j
+    const int len = (int)(tri_rows(d) - q0);
+    const float *src = M2 + tri_encode(dP, p, q0);
+    float *dst = out + simp4_encode(d, i, j, j, j);
+    for (int o = threadIdx.x; o < len; o += 128) dst[o] = src[o];
 }
 
 }  // namespace m4
@@ -195,7 +199,7 @@ extern "C" st_status st_sym_moment4(const float *X, int64_t N, int64_t d, int64_
                                  : st_sym_moment2(w + p.off_p, p.bf16 ? ST_BF16 : ST_F32, N, p.dP, p.dP, M2, w + p.off_ws,
                                                   (size_t)p.m2_ws, 0, stream_);
     if (rc != ST_OK) return rc;
-    simplex_gather_kernel<<<(unsigned)tet_rows(d), 64, 0, stream>>>(M2, out_packed, (int)d, p.dP, (unsigned *)w,
-                                                                    (const unsigned *)(w + p.off_ws));
+    simplex_gather_kernel<<<(unsigned)npairs, 128, 0, stream>>>(M2, out_packed, (int)d, p.dP, (unsigned *)w,
+                                                                (const unsigned *)(w + p.off_ws));
     return launch_status();
 }
