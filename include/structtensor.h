@@ -302,6 +302,17 @@ const char *st_status_string(st_status s);
 /* Version of the ABI described in this header. */
 int st_abi_version(void);
 
+/* 1 in the debug build of the library (compiled with -DST_BOUNDS_CHECK: every store whose index comes out of the
+ * packed-index arithmetic is range-checked on the device, a violation is recorded and the store skipped, and
+ * st_check_status -- with or without a workspace -- then returns ST_ERR_DEV_BOUNDS once); 0 in the normal build.
+ * The paper has no counterpart. */
+int st_bounds_checked_build(void);
+
+/* Debug build only (else ST_ERR_UNSUPPORTED): launches a kernel that hands the range check an index that is out
+ * of range by construction -- the check records it and nothing is loaded or stored -- so that the reporting path
+ * can be tested: the next st_check_status returns ST_ERR_DEV_BOUNDS, the one after it ST_OK. */
+st_status st_bounds_self_test(void *stream);
+
 #ifdef __cplusplus
 }
 #endif

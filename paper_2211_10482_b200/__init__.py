@@ -15,7 +15,9 @@ from dataclasses import dataclass
 import torch
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libstructtensor.so")
+# STRUCTTENSOR_LIB selects another build of the library, e.g. the range-checking debug build
+# libstructtensor_check.so (python -m paper_2211_10482_b200._build --check)
+LIB_PATH = os.environ.get("STRUCTTENSOR_LIB") or os.path.join(_HERE, "libstructtensor.so")
 
 # st_status
 ST_OK, ST_ERR_NULL, ST_ERR_SHAPE, ST_ERR_ALIGN, ST_ERR_DTYPE, ST_ERR_WORKSPACE, ST_ERR_UNSUPPORTED, \
@@ -40,7 +42,7 @@ EXPORTS = [
     "st_packed_elems", "st_dense_elems", "st_pack", "st_unpack", "st_workspace_bytes", "st_sym_moment2",
     "st_sym_moment3", "st_sym_moment3_static", "st_sym_moment4", "st_mttkrp_tri", "st_mttkrp_slice", "st_ttm_blockdiag", "st_ttm_packed",
     "st_thp", "st_packed_axpby", "st_packed_mul", "st_check_status", "st_status_string",
-    "st_abi_version",
+    "st_abi_version", "st_bounds_checked_build", "st_bounds_self_test",
 ]
 
 
@@ -92,6 +94,7 @@ def lib() -> ctypes.CDLL:
         L.st_unpack.argtypes = [LP, ci, vp, vp, ci, vp]
         L.st_workspace_bytes.argtypes = [ci, i64, i64, i64, i64, cu]
         L.st_workspace_bytes.restype = sz
+        L.st_bounds_self_test.argtypes = [vp]
         L.st_sym_moment2.argtypes = [vp, ci, i64, i64, i64, vp, vp, sz, cu, vp]
         L.st_sym_moment3.argtypes = [vp, i64, i64, i64, vp, vp, sz, cu, vp]
         L.st_sym_moment3_static.argtypes = [vp, i64, i64, i64, vp, cu, vp]

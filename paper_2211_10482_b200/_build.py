@@ -12,6 +12,10 @@ CSRC = os.path.join(HERE, "csrc")
 INCLUDE = os.path.join(ROOT, "include")
 OBJDIR = os.path.join(HERE, "_build")
 LIB = os.path.join(HERE, "libstructtensor.so")
+# debug build with device-side range checks (-DST_BOUNDS_CHECK; relocatable device code for its one device-wide word)
+OBJDIR_CHECK = os.path.join(HERE, "_build_check")
+LIB_CHECK = os.path.join(HERE, "libstructtensor_check.so")
+CHECK_FLAGS = ["-DST_BOUNDS_CHECK", "-rdc=true"]
 
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
@@ -32,12 +36,12 @@ def _deps_mtime():
     return m
 
 
-def _compile(src: str, verbose: bool) -> str:
-    obj = os.path.join(OBJDIR, src[:-3] + ".o")
+def _compile(src: str, verbose: bool, check: bool = False) -> str:
+    obj = os.path.join(OBJDIR_CHECK if check else OBJDIR, src[:-3] + ".o")
     spath = os.path.join(CSRC, src)
     if os.path.exists(obj) and os.path.getmtime(obj) >= max(os.path.getmtime(spath), _deps_mtime()):
         return obj
-    cmd = ["nvcc", *NVCC_FLAGS, "-c", spath, "-o", obj]
+    cmd = ["nvcc", *NVCC_FLAGS, *(CHECK_FLAGS if check else []), "-c", spath, "-o", obj]
     if verbose:
         cmd.insert(1, "-Xptxas=-v")
     res = subprocess.run(cmd, capture_output=True, text=True)
@@ -48,25 +52,26 @@ def _compile(src: str, verbose: bool) -> str:
     return obj
 
 
-def build(force: bool = False, verbose: bool = False) -> str:
-    """Compiles every .cu under csrc/ and links the shared library."""
-    os.makedirs(OBJDIR, exist_ok=True)
+def build(force: bool = False, verbose: bool = False, check: bool = False) -> str:
+    """Compiles every .cu under csrc/ and links the shared library (check=True: the range-checking debug build)."""
+    objdir, lib = (OBJDIR_CHECK, LIB_CHECK) if check else (OBJDIR, LIB)
+    os.makedirs(objdir, exist_ok=True)
     if force:
-        for f in os.listdir(OBJDIR):
+        for f in os.listdir(objdir):
             if f.endswith(".o"):
-                os.remove(os.path.join(OBJDIR, f))
+                os.remove(os.path.join(objdir, f))
     srcs = _sources()
     with concurrent.futures.ThreadPoolExecutor(max_workers=min(8, len(srcs))) as ex:
-        objs = list(ex.map(lambda s: _compile(s, verbose), srcs))
-    if force or not os.path.exists(LIB) or any(os.path.getmtime(o) > os.path.getmtime(LIB) for o in objs):
-        tmp = LIB + ".%d.tmp" % os.getpid()
-        cmd = ["nvcc", "-shared", "-gencode", "arch=compute_100a,code=sm_100a", "-o", tmp, *objs]
+        objs = list(ex.map(lambda s: _compile(s, verbose, check), srcs))
+    if force or not os.path.exists(lib) or any(os.path.getmtime(o) > os.path.getmtime(lib) for o in objs):
+        tmp = lib + ".%d.tmp" % os.getpid()
+        cmd = ["nvcc", "-shared", "-gencode", "arch=compute_100a,code=sm_100a", *(["-rdc=true"] if check else []), "-o", tmp, *objs]
         res = subprocess.run(cmd, capture_output=True, text=True)
         if res.returncode != 0:
             raise RuntimeError("link failed:\n%s\n%s" % (res.stdout, res.stderr))
-        os.replace(tmp, LIB)
-    return LIB
+        os.replace(tmp, lib)
+    return lib
 
 
 if __name__ == "__main__":
-    print(build(force="--force" in sys.argv, verbose="-v" in sys.argv))
+    print(build(force="--force" in sys.argv, verbose="-v" in sys.argv, check="--check" in sys.argv))

@@ -10,6 +10,17 @@ size_t ttm_split_workspace(int64_t rows, int64_t K, int64_t R);
 size_t mttkrp_workspace(int64_t rows, int64_t I, int64_t K, int64_t R, unsigned flags);
 }  // namespace st
 
+#ifdef ST_BOUNDS_CHECK
+namespace st {
+__device__ unsigned g_st_bounds[2] = {0u, 0u};
+// runs the range check on an index that is out of range by construction; nothing is loaded or stored
+__global__ void bounds_self_test_kernel()
+{
+    if (threadIdx.x == 0 && ST_BOUNDS_OK(5, 3, 99)) g_st_bounds[1] = 0xFFFFFFFFu;   // not reached
+}
+}
+#endif
+
 extern "C" {
 
 size_t st_workspace_bytes(st_op op, int64_t a, int64_t b, int64_t c, int64_t e, unsigned flags)
@@ -45,6 +56,18 @@ size_t st_workspace_bytes(st_op op, int64_t a, int64_t b, int64_t c, int64_t e, 
 st_status st_check_status(const void *ws, void *stream)
 {
     if (cudaStreamSynchronize((cudaStream_t)stream) != cudaSuccess) return ST_ERR_CUDA;
+#ifdef ST_BOUNDS_CHECK
+    {
+        // the range checks of the debug build report here whichever call tripped them; reading clears the record
+        unsigned b[2] = {0, 0};
+        const unsigned zero[2] = {0, 0};
+        if (cudaMemcpyFromSymbol(b, st::g_st_bounds, sizeof(b)) != cudaSuccess) return ST_ERR_CUDA;
+        if (b[0] != 0) {
+            (void)cudaMemcpyToSymbol(st::g_st_bounds, zero, sizeof(zero));
+            return ST_ERR_DEV_BOUNDS;
+        }
+    }
+#endif
     if (!ws) return ST_OK;
     unsigned words[2] = {0, 0};
     if (cudaMemcpy(words, ws, sizeof(words), cudaMemcpyDeviceToHost) != cudaSuccess) return ST_ERR_CUDA;
@@ -72,5 +95,25 @@ const char *st_status_string(st_status s)
 }
 
 int st_abi_version(void) { return 1; }
+
+int st_bounds_checked_build(void)
+{
+#ifdef ST_BOUNDS_CHECK
+    return 1;
+#else
+    return 0;
+#endif
+}
+
+st_status st_bounds_self_test(void *stream)
+{
+#ifdef ST_BOUNDS_CHECK
+    st::bounds_self_test_kernel<<<1, 32, 0, (cudaStream_t)stream>>>();
+    return cudaGetLastError() == cudaSuccess ? ST_OK : ST_ERR_CUDA;
+#else
+    (void)stream;
+    return ST_ERR_UNSUPPORTED;
+#endif
+}
 
 }  // extern "C"

@@ -229,7 +229,7 @@ __global__ void __launch_bounds__(RG_THREADS, 1) rowgemm_kernel(const RgArgs a)
                 for (int off = CT; off < 32; off <<= 1)
 #pragma unroll
                     for (int c = 0; c < 8; ++c) w[c] += __shfl_xor_sync(0xffffffffu, w[c], off);
-                if (lane < CT) {
+                if (lane < CT && ST_BOUNDS_OK(unit + g, mttkrp_slots(a.rows, WR, a.I, 1), 5)) {
                     float *o = a.out + (unit + g) * R_ + 4 * tc;
                     *reinterpret_cast<float4 *>(o) = make_float4(w[0], w[1], w[2], w[3]);
                     *reinterpret_cast<float4 *>(o + R_ / 2) = make_float4(w[4], w[5], w[6], w[7]);
@@ -271,6 +271,7 @@ mttkrp_rowsum_kernel(const float *__restrict__ part, float *__restrict__ A, int6
         if (e > s) {
             const float *p = part + ((u0 + i) * ksplit) * R + r;
             const int64_t n = (u1 - u0 + 1) * ksplit;
+            if (!ST_BOUNDS_OK((u0 + i) * ksplit + n - 1, mttkrp_slots(m.rows, unit_rows, m.I, ksplit), 6)) continue;
             int64_t k = 0;
             for (; k + 8 <= n; k += 8) {               // eight independent loads in flight
                 float t[8];

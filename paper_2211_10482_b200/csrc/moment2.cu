@@ -190,7 +190,7 @@ moment2_f32_reduce_kernel(const float *__restrict__ partials, float *__restrict_
 #pragma unroll
             for (int u = 0; u < 32; ++u) s += v[u];
         }
-        out[tri_encode(d, gi, gj)] = s;
+        if (ST_BOUNDS_OK(tri_encode(d, gi, gj), tri_rows(d), 2)) out[tri_encode(d, gi, gj)] = s;
     }
 }
 

@@ -248,7 +248,8 @@ moment2_small_reduce_kernel(const float *__restrict__ partials, float *__restric
 #pragma unroll
         for (int u = 0; u < 32; ++u) s += v[u];
     }
-    out[tri_encode(d, ci < cj ? ci : cj, ci < cj ? cj : ci)] = s;
+    const int64_t at = tri_encode(d, ci < cj ? ci : cj, ci < cj ? cj : ci);
+    if (ST_BOUNDS_OK(at, tri_rows(d), 2)) out[at] = s;
 }
 
 struct M2SmallPlan {

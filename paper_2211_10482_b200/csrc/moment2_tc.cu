@@ -235,7 +235,7 @@ moment2_tc_reduce_kernel(const float *__restrict__ partials, float *__restrict__
 #pragma unroll
                 for (int u = 0; u < 8; ++u) s += v[u];
             }
-            out[tri_encode(d, gi, gj)] = s;
+            if (ST_BOUNDS_OK(tri_encode(d, gi, gj), tri_rows(d), 2)) out[tri_encode(d, gi, gj)] = s;
         }
     }
 }
@@ -472,7 +472,7 @@ moment2_tc_pair_reduce_kernel(const float *__restrict__ partials, float *__restr
 #pragma unroll
                 for (int u = 0; u < 8; ++u) s += v[u];
             }
-            out[tri_encode(d, gi, gj)] = s;
+            if (ST_BOUNDS_OK(tri_encode(d, gi, gj), tri_rows(d), 2)) out[tri_encode(d, gi, gj)] = s;
         }
     }
 }

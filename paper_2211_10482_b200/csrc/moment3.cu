@@ -246,8 +246,8 @@ moment3_kernel(const M3Args a, const __grid_constant__ M3Table<WARPS> tab)
             float lo, hi;
             unpack2(acc[r][c], lo, hi);
             const int k = 8 * tkb + 2 * c;
-            if (k >= j && k < d) mine[base + (k - j)] = lo;
-            if (k + 1 >= j && k + 1 < d) mine[base + (k + 1 - j)] = hi;
+            if (k >= j && k < d && ST_BOUNDS_OK(base + (k - j), out_elems, 3)) mine[base + (k - j)] = lo;
+            if (k + 1 >= j && k + 1 < d && ST_BOUNDS_OK(base + (k + 1 - j), out_elems, 3)) mine[base + (k + 1 - j)] = hi;
         }
     }
 }

@@ -249,8 +249,8 @@ moment3_tc_kernel(const __grid_constant__ Args a)
                     }
 #pragma unroll
                     for (int u = 0; u < 8; ++u) {
-                        if (lane < len[u]) mine[base[u] + lane] = v0[u];
-                        if (lane + 32 < len[u]) mine[base[u] + lane + 32] = v1[u];
+                        if (lane < len[u] && ST_BOUNDS_OK(base[u] + lane, a.out_elems, 4)) mine[base[u] + lane] = v0[u];
+                        if (lane + 32 < len[u] && ST_BOUNDS_OK(base[u] + lane + 32, a.out_elems, 4)) mine[base[u] + lane + 32] = v1[u];
                     }
                 }
                 __syncwarp();

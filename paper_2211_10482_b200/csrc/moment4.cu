@@ -149,6 +149,9 @@ simplex_gather_kernel(const float *__restrict__ M2, float *__restrict__ out, int
     const int len = (int)(tri_rows(d) - q0);
     const float *src = M2 + tri_encode(dP, p, q0);
     float *dst = out + simp4_encode(d, i, j, j, j);
+    if (!(ST_BOUNDS_OK(tri_encode(dP, p, q0) + len - 1, tri_rows(dP), 7) &&
+          ST_BOUNDS_OK(simp4_encode(d, i, j, j, j) + len - 1, simp4_rows(d), 7)))
+        return;
     for (int o = threadIdx.x; o < len; o += 128) dst[o] = src[o];
 }
 

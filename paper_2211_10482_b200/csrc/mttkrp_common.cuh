@@ -88,15 +88,17 @@ __device__ __forceinline__ WarpRuns warp_runs(bool valid, int gi32, int lane)
 
 // Writes the sums of the warp's runs for the 32 columns c0.. held in v (v[c] = C[j,c0+c] * Y[fibre,c0+c],
 // zeros in lanes without a fibre) to the partial slots (unit + i).  Call with all 32 lanes.
+// nslots: number of partial slots behind `part` (read by the range checks of the debug build only).
 __device__ __forceinline__ void warp_store_runs(float (&v)[32], const WarpRuns &w, bool valid, int gi32, int64_t unit,
-                                                int lane, float *part, int R, int c0)
+                                                int lane, float *part, int R, int c0, int64_t nslots)
 {
     if (w.heads == 0u) return;                 // no fibre in this warp
     if (w.heads == 1u) {                       // one run: the whole warp
         const float sum = warp_transpose_sum32(v, lane);
-        part[(unit + __shfl_sync(0xffffffffu, gi32, 0)) * R + c0 + lane] = sum;
+        const int64_t slot = unit + __shfl_sync(0xffffffffu, gi32, 0);
+        if (ST_BOUNDS_OK(slot, nslots, 5)) part[slot * R + c0 + lane] = sum;
     } else if (w.heads == w.vmask) {           // every fibre is a run of its own
-        if (valid) {
+        if (valid && ST_BOUNDS_OK(unit + gi32, nslots, 5)) {
             float4 *dst = reinterpret_cast<float4 *>(part + (unit + gi32) * R + c0);
 #pragma unroll
             for (int e = 0; e < 8; ++e) dst[e] = make_float4(v[4 * e], v[4 * e + 1], v[4 * e + 2], v[4 * e + 3]);
@@ -112,22 +114,23 @@ __device__ __forceinline__ void warp_store_runs(float (&v)[32], const WarpRuns &
 #pragma unroll
             for (int e = 0; e < 32; ++e) t[e] = in ? v[e] : 0.f;
             const float sum = warp_transpose_sum32(t, lane);
-            part[(unit + __shfl_sync(0xffffffffu, gi32, s0)) * R + c0 + lane] = sum;
+            const int64_t slot = unit + __shfl_sync(0xffffffffu, gi32, s0);
+            if (ST_BOUNDS_OK(slot, nslots, 5)) part[slot * R + c0 + lane] = sum;
         }
     }
 }
 
 // The same for the 16 columns c0.. held in v.
 __device__ __forceinline__ void warp_store_runs16(float (&v)[16], const WarpRuns &w, bool valid, int gi32, int64_t unit,
-                                                  int lane, float *part, int R, int c0)
+                                                  int lane, float *part, int R, int c0, int64_t nslots)
 {
     if (w.heads == 0u) return;
     if (w.heads == 1u) {
         const float sum = warp_transpose_sum16(v, lane);
         const int gi0 = __shfl_sync(0xffffffffu, gi32, 0);
-        if (lane < 16) part[(unit + gi0) * R + c0 + lane] = sum;
+        if (lane < 16 && ST_BOUNDS_OK(unit + gi0, nslots, 5)) part[(unit + gi0) * R + c0 + lane] = sum;
     } else if (w.heads == w.vmask) {
-        if (valid) {
+        if (valid && ST_BOUNDS_OK(unit + gi32, nslots, 5)) {
             float4 *dst = reinterpret_cast<float4 *>(part + (unit + gi32) * R + c0);
 #pragma unroll
             for (int e = 0; e < 4; ++e) dst[e] = make_float4(v[4 * e], v[4 * e + 1], v[4 * e + 2], v[4 * e + 3]);
@@ -144,7 +147,7 @@ __device__ __forceinline__ void warp_store_runs16(float (&v)[16], const WarpRuns
             for (int e = 0; e < 16; ++e) t[e] = in ? v[e] : 0.f;
             const float sum = warp_transpose_sum16(t, lane);
             const int gis = __shfl_sync(0xffffffffu, gi32, s0);
-            if (lane < 16) part[(unit + gis) * R + c0 + lane] = sum;
+            if (lane < 16 && ST_BOUNDS_OK(unit + gis, nslots, 5)) part[(unit + gis) * R + c0 + lane] = sum;
         }
     }
 }

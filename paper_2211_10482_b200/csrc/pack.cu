@@ -158,6 +158,7 @@ structured_copy_kernel(const U *__restrict__ src, U *__restrict__ dst, LayoutArg
     for (int64_t row = tid >> group_shift; row < rows; row += groups) {
         const int64_t srow = PACK ? dense_row_of_packed<KIND>(a, row) : packed_row_of_dense<KIND>(a, row);
         U *out = dst + row * a.chunks;
+        if (srow >= 0 && !ST_BOUNDS_OK(srow, PACK ? a.dense_rows : a.packed_rows, 1)) continue;
         if (srow >= 0) {
             const U *in = src + srow * a.chunks;
             for (int64_t c = lane; c < a.chunks; c += g) out[c] = in[c];
@@ -240,6 +241,10 @@ slice_copy_kernel(const U *__restrict__ src, U *__restrict__ dst, LayoutArgs a, 
         const int64_t part = item - s * parts;
         int64_t lo, hi, prow;
         slice_run<KIND>(a, s, lo, hi, prow);
+        // a non-empty run lies inside the slice and inside the packed array
+        if (hi > lo && !(ST_BOUNDS_OK(lo, a.d, 1) && ST_BOUNDS_OK(hi - 1, a.d, 1) && ST_BOUNDS_OK(prow, a.packed_rows, 1) &&
+                         ST_BOUNDS_OK(prow + (hi - lo) - 1, a.packed_rows, 1)))
+            continue;
         const int64_t c0 = lo * a.chunks, c1 = hi * a.chunks;  // units of the run inside the slice
         // pack splits the run itself into parts, unpack the whole dense slice (it writes all of it)
         const int64_t r0 = PACK ? c0 : 0, r1 = PACK ? c1 : su;

@@ -17,6 +17,25 @@ constexpr int kWsStatusWord = 0;
 constexpr int kWsDetailWord = 1;
 constexpr int kWsTicketWord = 8;
 
+// Debug build (-DST_BOUNDS_CHECK, relocatable device code): every store whose index comes out of packed-index
+// arithmetic is range-checked first; a violation records the site in a device-wide word, the store is skipped
+// and st_check_status reports ST_ERR_DEV_BOUNDS.  In the normal build the macro is the constant true.
+#ifdef ST_BOUNDS_CHECK
+extern __device__ unsigned g_st_bounds[2];          // [0] = number of violations, [1] = site of the last one
+__device__ __forceinline__ bool st_bounds_ok(long long idx, long long n, unsigned site)
+{
+    if (idx >= 0 && idx < n) return true;
+    atomicAdd(&g_st_bounds[0], 1u);
+    g_st_bounds[1] = site;
+    return false;
+}
+#define ST_BOUNDS_OK(idx, n, site) ::st::st_bounds_ok((long long)(idx), (long long)(n), (site))
+#else
+#define ST_BOUNDS_OK(idx, n, site) true
+#endif
+// sites: 1 pack/unpack copy, 2 second-moment reductions, 3 third-moment partial sums, 4 tensor-core third moment,
+// 5 MTTKRP partial slots, 6 MTTKRP row sums, 7 fourth-moment gather, 8 TTM rows
+
 inline bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 inline bool aligned256(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 255u) == 0; }
 inline size_t round_up(size_t x, size_t a) { return (x + a - 1) / a * a; }

@@ -266,7 +266,8 @@ __global__ void __launch_bounds__(split::THREADS, 1) ttm_split_kernel(const Spli
                         v[4 * e + 2] *= cv[e].z;
                         v[4 * e + 3] *= cv[e].w;
                     }
-                    warp_store_runs16(v, runs, valid, (int)gi, tile * (BM / 32) + q, lane, a.out, R, c0);
+                    warp_store_runs16(v, runs, valid, (int)gi, tile * (BM / 32) + q, lane, a.out, R, c0,
+                                      mttkrp_slots(a.rows, 32, a.I, 1));
                 }
             };
             if (pre) {

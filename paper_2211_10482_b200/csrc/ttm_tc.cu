@@ -253,7 +253,7 @@ ttm_tc_kernel(const __grid_constant__ CUtensorMap tmap, const TtmTcArgs a)
 #pragma unroll
                         for (int e = 0; e < 32; ++e) v[e] = 0.f;
                     }
-                    warp_store_runs(v, runs, valid, gi32, unit, lane, a.out, a.R, c0);
+                    warp_store_runs(v, runs, valid, gi32, unit, lane, a.out, a.R, c0, mttkrp_slots(a.rows, 32, a.I, 1));
                 }
             }
             tc_fence_before();
