@@ -19,6 +19,7 @@
 #include "st_common.cuh"
 #include "st_index.cuh"
 #include <cuda_bf16.h>
+#include <type_traits>
 
 namespace st {
 
@@ -83,12 +84,13 @@ __device__ __forceinline__ void store4(__nv_bfloat16 *dst, float a, float b, flo
 // row with one 8- or 16-byte store.  HBM bound: the write of P.
 // SPLIT: every product p is written twice, hi = bf16(p) in row n and lo = bf16(p - hi) in row Np + n; the rows
 // N .. Np-1 of either part are zero.
-template <typename OutT, bool SPLIT>
+// COLS: columns of a staged row per lane, (d + 1 + 31) / 32 rounded up to an instance (2, 3 or 5).
+template <typename OutT, bool SPLIT, int COLS>
 __global__ void __launch_bounds__(EXP_THREADS)
 pair_expand_kernel(const float *__restrict__ X, int64_t N, int d, int64_t ldx, OutT *__restrict__ P, int dP, int npairs,
                    int64_t Np)
 {
-    extern __shared__ __align__(16) float xs[];                       // [EXP_ROWS][d + 1], column d is zero
+    extern __shared__ __align__(16) float xs[];                       // 2 x [EXP_ROWS][d + 1], column d is zero
     const int pitch = d + 1;
     // gridDim.x = column groups, gridDim.y = row groups
     const int p = (blockIdx.x * EXP_THREADS + threadIdx.x) * 4;       // this thread's columns p .. p+3
@@ -105,18 +107,48 @@ pair_expand_kernel(const float *__restrict__ X, int64_t N, int d, int64_t ldx, O
     }
     const bool inside = p < dP;
     const int64_t rows_total = SPLIT ? Np : N;
-    for (int64_t row0 = (int64_t)blockIdx.y * EXP_ROWS; row0 < rows_total; row0 += (int64_t)gridDim.y * EXP_ROWS) {
-        const int nrows = rows_total - row0 < EXP_ROWS ? (int)(rows_total - row0) : EXP_ROWS;
-        __syncthreads();
-        for (int r = threadIdx.x >> 5; r < nrows; r += EXP_THREADS / 32) {
-            const float *xr = X + (row0 + r) * ldx;
-            const bool row_in = !SPLIT || row0 + r < N;
-            for (int c = threadIdx.x & 31; c < pitch; c += 32) xs[r * pitch + c] = (c < d && row_in) ? xr[c] : 0.f;
+    // Two stage buffers: the rows of the next pass travel from global memory into registers while the current ones are
+    // multiplied, and one block barrier per pass is enough (a buffer is rewritten two passes later, after every
+    // thread has gone through the barrier of the pass in between).
+    constexpr int NW = EXP_THREADS / 32, RPW = (EXP_ROWS + NW - 1) / NW;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    float reg[RPW][COLS];
+    auto gload = [&](int64_t row0) {
+#pragma unroll
+        for (int q = 0; q < RPW; ++q) {
+            const int64_t n = row0 + warp + q * NW;
+            const bool row_in = warp + q * NW < EXP_ROWS && n < N;
+#pragma unroll
+            for (int c = 0; c < COLS; ++c) {
+                const int col = lane + 32 * c;
+                reg[q][c] = (row_in && col < d) ? X[n * ldx + col] : 0.f;
+            }
         }
+    };
+    auto sstore = [&](float *buf) {
+#pragma unroll
+        for (int q = 0; q < RPW; ++q) {
+            const int r = warp + q * NW;
+#pragma unroll
+            for (int c = 0; c < COLS; ++c) {
+                const int col = lane + 32 * c;
+                if (r < EXP_ROWS && col < pitch) buf[r * pitch + col] = reg[q][c];
+            }
+        }
+    };
+    const int64_t step = (int64_t)gridDim.y * EXP_ROWS;
+    int64_t row0 = (int64_t)blockIdx.y * EXP_ROWS;
+    if (row0 < rows_total) gload(row0);
+    int buf = 0;
+    for (; row0 < rows_total; row0 += step, buf ^= 1) {
+        const int nrows = rows_total - row0 < EXP_ROWS ? (int)(rows_total - row0) : EXP_ROWS;
+        float *xb = xs + buf * (EXP_ROWS * pitch);
+        sstore(xb);
         __syncthreads();
+        if (row0 + step < rows_total) gload(row0 + step);
         if (!inside) continue;
         OutT *dst = P + row0 * dP + p;
-        const float *x = xs;
+        const float *x = xb;
 #pragma unroll 4
         for (int r = 0; r < nrows; ++r, dst += dP, x += pitch) {
             const float v0 = x[ci[0]] * x[cj[0]], v1 = x[ci[1]] * x[cj[1]], v2 = x[ci[2]] * x[cj[2]], v3 = x[ci[3]] * x[cj[3]];
@@ -183,20 +215,25 @@ extern "C" st_status st_sym_moment4(const float *X, int64_t N, int64_t d, int64_
     unsigned char *w = (unsigned char *)ws;
     float *M2 = (float *)(w + p.off_m2);
     const int npairs = (int)tri_rows(d);
-    const size_t smem = (size_t)EXP_ROWS * (d + 1) * sizeof(float);
+    const size_t smem = (size_t)2 * EXP_ROWS * (d + 1) * sizeof(float);
     const unsigned col_groups = (unsigned)((p.dP + 4 * EXP_THREADS - 1) / (4 * EXP_THREADS));
     const int64_t passes = ((p.split ? p.Np : N) + EXP_ROWS - 1) / EXP_ROWS;
     const int64_t cap = ((int64_t)sm_count_or_default() * 8 + col_groups - 1) / col_groups;
     const dim3 grid(col_groups, (unsigned)(passes < cap ? passes : cap));
-    if (p.split)
-        pair_expand_kernel<__nv_bfloat16, true><<<grid, EXP_THREADS, smem, stream>>>(
-            X, N, (int)d, ldx, (__nv_bfloat16 *)(w + p.off_p), (int)p.dP, npairs, p.Np);
-    else if (p.bf16)
-        pair_expand_kernel<__nv_bfloat16, false><<<grid, EXP_THREADS, smem, stream>>>(
-            X, N, (int)d, ldx, (__nv_bfloat16 *)(w + p.off_p), (int)p.dP, npairs, p.Np);
-    else
-        pair_expand_kernel<float, false><<<grid, EXP_THREADS, smem, stream>>>(X, N, (int)d, ldx, (float *)(w + p.off_p),
-                                                                               (int)p.dP, npairs, p.Np);
+    auto expand = [&](auto tag, auto split_tag) {
+        using T = decltype(tag);
+        constexpr bool SP = decltype(split_tag)::value;
+        T *dst = (T *)(w + p.off_p);
+        if (d + 1 <= 64)
+            pair_expand_kernel<T, SP, 2><<<grid, EXP_THREADS, smem, stream>>>(X, N, (int)d, ldx, dst, (int)p.dP, npairs, p.Np);
+        else if (d + 1 <= 96)
+            pair_expand_kernel<T, SP, 3><<<grid, EXP_THREADS, smem, stream>>>(X, N, (int)d, ldx, dst, (int)p.dP, npairs, p.Np);
+        else
+            pair_expand_kernel<T, SP, 5><<<grid, EXP_THREADS, smem, stream>>>(X, N, (int)d, ldx, dst, (int)p.dP, npairs, p.Np);
+    };
+    if (p.split) expand(__nv_bfloat16(), std::true_type());
+    else if (p.bf16) expand(__nv_bfloat16(), std::false_type());
+    else expand(float(), std::false_type());
     if (cudaGetLastError() != cudaSuccess) return ST_ERR_CUDA;
     const st_status rc = p.split ? moment2_split_tc_parts(w + p.off_p, N, p.dP, M2, w + p.off_ws, (size_t)p.m2_ws, stream)
                                  : st_sym_moment2(w + p.off_p, p.bf16 ? ST_BF16 : ST_F32, N, p.dP, p.dP, M2, w + p.off_ws,
