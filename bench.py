@@ -102,6 +102,9 @@ def call_table(cfg):
     t["sym_moment3"] = dict(m3, bound="alu", launches=2)
     t["sym_moment3_tf32"] = dict(m3, bound="tensor", launches=2, tensor_scale=TF32_OVER_BF16)
     t["sym_moment3_bf16"] = dict(m3, bound="tensor", launches=2, tensor_scale=1.0)
+    dw = cfg["moment3_wide_d"]         # the third moment beyond the 64 features of the named configuration
+    t["sym_moment3_d%d" % dw] = dict(flops=2 * c2["N"] * tet(dw) + c2["N"] * tri(dw), bytes=4 * (c2["N"] * dw + tet(dw)),
+                                     bound="alu", launches=2)
     for d4 in cfg["moment4_d"]:
         m4 = dict(flops=2 * c2["N"] * simp4(d4) + c2["N"] * tri(d4), bytes=4 * (c2["N"] * d4 + simp4(d4)))
         t["sym_moment4_d%d" % d4] = dict(m4, bound="tensor", launches=4, tensor_scale=1.0 / 3.0)   # split pair features, three products
@@ -222,6 +225,7 @@ class ClockSampler:
 def bench_config():
     cfg = {k: dict(v) for k, v in workloads.CONFIGS.items()}
     cfg["band"] = dict(d=2048, kl=512, ku=511, inner=16)
+    cfg["moment3_wide_d"] = 128
     cfg["moment4_d"] = (32, 64)       # the fourth moment runs on the first d features of the third moment's samples
     return cfg
 
@@ -232,7 +236,7 @@ def bench_config():
 STEP_CALLS = ["sym_moment2_large", "pack_tri_x_k", "unpack_tri_sym_large", "ttm_blockdiag_tf32", "pack_band",
               "unpack_blockdiag", "mttkrp_tri_split", "sym_moment3", "sym_moment2", "unpack_tet_sym", "unpack_tri_sym"]
 # Timed on their own only (variants and widened rows)
-EXTRA_CALLS = ["mttkrp_tri", "mttkrp_tri_tf32", "ttm_blockdiag", "ttm_blockdiag_split", "sym_moment3_tf32", "sym_moment3_bf16", "sym_moment4_d32",
+EXTRA_CALLS = ["mttkrp_tri", "mttkrp_tri_tf32", "ttm_blockdiag", "ttm_blockdiag_split", "sym_moment3_tf32", "sym_moment3_bf16", "sym_moment3_d128", "sym_moment4_d32",
                "sym_moment4_d32_bf16", "sym_moment4_d64", "sym_moment4_d64_bf16", "thp_tri_x_k", "sym_moment2_large_f32",
                "sym_moment2_large_f32_tf32", "sym_moment2_large_f32_split"]
 
@@ -293,7 +297,8 @@ class Workload:
                       st.st_workspace_bytes(st.ST_OP_MTTKRP_TRI, c3["I"], c3["K"], c3["R"], 0, 0),
                       st.st_workspace_bytes(st.ST_OP_TTM_BLOCKDIAG, c4["nb"], c4["bs"], c4["K"], c4["R"], 0),
                       st.st_workspace_bytes(st.ST_OP_TTM_BLOCKDIAG, c4["nb"], c4["bs"], c4["K"], c4["R"], SP),
-                      st.st_workspace_bytes(st.ST_OP_SYM_MOMENT2, c5["N"], c5["d"], st.ST_F32)]
+                      st.st_workspace_bytes(st.ST_OP_SYM_MOMENT2, c5["N"], c5["d"], st.ST_F32),
+                      st.st_workspace_bytes(st.ST_OP_SYM_MOMENT3, c2["N"], cfg["moment3_wide_d"])]
             for d4 in cfg["moment4_d"]:
                 sizes += [st.st_workspace_bytes(st.ST_OP_SYM_MOMENT4, c2["N"], d4, 0, 0, 0),
                           st.st_workspace_bytes(st.ST_OP_SYM_MOMENT4, c2["N"], d4, 0, 0, BF)]
@@ -335,6 +340,10 @@ class Workload:
         f32 = dict(dtype=torch.float32, device=self.device)
         if self._extra is None:
             self._extra = {"thp3": torch.empty_like(o["Bp3"]), "m3_tc": torch.empty_like(o["m3"])}
+            dw = c["moment3_wide_d"]
+            gen = torch.Generator(device=self.device).manual_seed(workloads.SEEDS["moment3"] + dw)
+            self._extra["X3w"] = torch.randn((c["moment3"]["N"], dw), generator=gen, **f32)
+            self._extra["m3w"] = torch.empty(tet(dw), **f32)
             for d4 in c["moment4_d"]:
                 self._extra["X4_%d" % d4] = d["X2"][:, :d4].contiguous()
                 self._extra["m4_%d" % d4] = torch.empty(simp4(d4), **f32)
@@ -348,6 +357,7 @@ class Workload:
             "sym_moment3_tf32": lambda: st.st_sym_moment3(d["X2"], out=x["m3_tc"], ws=ws, flags=st.ST_FLAG_TC_TF32),
             "sym_moment3_bf16": lambda: st.st_sym_moment3(d["X2"], out=x["m3_tc"], ws=ws, flags=st.ST_FLAG_TC_BF16),
             "thp_tri_x_k": lambda: st.st_thp(o["Bp3"], d["B3"], self.lay3, out=x["thp3"]),
+            "sym_moment3_d%d" % c["moment3_wide_d"]: lambda: st.st_sym_moment3(x["X3w"], out=x["m3w"], ws=ws),
         }
         for d4 in c["moment4_d"]:
             calls["sym_moment4_d%d" % d4] = (lambda d4=d4: st.st_sym_moment4(x["X4_%d" % d4], out=x["m4_%d" % d4], ws=ws))
