@@ -8,8 +8,9 @@
 //   MTTKRP  m = p(i,j) runs over i<=j only; W = D; then A[i,r] += C[j,r] * Y[m,r], the
 //           product with C hoisted out of the k loop (Section 5.5, loop-invariant code motion).
 //
-// A warp owns a unit of consecutive fibres (32 for R = 64, 64 otherwise) and each of its threads keeps
-// 8 x 8 sums (fewer rows for R < 32) in registers.  That shape is set by what limits an fp32 FMA kernel that is
+// A warp owns a unit of consecutive fibres (32 for R >= 32, 64 below) and each of its threads keeps
+// 8 x 8 sums (4 x 8 for R = 32, where the finer units balance the SMs better than the larger tile pays; fewer
+// rows still below) in registers.  That shape is set by what limits an fp32 FMA kernel that is
 // fed from shared memory on this GPU: an SM can issue 128 FMAs but deliver only 32 words from shared memory to its
 // registers per cycle, broadcasts included (an inner-loop probe ran at 0.87 of the FMA peak on registers alone,
 // 0.73 with an 8 x 8 tile, 0.67 with 8 x 4), so a thread must not read more than 16 words per 64 FMAs.
@@ -309,9 +310,12 @@ st_status mttkrp_rowsum_launch(const float *part, float *A_full, int64_t I_full,
 // tile shape by R: {TM, stages}; a warp owns TM * 32 / (R/8) consecutive fibres, a tile is the block's 16 warps
 static void rowgemm_shape(int64_t R, int &tm, int &stages)
 {
-    if (R == 64) { tm = 8; stages = 6; }          // 512 fibres per tile, 36 KiB per stage
-    else if (R == 32) { tm = 8; stages = 3; }     // 1024 fibres per tile from here on, 66 KiB per stage
-    else { tm = (int)R / 4; stages = 3; }
+    // measured at the benchmark sizes: R = 64 runs 213 / 205 / 208 us with 6 / 4 / 3 stages; R = 32 runs 151 us with
+    // 8 fibres per thread (14 units of 64 fibres per SM: 3.5 per scheduler) and 136 us with 4 (28 units of 32), whatever
+    // the stage count from 2 to 6
+    if (R == 64) { tm = 8; stages = 4; }          // 512 fibres per tile, 36 KiB per stage
+    else if (R == 32) { tm = 4; stages = 4; }     // 512 fibres per tile, 34 KiB per stage
+    else { tm = (int)R / 4; stages = 3; }         // 1024 fibres per tile
 }
 static int64_t rowgemm_warp_rows(int64_t R)
 {
@@ -368,8 +372,8 @@ static st_status rowgemm_launch(const RgArgs &a0, cudaStream_t stream)
     switch (a.R) {
     case 8: return run(rowgemm_kernel<2, 1, 3, MODE>);
     case 16: return run(rowgemm_kernel<4, 2, 3, MODE>);
-    case 32: return run(rowgemm_kernel<8, 4, 3, MODE>);
-    case 64: return run(rowgemm_kernel<8, 8, 6, MODE>);
+    case 32: return run(rowgemm_kernel<4, 4, 4, MODE>);
+    case 64: return run(rowgemm_kernel<8, 8, 4, MODE>);
     default: return ST_ERR_UNSUPPORTED;
     }
 }
